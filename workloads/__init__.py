@@ -1,0 +1,363 @@
+"""Seeded synthetic inputs for the KV Prediction time-to-first-token path.
+
+This module only *describes* and *generates* inputs: model shapes, layer maps
+given as literal integer lists, random-init weights, token streams and prompt
+lengths.  It holds none of the method's arithmetic (no norm, no attention, no
+projection), so both the CPU oracle and the CUDA binding may import it without
+sharing any computation.
+
+Everything is a pure function of (config name, seed): weights come from a
+counter-based Philox stream keyed by (seed, tensor name), so any tensor can be
+regenerated alone, in any order, on any machine.
+
+The workloads stand in for the paper's OpenELM models and its TriviaQA /
+HumanEval prompts (Sec. 5, Sec. 6): same kind of shapes, prompt lengths and
+token-frequency structure, but random-init weights and synthetic token ids.
+"""
+from __future__ import annotations
+
+import hashlib
+from concurrent.futures import ThreadPoolExecutor
+from dataclasses import dataclass, field
+from typing import Dict, List, Optional, Sequence, Tuple
+
+import numpy as np
+
+PAGE_TOKENS = 64
+
+
+# ----------------------------------------------------------------------------
+# shapes
+# ----------------------------------------------------------------------------
+@dataclass(frozen=True)
+class LayerCfg:
+    n_q_heads: int
+    n_kv_heads: int
+    head_dim: int
+    ffn_dim: int
+
+    @property
+    def d_q(self) -> int:
+        return self.n_q_heads * self.head_dim
+
+    @property
+    def d_kv(self) -> int:
+        return self.n_kv_heads * self.head_dim
+
+
+@dataclass(frozen=True)
+class ModelCfg:
+    d_model: int
+    vocab: int
+    layers: Tuple[LayerCfg, ...]
+    rope_theta: float = 10000.0
+    rms_eps: float = 1e-6
+
+    @property
+    def n_layers(self) -> int:
+        return len(self.layers)
+
+
+@dataclass(frozen=True)
+class PairCfg:
+    """An (auxiliary, base, layer map) triple plus the run dtype."""
+    name: str
+    aux: ModelCfg
+    base: ModelCfg
+    layer_map: Tuple[int, ...]          # j_i for every base layer i (Sec. 4.2)
+    dtype: str = "bf16"                 # "bf16" | "f32"
+    predictor_bias: bool = False
+
+
+def uniform_model(n_layers, d_model, n_q, n_kv, head_dim, ffn, vocab) -> ModelCfg:
+    return ModelCfg(d_model=d_model, vocab=vocab,
+                    layers=tuple(LayerCfg(n_q, n_kv, head_dim, ffn) for _ in range(n_layers)))
+
+
+def layerwise_scaled_model(n_layers, d_model, q0, q1, head_dim, vocab,
+                           ffn_mult0=0.5, ffn_mult1=4.0) -> ModelCfg:
+    """Layer-wise scaling in the OpenELM spirit: head count and FFN width grow
+    linearly with the layer index.  This is this repository's own definition
+    (4 q heads per kv head, q heads rounded to a multiple of 4, FFN width to a
+    multiple of 128); it copies no published table."""
+    layers = []
+    for l in range(n_layers):
+        a = l / (n_layers - 1)
+        nq = 4 * int((q0 + (q1 - q0) * a) / 4 + 0.5)
+        nkv = nq // 4
+        ffn = 128 * int(d_model * (ffn_mult0 + (ffn_mult1 - ffn_mult0) * a) / 128 + 0.5)
+        layers.append(LayerCfg(nq, nkv, head_dim, ffn))
+    return ModelCfg(d_model=d_model, vocab=vocab, layers=tuple(layers))
+
+
+def _uniform_map(n_base: int, n_aux: int) -> Tuple[int, ...]:
+    return tuple((i * n_aux) // n_base for i in range(n_base))
+
+
+# Table 1 of the paper, row OE1.1B-KVP-C-270M (28 base layers <- 16 aux layers),
+# typed in as data: it is the "non-uniform layer map" of the layer-wise-scaled pair.
+_MAP_28_FROM_16 = (0, 0, 1, 1, 2, 2, 3, 3, 4, 4, 5, 5, 6, 6, 7, 7, 8, 8, 9, 9,
+                   10, 10, 11, 11, 12, 13, 14, 15)
+
+
+def pair(name: str) -> PairCfg:
+    """The five configurations of the benchmark plan plus small test pairs."""
+    if name == "c1":      # tiny fp32 pair
+        aux = uniform_model(2, 64, 4, 4, 16, 172, 512)
+        base = uniform_model(4, 128, 8, 4, 16, 344, 512)
+        return PairCfg("c1", aux, base, (0, 0, 1, 1), dtype="f32")
+    if name == "c1_bf16":
+        p = pair("c1")
+        return PairCfg("c1_bf16", p.aux, p.base, p.layer_map, dtype="bf16")
+    if name == "c2":      # 1.1B-shaped base, 270M-shaped aux
+        aux = uniform_model(16, 1280, 20, 5, 64, 3456, 32000)
+        base = uniform_model(28, 2048, 32, 8, 64, 5632, 32000)
+        return PairCfg("c2", aux, base, _uniform_map(28, 16))
+    if name in ("c3", "c5"):  # 3B-shaped base, 450M-shaped aux
+        aux = uniform_model(20, 1536, 12, 3, 128, 4096, 32000)
+        base = uniform_model(36, 3072, 24, 6, 128, 8192, 32000)
+        return PairCfg(name, aux, base, _uniform_map(36, 20))
+    if name == "c4":      # layer-wise scaled pair, non-uniform map
+        aux = layerwise_scaled_model(16, 1280, 8, 20, 64, 32000)
+        base = layerwise_scaled_model(28, 2048, 12, 32, 64, 32000)
+        return PairCfg("c4", aux, base, _MAP_28_FROM_16)
+    # ---- reduced pairs used by tests (several tiles, ragged tails, odd widths) ----
+    if name == "t_small":     # bf16, head_dim 64, GQA 4:1, non-multiple-of-128 widths
+        aux = uniform_model(3, 192, 4, 1, 64, 320, 1000)
+        base = uniform_model(5, 256, 8, 2, 64, 448, 1000)
+        return PairCfg("t_small", aux, base, (0, 0, 1, 1, 2))
+    if name == "t_small_f32":
+        p = pair("t_small")
+        return PairCfg("t_small_f32", p.aux, p.base, p.layer_map, dtype="f32")
+    if name == "t_hd128":     # head_dim 128 like the 3B pair, scaled down
+        aux = uniform_model(3, 384, 3, 1, 128, 1024, 2048)
+        base = uniform_model(4, 768, 6, 2, 128, 2048, 2048)
+        return PairCfg("t_hd128", aux, base, (0, 1, 1, 2))
+    if name == "t_scaled":    # heterogeneous layers like c4, scaled down
+        aux = layerwise_scaled_model(4, 256, 4, 8, 64, 1500, 0.5, 2.0)
+        base = layerwise_scaled_model(6, 384, 4, 12, 64, 1500, 0.5, 2.0)
+        return PairCfg("t_scaled", aux, base, (0, 0, 1, 1, 2, 3))
+    if name == "t_bias":      # predictor with bias terms
+        p = pair("t_small")
+        return PairCfg("t_bias", p.aux, p.base, p.layer_map, predictor_bias=True)
+    raise KeyError(name)
+
+
+def identity_pair(model: ModelCfg, dtype: str = "f32") -> PairCfg:
+    """aux == base, map j_i = i: used by the identity-predictor invariant."""
+    return PairCfg("identity", model, model, tuple(range(model.n_layers)), dtype=dtype)
+
+
+# ----------------------------------------------------------------------------
+# dtype helpers (input preparation only)
+# ----------------------------------------------------------------------------
+def round_to_bf16(x: np.ndarray) -> np.ndarray:
+    """Round fp32 values to the nearest bf16 (ties to even); result stays fp32."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    bias = ((u >> 16) & 1) + np.uint32(0x7FFF)
+    r = ((u + bias) & np.uint32(0xFFFF0000)).astype(np.uint32)
+    return r.view(np.float32)
+
+
+def bf16_bits(x: np.ndarray) -> np.ndarray:
+    """uint16 bit patterns of values that are already bf16-representable."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    return (u >> 16).astype(np.uint16)
+
+
+# ----------------------------------------------------------------------------
+# weights
+# ----------------------------------------------------------------------------
+def weight_shapes(p: PairCfg, with_aux_head: bool = False) -> Dict[str, Tuple[int, ...]]:
+    """Tensor name -> shape.  Matrices are [out_features, in_features] row-major."""
+    s: Dict[str, Tuple[int, ...]] = {}
+
+    def model(prefix: str, m: ModelCfg, head: bool):
+        s[f"{prefix}.embed"] = (m.vocab, m.d_model)
+        for l, lc in enumerate(m.layers):
+            b = f"{prefix}.L{l}."
+            s[b + "attn_norm"] = (m.d_model,)
+            s[b + "wq"] = (lc.d_q, m.d_model)
+            s[b + "wk"] = (lc.d_kv, m.d_model)
+            s[b + "wv"] = (lc.d_kv, m.d_model)
+            s[b + "wo"] = (m.d_model, lc.d_q)
+            s[b + "ffn_norm"] = (m.d_model,)
+            s[b + "w_gate"] = (lc.ffn_dim, m.d_model)
+            s[b + "w_up"] = (lc.ffn_dim, m.d_model)
+            s[b + "w_down"] = (m.d_model, lc.ffn_dim)
+        if head:
+            s[f"{prefix}.final_norm"] = (m.d_model,)
+            s[f"{prefix}.lm_head"] = (m.vocab, m.d_model)
+
+    model("aux", p.aux, with_aux_head)
+    model("base", p.base, True)
+    for i, j in enumerate(p.layer_map):
+        din, dout = p.aux.layers[j].d_kv, p.base.layers[i].d_kv
+        s[f"pred.L{i}.fk"] = (dout, din)
+        s[f"pred.L{i}.fv"] = (dout, din)
+        if p.predictor_bias:
+            s[f"pred.L{i}.bk"] = (dout,)
+            s[f"pred.L{i}.bv"] = (dout,)
+    return s
+
+
+def _stream(seed: int, name: str) -> np.random.Generator:
+    h = hashlib.sha256(f"{seed}:{name}".encode()).digest()
+    key = int.from_bytes(h[:16], "little")
+    return np.random.Generator(np.random.Philox(key=key))
+
+
+def make_tensor(p: PairCfg, name: str, shape: Sequence[int], seed: int, regime: str) -> np.ndarray:
+    """One weight tensor as fp32 (already rounded to bf16 when p.dtype == 'bf16').
+
+    regime "n002": every matrix, embedding and bias ~ N(0, 0.02^2), norm gains 1.
+    regime "fanin": matrices ~ N(0, 1/fan_in), embeddings ~ N(0,1), gains
+                    1 + N(0, 0.1^2), biases ~ N(0, 0.1^2): peaked softmax, O(1)
+                    activations; a harder numerical test than "n002".
+    """
+    g = _stream(seed, name)
+    leaf = name.split(".")[-1]
+    shape = tuple(int(x) for x in shape)
+    if leaf.endswith("norm"):
+        w = np.ones(shape, np.float32)
+        if regime == "fanin":
+            w = w + 0.1 * g.standard_normal(shape, dtype=np.float32)
+    else:
+        w = g.standard_normal(shape, dtype=np.float32)
+        if regime == "n002":
+            w *= np.float32(0.02)
+        elif regime == "fanin":
+            if leaf == "embed":
+                pass
+            elif len(shape) == 1:
+                w *= np.float32(0.1)
+            else:
+                w *= np.float32(1.0 / np.sqrt(shape[-1]))
+        else:
+            raise KeyError(regime)
+    if p.dtype == "bf16":
+        w = round_to_bf16(w)
+    return w
+
+
+def make_weights(p: PairCfg, seed: int = 0, regime: str = "n002",
+                 with_aux_head: bool = False, threads: int = 8) -> Dict[str, np.ndarray]:
+    shapes = weight_shapes(p, with_aux_head)
+    names = list(shapes)
+    with ThreadPoolExecutor(max_workers=threads) as ex:
+        arrs = list(ex.map(lambda n: make_tensor(p, n, shapes[n], seed, regime), names))
+    return dict(zip(names, arrs))
+
+
+# ----------------------------------------------------------------------------
+# prompts
+# ----------------------------------------------------------------------------
+def zipf_tokens(n: int, vocab: int, seed: int, s: float = 1.1, tag: str = "tokens") -> np.ndarray:
+    """Token ids with P(id = r-1) proportional to r^-s, r = 1..vocab (ids not permuted):
+    a few very frequent ids and a long tail, like natural-language prompts."""
+    g = _stream(seed, tag)
+    w = np.arange(1, vocab + 1, dtype=np.float64) ** (-s)
+    cdf = np.cumsum(w)
+    cdf /= cdf[-1]
+    u = g.random(n)
+    return np.minimum(np.searchsorted(cdf, u, side="left"), vocab - 1).astype(np.int32)
+
+
+def uniform_tokens(n: int, vocab: int, seed: int, tag: str = "tokens") -> np.ndarray:
+    g = _stream(seed, tag)
+    return g.integers(0, vocab, size=n, dtype=np.int64).astype(np.int32)
+
+
+def ragged_lengths(batch: int, lo: int, hi: int, seed: int, tag: str = "lengths") -> np.ndarray:
+    g = _stream(seed, tag)
+    return g.integers(lo, hi + 1, size=batch, dtype=np.int64).astype(np.int32)
+
+
+@dataclass
+class Prompts:
+    tokens: np.ndarray      # int32 [sum(lengths)], sequences packed back to back
+    lengths: np.ndarray     # int32 [batch]
+
+    @property
+    def batch(self) -> int:
+        return int(self.lengths.shape[0])
+
+    @property
+    def total(self) -> int:
+        return int(self.lengths.sum())
+
+    def seq(self, b: int) -> np.ndarray:
+        o = int(self.lengths[:b].sum())
+        return self.tokens[o:o + int(self.lengths[b])]
+
+
+def prompts(name: str, seed: int = 0) -> Prompts:
+    """Prompt batch of a named benchmark configuration."""
+    v = pair(name).base.vocab
+    if name in ("c1", "c1_bf16"):
+        lens = np.array([64], np.int32)
+        return Prompts(uniform_tokens(64, v, seed), lens)
+    if name == "c2":
+        lens = np.array([1024], np.int32)
+        return Prompts(zipf_tokens(1024, v, seed), lens)
+    if name == "c3":
+        lens = ragged_lengths(8, 512, 4096, seed)
+        return Prompts(zipf_tokens(int(lens.sum()), v, seed), lens)
+    if name == "c4":
+        lens = np.full(32, 2048, np.int32)
+        return Prompts(zipf_tokens(int(lens.sum()), v, seed), lens)
+    if name == "c5":
+        lens = np.full(4, 16384, np.int32)
+        return Prompts(uniform_tokens(int(lens.sum()), v, seed), lens)
+    raise KeyError(name)
+
+
+def custom_prompts(vocab: int, lengths: Sequence[int], seed: int = 0, zipf: bool = True) -> Prompts:
+    lens = np.asarray(lengths, np.int32)
+    n = int(lens.sum())
+    toks = zipf_tokens(n, vocab, seed) if zipf else uniform_tokens(n, vocab, seed)
+    return Prompts(toks, lens)
+
+
+# ----------------------------------------------------------------------------
+# work accounting (counts of what the method must compute; no arithmetic of it)
+# ----------------------------------------------------------------------------
+def algorithmic_work(p: PairCfg, lengths: Sequence[int]) -> Dict[str, float]:
+    """FLOPs and bytes the TTFT path must perform for these prompt lengths.
+
+    Causal attention counts L(L+1)/2 (query, key) pairs; the auxiliary layers
+    above the last one the map uses, and everything after the K/V projection in
+    that last layer, are not needed for the outputs and are not credited.
+    """
+    lens = [int(x) for x in lengths]
+    T = sum(lens)
+    pairs = sum(l * (l + 1) // 2 for l in lens)
+    j_max = max(p.layer_map)
+    eb = 2 if p.dtype == "bf16" else 4
+    gemm = attn = 0.0
+    for j, lc in enumerate(p.aux.layers):
+        d = p.aux.d_model
+        if j < j_max:
+            gemm += 2.0 * T * (d * (lc.d_q + 2 * lc.d_kv) + lc.d_q * d + 3 * d * lc.ffn_dim)
+            attn += 4.0 * lc.d_q * pairs
+        elif j == j_max:
+            gemm += 2.0 * T * d * 2 * lc.d_kv
+    pred = 0.0
+    cache_bytes = 0.0
+    for i, j in enumerate(p.layer_map):
+        pred += 4.0 * T * p.aux.layers[j].d_kv * p.base.layers[i].d_kv
+        cache_bytes += 2.0 * T * p.base.layers[i].d_kv * eb
+    step_w = 0.0
+    step_flops = 0.0
+    B = len(lens)
+    for lc in p.base.layers:
+        d = p.base.d_model
+        n = d * lc.d_q * 2 + 3 * d * lc.ffn_dim
+        step_w += n * eb
+        step_flops += 2.0 * B * n
+    step_w += p.base.vocab * p.base.d_model * eb
+    step_flops += 2.0 * B * p.base.vocab * p.base.d_model
+    return dict(tokens=T, aux_gemm_flops=gemm, attn_flops=attn, pred_flops=pred,
+                tensor_flops=gemm + attn + pred, cache_bytes=cache_bytes,
+                step_weight_bytes=step_w, step_bytes=step_w + cache_bytes,
+                step_flops=step_flops)
