@@ -1,0 +1,205 @@
+/*
+ * kvp.h - C ABI of the KV Prediction time-to-first-token library (CUDA, sm_100a).
+ *
+ * The library runs the inference algorithm of KV Prediction (arXiv 2410.08391,
+ * Fig. 2(b) "KV Prediction Inference", Sec. 4.1 "Inference"):
+ *
+ *     a, KV_A  <- A(I)                auxiliary model over the whole prompt
+ *     KV_B_hat <- P(KV_A)             per-base-layer linear maps (Sec. 4.2)
+ *     b        <- B(I[-1], KV_B_hat)  one base-model step on the predicted cache
+ *     loop:  b, p <- B(I[-1], KV_B_hat);  KV_B_hat <- KV_B_hat + p
+ *
+ * General conventions
+ *   - Every call returns a kvp_status (0 = KVP_OK, negative = error).  Nothing
+ *     throws, aborts or keeps global state.  kvp_last_error() returns a message
+ *     owned by the handle, valid until the next call on that handle.
+ *   - "dev" pointers are CUDA device pointers on the device that was current when
+ *     kvp_create() ran; "host" pointers are ordinary host memory.
+ *   - The caller owns ALL device memory (weights, packed weights, workspace, cache
+ *     pools, block table, outputs).  The handle borrows the packed-weight pointer
+ *     until kvp_destroy(); it owns only host metadata and TMA descriptors.
+ *   - Calls that take a stream only enqueue work on it and return without
+ *     synchronising (except the *_host variant, which synchronises the stream);
+ *     arguments are validated on the host before anything is launched.
+ *   - Device-side waits are bounded; a kernel that gives up, or that meets an
+ *     out-of-range token id or page index, records a code in a status word inside
+ *     the workspace and skips the access.  kvp_poll_status() reads it.  The status
+ *     word is cleared by kvp_prefill_predict() at its start and by kvp_poll_status();
+ *     poll once on a fresh workspace before using it for kvp_decode_step() alone.
+ *   - Matrices are [out_features, in_features], row-major, dense.
+ */
+#ifndef KVP_H_
+#define KVP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t kvp_status;
+enum {
+  KVP_OK = 0,
+  KVP_ERR_INVALID_ARG = -1, /* NULL pointer, bad enum, batch <= 0, length <= 0 ...          */
+  KVP_ERR_SHAPE = -2,       /* tensor shape or model dimensions inconsistent                 */
+  KVP_ERR_UNSUPPORTED = -3, /* valid but not implemented (e.g. odd head_dim)                 */
+  KVP_ERR_NOT_LOADED = -4,  /* compute call before kvp_load_weights() supplied every tensor  */
+  KVP_ERR_CACHE_FULL = -5,  /* prompt needs more pages than block table / pools provide      */
+  KVP_ERR_CUDA = -6,        /* a CUDA runtime or driver call failed                          */
+  KVP_ERR_TIMEOUT = -7,     /* a bounded device-side wait ran out                            */
+  KVP_ERR_WORKSPACE = -8,   /* workspace or packed-weight buffer too small or misaligned     */
+  KVP_ERR_BAD_INDEX = -9    /* device met a token id or page index out of range              */
+};
+
+enum { KVP_F32 = 0, KVP_BF16 = 1 };
+
+#define KVP_MAX_BATCH 256
+
+/* One transformer layer.  OpenELM-style models vary these per layer (Sec. 4.2
+ * "OpenELM KV Prediction Specification": the KV cache width differs per layer). */
+typedef struct {
+  int32_t n_q_heads;  /* multiple of n_kv_heads                       */
+  int32_t n_kv_heads; /* >= 1                                         */
+  int32_t head_dim;   /* even; same for every layer of one model      */
+  int32_t ffn_dim;    /* SwiGLU hidden width                          */
+} kvp_layer_cfg;
+
+/* A pre-norm decoder: RMSNorm -> GQA attention with RoPE (rotate-half pairing)
+ * -> residual; RMSNorm -> SwiGLU FFN -> residual; final RMSNorm -> LM head. */
+typedef struct {
+  int32_t n_layers;
+  int32_t d_model;
+  int32_t vocab;
+  float rope_theta;
+  float rms_eps;
+  const kvp_layer_cfg* layers; /* host, [n_layers]; copied by kvp_create */
+} kvp_model_cfg;
+
+typedef struct {
+  int32_t dtype;          /* KVP_F32 | KVP_BF16: storage type of weights, activations and cache.
+                             Accumulation, norms, softmax and the base step's activations are fp32. */
+  int32_t page_tokens;    /* tokens per cache page; must be 64                                       */
+  int32_t predictor_bias; /* 1: the predictor has bias vectors pred.L{i}.bk / bv                     */
+  int32_t reserved;       /* must be 0                                                               */
+} kvp_options;
+
+/* A named tensor handed to kvp_load_weights().  Names:
+ *   "aux.embed" [vocab, d_A]
+ *   "aux.L{j}.attn_norm" [d_A]   "aux.L{j}.ffn_norm" [d_A]
+ *   "aux.L{j}.wq" [nq*hd, d_A]   "aux.L{j}.wk" / "wv" [nkv*hd, d_A]   "aux.L{j}.wo" [d_A, nq*hd]
+ *   "aux.L{j}.w_gate" / "w_up" [ffn, d_A]   "aux.L{j}.w_down" [d_A, ffn]
+ *   the same under "base.", plus "base.final_norm" [d_B] and "base.lm_head" [vocab, d_B]
+ *   "pred.L{i}.fk" / "fv" [d_kvB_i, d_kvA_{j_i}]  and, with predictor_bias, "pred.L{i}.bk" / "bv" [d_kvB_i]
+ * Auxiliary layers above max_i j_i, "aux.final_norm" and "aux.lm_head" are never read
+ * (the auxiliary logits are unused at inference, Sec. 4.3) and may be omitted. */
+typedef struct {
+  const char* name;
+  const void* data;  /* dev, dense row-major                      */
+  int32_t dtype;     /* KVP_F32 | KVP_BF16 (converted on load)    */
+  int32_t ndim;      /* 1 or 2                                    */
+  int64_t shape[2];
+} kvp_tensor;
+
+/* The paged base-model KV cache, the user-visible product of prefill (Sec. 4.1:
+ * the predicted cache is what the base model's attention then consumes).
+ * Base layer i has one K pool and one V pool of n_pages pages; a page is
+ * [n_kv_heads_i][page_tokens][head_dim] elements of the run dtype.  Entry t of
+ * sequence b lives in page block_table[b * max_pages_per_seq + t / page_tokens]
+ * at row t % page_tokens, in every layer's pools.  Keys are stored after RoPE.
+ * Rows at or beyond a sequence's length are unspecified. */
+typedef struct {
+  void* const* k_pools;        /* host array [n_base_layers] of dev pointers            */
+  void* const* v_pools;        /* host array [n_base_layers] of dev pointers            */
+  const int32_t* block_table;  /* dev, [>= batch][max_pages_per_seq], filled by caller  */
+  int32_t* seq_lens;           /* dev, [>= batch]; written by prefill, +1 per decode    */
+  int32_t max_pages_per_seq;
+  int32_t n_pages;             /* pages in every pool                                   */
+} kvp_cache;
+
+typedef struct kvp_handle kvp_handle;
+
+/* Validates both models and the layer map j_i (Sec. 4.2: j_i in [0, n_A), here also
+ * required non-decreasing; both models share one vocabulary) and builds the kernel
+ * plan.  aux/base/layer_map/opt: host.  *out receives the handle. */
+kvp_status kvp_create(const kvp_model_cfg* aux, const kvp_model_cfg* base,
+                      const int32_t* layer_map /* host [base->n_layers] */,
+                      const kvp_options* opt, kvp_handle** out);
+
+void kvp_destroy(kvp_handle* h);
+
+/* NUL-terminated description of the last error on this handle ("" if none). */
+const char* kvp_last_error(const kvp_handle* h);
+
+/* Layer-map helpers (Sec. 4.2 and Table 1): write j_0..j_{n_base-1} to out (host).
+ * canonical: consecutive base layers share an aux layer, the first n_base mod n_aux aux
+ *            layers feed one more base layer than the rest (the KVP-C rows of Table 1);
+ * pruned:    aux = base with only `retained` layers kept (ascending, retained[0] == 0);
+ *            j_i = index of the largest retained layer <= i (the KVP-LP rows);
+ * uniform:   j_i = floor(i * n_aux / n_base). */
+kvp_status kvp_layer_map_canonical(int32_t n_base, int32_t n_aux, int32_t* out);
+kvp_status kvp_layer_map_pruned(int32_t n_base, const int32_t* retained, int32_t n_aux, int32_t* out);
+kvp_status kvp_layer_map_uniform(int32_t n_base, int32_t n_aux, int32_t* out);
+
+/* Bytes of the packed-weight buffer kvp_load_weights() fills (256-byte aligned dev memory). */
+kvp_status kvp_packed_weight_bytes(const kvp_handle* h, size_t* bytes);
+
+/* Bytes of workspace for calls with batch <= max_batch and sum of lengths <= max_total_tokens. */
+kvp_status kvp_workspace_bytes(const kvp_handle* h, int32_t max_batch, int64_t max_total_tokens,
+                               size_t* bytes);
+
+/* Bytes of one page of base layer `base_layer` (K or V; both are equal). */
+kvp_status kvp_cache_layout(const kvp_handle* h, int32_t base_layer, size_t* bytes_per_page);
+
+/* Converts and re-lays-out the n given tensors into `packed` (dev) with kernels enqueued on
+ * `stream`.  May be called several times with disjoint subsets; compute calls need every
+ * required tensor.  Once the enqueued work has finished the source tensors may be freed;
+ * `packed` must stay alive until kvp_destroy().  Shape or name mismatch -> KVP_ERR_SHAPE. */
+kvp_status kvp_load_weights(kvp_handle* h, const kvp_tensor* tensors, int32_t n,
+                            void* packed, size_t packed_bytes, void* stream);
+
+/* The time-to-first-token path (Fig. 2(b), first three statements): auxiliary prefill over
+ * all prompts, KV prediction into the paged cache, one base step per sequence on its last
+ * prompt token at position L_b - 1 attending to predicted entries 0..L_b-1 (nothing is
+ * appended; the base K/V projections are unused).
+ *   tokens        dev  int32 [sum(lengths)]  prompts packed back to back
+ *   lengths       host int32 [batch]         each >= 1
+ *   cache              pools and block table as described above; seq_lens[b] <- L_b
+ *   workspace     dev, 256-byte aligned, >= kvp_workspace_bytes(batch, sum(lengths))
+ *   logits_out    dev  fp32 [batch, vocab]
+ *   first_token   dev  int32 [batch], argmax of logits (lowest index on ties); may be NULL */
+kvp_status kvp_prefill_predict(kvp_handle* h, const int32_t* tokens, const int32_t* lengths,
+                               int32_t batch, const kvp_cache* cache, void* workspace,
+                               size_t workspace_bytes, float* logits_out, int32_t* first_token,
+                               void* stream);
+
+/* Same path with HOST tokens and HOST outputs: copies the tokens to the device, runs
+ * kvp_prefill_predict, copies logits (if logits_host != NULL) and first tokens back and
+ * synchronises `stream`.  The token staging area lives at the end of the workspace
+ * (accounted for by kvp_workspace_bytes); logits_dev is a dev scratch [batch, vocab]. */
+kvp_status kvp_prefill_predict_host(kvp_handle* h, const int32_t* tokens_host,
+                                    const int32_t* lengths, int32_t batch, const kvp_cache* cache,
+                                    void* workspace, size_t workspace_bytes, float* logits_dev,
+                                    float* logits_host, int32_t* first_token_host, void* stream);
+
+/* One generation step (Fig. 2(b), loop body): for every sequence the base model computes
+ * q, k, v of `tokens[b]` with its own projections at position seq_lens[b], appends k
+ * (after RoPE) and v to the cache, attends over seq_lens[b] + 1 entries and emits logits;
+ * seq_lens[b] += 1.  lengths_host[b] must equal the current seq_lens[b] (host copy used
+ * for validation and scheduling).  KVP_ERR_CACHE_FULL if a sequence has no room left. */
+kvp_status kvp_decode_step(kvp_handle* h, const int32_t* tokens /* dev [batch] */,
+                           const int32_t* lengths_host, int32_t batch, const kvp_cache* cache,
+                           void* workspace, size_t workspace_bytes, float* logits_out,
+                           int32_t* next_token, void* stream);
+
+/* Synchronises `stream`, reads the device status word of `workspace`, clears it and returns
+ * KVP_OK, KVP_ERR_TIMEOUT, KVP_ERR_BAD_INDEX or KVP_ERR_CUDA. */
+kvp_status kvp_poll_status(kvp_handle* h, void* workspace, void* stream);
+
+/* Number of kernels the handle launched since creation (for launch accounting). */
+int64_t kvp_launch_count(const kvp_handle* h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KVP_H_ */
