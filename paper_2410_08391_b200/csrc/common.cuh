@@ -1,0 +1,120 @@
+// Shared device helpers and launch-function declarations for the KV Prediction library.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+typedef __nv_bfloat16 bf16;
+
+// Codes kernels write into the device status word (first int of the workspace).
+enum : int { DEV_OK = 0, DEV_TIMEOUT = 1, DEV_BAD_TOKEN = 2, DEV_BAD_PAGE = 3 };
+
+constexpr int PAGE_TOKENS = 64;
+constexpr int MAX_PRED_SEG = 8;   // base layers fed by one auxiliary layer
+
+__device__ __forceinline__ float to_f(float v) { return v; }
+__device__ __forceinline__ float to_f(bf16 v) { return __bfloat162float(v); }
+template <class T> __device__ __forceinline__ T from_f(float v);
+template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ bf16 from_f<bf16>(float v) { return __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ void dev_flag(int* status, int code) { atomicCAS(status, DEV_OK, code); }
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// RoPE angle pos * inv_freq reduced to [0, 2 pi) in fp64 before the fp32 sincos: at
+// position 16 000 an fp32 product would already be off by about 1e-3 rad.
+struct InvFreq { double f[64]; };   // theta^(-2c/hd), c < hd/2 <= 64
+__device__ __forceinline__ void rope_sincos(int pos, double inv_freq, float* s, float* c) {
+  double a = (double)pos * inv_freq;
+  const double two_pi = 6.283185307179586476925286766559;
+  a -= two_pi * floor(a / two_pi);
+  sincosf((float)a, s, c);
+}
+void fill_inv_freq(InvFreq* f, int hd, float theta);
+
+// Where the predictor GEMM scatters its columns: the concatenated outputs of all base
+// layers fed by one auxiliary layer; segment s covers columns [col0[s], col0[s+1]).
+struct PagedOut {
+  int n_seg;
+  int col0[MAX_PRED_SEG + 1];
+  int n_kv[MAX_PRED_SEG];
+  void* pool[MAX_PRED_SEG];
+  const float* bias;     // concatenated, may be null
+  const int* tok_slot;   // [M] page * PAGE_TOKENS + row, or -1
+  int head_dim;
+};
+
+// Row placement used when packing weights: plain offset, or gate/up block interleave.
+struct RowMap {
+  int row_offset;   // G == 0: dst_row = r + row_offset
+  int G;            // G > 0: rows interleaved in blocks of G (gate block, then up block)
+  int which;        // 0 = gate, 1 = up
+  int n_rows_total; // ffn (rows of gate, and of up)
+};
+__host__ __device__ __forceinline__ int map_row(const RowMap& m, int r) {
+  if (m.G == 0) return r + m.row_offset;
+  int blk = r / m.G;
+  int rem = m.n_rows_total - blk * m.G;
+  int gb = rem < m.G ? rem : m.G;
+  return 2 * blk * m.G + m.which * gb + (r - blk * m.G);
+}
+
+enum GemmEpi : int { EPI_STORE = 0, EPI_RESID = 1, EPI_PAGED = 2 };
+
+struct GemmArgs {
+  const void* A; int lda;        // [M, K] run dtype
+  const void* W; int ldw;        // [N, K] run dtype
+  int M, N, K;
+  void* C; int ldc;              // EPI_STORE: run dtype [M, N]
+  float* X; int ldx;             // EPI_RESID: fp32 residual, X += A W^T
+  PagedOut paged;                // EPI_PAGED
+};
+
+// ---- launchers (defined in the .cu files); all enqueue on `st` and count launches ----
+struct LaunchCtx {
+  cudaStream_t st;
+  int64_t* n_launch;
+  int* status;      // device status word
+  int dtype;        // 0 f32, 1 bf16
+};
+
+void launch_pack_rows(const LaunchCtx&, const void* src, int src_dtype, void* dst, int dst_dtype,
+                      int rows, int cols, RowMap map);
+void launch_build_index(const LaunchCtx&, const int* cu_host /*[B+1]*/, int batch, int total,
+                        int* cu_dev, int* tok_pos, int* tok_slot, int* last_tok_idx,
+                        const int* block_table, int max_pages_per_seq, int n_pages, int* seq_lens);
+void launch_embed(const LaunchCtx&, const int* tokens, const int* gather_idx, int n_rows,
+                  const void* table, int vocab, int d, float* x);
+void launch_rmsnorm(const LaunchCtx&, const float* x, const float* gain, float eps, int rows, int d,
+                    void* out, int out_dtype);
+void launch_rope(const LaunchCtx&, void* qkv, int ld, int rows, int n_heads_rot, int head_dim,
+                 const int* tok_pos, float theta);
+void launch_swiglu(const LaunchCtx&, const void* gu, int rows, int ffn, int G, void* act);
+void launch_gemm_simt(const LaunchCtx&, const GemmArgs&, int epi);
+void launch_attn_prefill_simt(const LaunchCtx&, const void* qkv, int ld, int nq, int nkv, int hd,
+                              const int* cu_dev, int batch, int total, void* out, int ldo);
+
+// base single-token step
+enum StepGemvMode : int { GEMV_STORE = 0, GEMV_RESID = 1, GEMV_SWIGLU = 2 };
+void launch_step_gemv(const LaunchCtx&, const void* W, int ldw, int N, int K, const float* x, int ldx,
+                      int batch, float* y, int ldy, int mode, int G, int ffn);
+void launch_step_attn(const LaunchCtx&, const float* q, int ldq, int nq, int nkv, int hd, float theta,
+                      const void* kpool, const void* vpool, const int* block_table,
+                      int max_pages_per_seq, int n_pages, const int* seq_lens, int extra, int batch,
+                      int max_keys, float* part, float* out);
+void launch_step_append(const LaunchCtx&, const float* qkv, int nq, int nkv, int hd, float theta,
+                        void* kpool, void* vpool, const int* block_table, int max_pages_per_seq,
+                        int n_pages, const int* seq_lens, int batch);
+void launch_argmax(const LaunchCtx&, const float* logits, int batch, int vocab, int* out);
+void launch_add_int(const LaunchCtx&, int* v, int n, int delta);
+int step_attn_splits(int batch, int nkv, int max_keys);

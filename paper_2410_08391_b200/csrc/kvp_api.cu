@@ -1,0 +1,544 @@
+// C ABI of the KV Prediction library: validation, plan, weight packing and the kernel
+// schedule of the time-to-first-token path and of the generation step.
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <algorithm>
+#include <new>
+
+#include "kvp_internal.h"
+
+namespace {
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+kvp_status fail(kvp_handle* h, kvp_status code, const char* fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof buf, fmt, ap);
+  va_end(ap);
+  if (h) h->err = buf;
+  return code;
+}
+
+const char* validate_model(const kvp_model_cfg* m) {
+  if (!m || !m->layers) return "model config or its layer array is NULL";
+  if (m->n_layers <= 0 || m->n_layers > 1024) return "n_layers out of range";
+  if (m->d_model <= 0 || m->vocab <= 0) return "d_model and vocab must be positive";
+  if (!(m->rope_theta > 0.f) || !(m->rms_eps >= 0.f)) return "rope_theta must be > 0 and rms_eps >= 0";
+  for (int l = 0; l < m->n_layers; ++l) {
+    const kvp_layer_cfg& c = m->layers[l];
+    if (c.n_q_heads <= 0 || c.n_kv_heads <= 0 || c.head_dim <= 0 || c.ffn_dim <= 0) return "layer dimensions must be positive";
+    if (c.n_q_heads % c.n_kv_heads) return "n_q_heads must be a multiple of n_kv_heads";
+    if (c.head_dim != m->layers[0].head_dim) return "head_dim must be the same in every layer of a model";
+  }
+  return nullptr;
+}
+
+const char* unsupported_model(const kvp_model_cfg* m) {
+  for (int l = 0; l < m->n_layers; ++l) {
+    const kvp_layer_cfg& c = m->layers[l];
+    if (c.head_dim % 2 || c.head_dim > 128) return "head_dim must be even and <= 128";
+    if (c.n_q_heads / c.n_kv_heads > 8) return "more than 8 query heads per kv head";
+  }
+  return nullptr;
+}
+
+void plan_model(ModelPlan& p, const kvp_model_cfg* m, int es, bool bf16_mode, size_t& off, bool with_head) {
+  p.n_layers = m->n_layers; p.d = m->d_model; p.vocab = m->vocab; p.theta = m->rope_theta; p.eps = m->rms_eps;
+  p.max_nqkv = p.max_dq = p.max_ffn = p.max_group = p.max_nkv = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  p.embed = take((size_t)m->vocab * m->d_model * es);
+  p.L.resize(m->n_layers);
+  for (int l = 0; l < m->n_layers; ++l) {
+    LayerPlan& L = p.L[l];
+    const kvp_layer_cfg& c = m->layers[l];
+    L.nq = c.n_q_heads; L.nkv = c.n_kv_heads; L.hd = c.head_dim; L.ffn = c.ffn_dim;
+    L.dq = L.nq * L.hd; L.dkv = L.nkv * L.hd; L.nqkv = L.dq + 2 * L.dkv;
+    L.G = (bf16_mode && L.ffn % 64 == 0) ? 64 : 0;
+    L.wqkv = take((size_t)L.nqkv * p.d * es);
+    L.wo = take((size_t)p.d * L.dq * es);
+    L.wgu = take((size_t)2 * L.ffn * p.d * es);
+    L.wd = take((size_t)p.d * L.ffn * es);
+    L.attn_norm = take((size_t)p.d * 4);
+    L.ffn_norm = take((size_t)p.d * 4);
+    p.max_nqkv = std::max(p.max_nqkv, L.nqkv); p.max_dq = std::max(p.max_dq, L.dq);
+    p.max_ffn = std::max(p.max_ffn, L.ffn); p.max_group = std::max(p.max_group, L.nq / L.nkv);
+    p.max_nkv = std::max(p.max_nkv, L.nkv);
+  }
+  p.final_norm = p.lm_head = 0;
+  if (with_head) {
+    p.final_norm = take((size_t)p.d * 4);
+    p.lm_head = take((size_t)m->vocab * m->d_model * es);
+  }
+}
+
+void add_model_slots(kvp_handle* h, const char* prefix, const ModelPlan& p, int n_live_layers, bool with_head) {
+  int dt = h->opt.dtype;
+  auto name = [&](int l, const char* leaf) { char b[96]; snprintf(b, sizeof b, "%s.L%d.%s", prefix, l, leaf); return std::string(b); };
+  h->slots[std::string(prefix) + ".embed"] = PackSlot{p.embed, p.vocab, p.d, dt, RowMap{0, 0, 0, 0}};
+  for (int l = 0; l < n_live_layers; ++l) {
+    const LayerPlan& L = p.L[l];
+    h->slots[name(l, "attn_norm")] = PackSlot{L.attn_norm, 1, p.d, 0, RowMap{0, 0, 0, 0}};
+    h->slots[name(l, "ffn_norm")] = PackSlot{L.ffn_norm, 1, p.d, 0, RowMap{0, 0, 0, 0}};
+    h->slots[name(l, "wq")] = PackSlot{L.wqkv, L.dq, p.d, dt, RowMap{0, 0, 0, 0}};
+    h->slots[name(l, "wk")] = PackSlot{L.wqkv, L.dkv, p.d, dt, RowMap{L.dq, 0, 0, 0}};
+    h->slots[name(l, "wv")] = PackSlot{L.wqkv, L.dkv, p.d, dt, RowMap{L.dq + L.dkv, 0, 0, 0}};
+    h->slots[name(l, "wo")] = PackSlot{L.wo, p.d, L.dq, dt, RowMap{0, 0, 0, 0}};
+    h->slots[name(l, "w_gate")] = PackSlot{L.wgu, L.ffn, p.d, dt, RowMap{0, L.G, 0, L.ffn}};
+    h->slots[name(l, "w_up")] = PackSlot{L.wgu, L.ffn, p.d, dt, RowMap{L.G == 0 ? L.ffn : 0, L.G, 1, L.ffn}};
+    h->slots[name(l, "w_down")] = PackSlot{L.wd, p.d, L.ffn, dt, RowMap{0, 0, 0, 0}};
+  }
+  if (with_head) {
+    h->slots[std::string(prefix) + ".final_norm"] = PackSlot{p.final_norm, 1, p.d, 0, RowMap{0, 0, 0, 0}};
+    h->slots[std::string(prefix) + ".lm_head"] = PackSlot{p.lm_head, p.vocab, p.d, dt, RowMap{0, 0, 0, 0}};
+  }
+}
+
+WsLayout ws_layout(const kvp_handle* h, int64_t Bm, int64_t Tm) {
+  WsLayout w;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  const ModelPlan &A = h->aux, &B = h->base;
+  size_t es = h->es;
+  w.status = take(256);
+  w.cu = take((Bm + 1) * 4);
+  w.last_idx = take(Bm * 4);
+  w.tok_pos = take(Tm * 4);
+  w.tok_slot = take(Tm * 4);
+  w.x = take(Tm * A.d * 4);
+  w.h = take(Tm * A.d * es);
+  w.qkv = take(Tm * A.max_nqkv * es);
+  w.attn = take(Tm * A.max_dq * es);
+  w.gu = take(Tm * 2 * (size_t)A.max_ffn * es);
+  w.act = take(Tm * (size_t)A.max_ffn * es);
+  w.xb = take(Bm * B.d * 4);
+  w.hb = take(Bm * B.d * 4);
+  w.qkvb = take(Bm * B.max_nqkv * 4);
+  w.ab = take(Bm * B.max_dq * 4);
+  w.actb = take(Bm * (size_t)B.max_ffn * 4);
+  w.part = take((size_t)(2 * 148 + Bm * B.max_nkv) * B.max_group * (B.L[0].hd + 2) * 4);
+  w.tok_stage = take(Tm * 4);
+  w.first_stage = take(Bm * 4);
+  w.total = off;
+  return w;
+}
+
+kvp_status check_cuda(kvp_handle* h, const char* what) {
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(h, KVP_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+  return KVP_OK;
+}
+
+struct CallShape { std::vector<int> cu; int total; int max_len; };
+
+kvp_status common_checks(kvp_handle* h, const int32_t* lengths, int32_t batch, const kvp_cache* cache, void* ws,
+                         int extra_tokens, CallShape* cs) {
+  if (!h) return KVP_ERR_INVALID_ARG;
+  h->err.clear();
+  if (!lengths || !cache || !ws) return fail(h, KVP_ERR_INVALID_ARG, "NULL argument");
+  if (batch <= 0 || batch > KVP_MAX_BATCH) return fail(h, KVP_ERR_INVALID_ARG, "batch %d outside [1, %d]", batch, KVP_MAX_BATCH);
+  if (!cache->k_pools || !cache->v_pools || !cache->block_table || !cache->seq_lens)
+    return fail(h, KVP_ERR_INVALID_ARG, "cache has a NULL member");
+  if (cache->max_pages_per_seq <= 0 || cache->n_pages <= 0) return fail(h, KVP_ERR_INVALID_ARG, "cache has no pages");
+  for (int i = 0; i < h->base.n_layers; ++i)
+    if (!cache->k_pools[i] || !cache->v_pools[i]) return fail(h, KVP_ERR_INVALID_ARG, "cache pool of base layer %d is NULL", i);
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return check_cuda(h, "cudaGetDevice");
+  if (dev != h->device) return fail(h, KVP_ERR_INVALID_ARG, "current device %d is not the handle's device %d", dev, h->device);
+  cs->cu.assign(batch + 1, 0);
+  cs->max_len = 0;
+  int64_t total = 0, pages = 0;
+  for (int b = 0; b < batch; ++b) {
+    if (lengths[b] <= 0) return fail(h, KVP_ERR_INVALID_ARG, "lengths[%d] = %d must be >= 1", b, lengths[b]);
+    int64_t need = ((int64_t)lengths[b] + extra_tokens + PAGE_TOKENS - 1) / PAGE_TOKENS;
+    if (need > cache->max_pages_per_seq)
+      return fail(h, KVP_ERR_CACHE_FULL, "sequence %d needs %lld pages, block table has %d per sequence", b, (long long)need, cache->max_pages_per_seq);
+    pages += need;
+    total += lengths[b];
+    if (total > 0x7fffffff / 2) return fail(h, KVP_ERR_INVALID_ARG, "too many tokens");
+    cs->cu[b + 1] = (int)total;
+    cs->max_len = std::max(cs->max_len, (int)lengths[b]);
+  }
+  if (pages > cache->n_pages) return fail(h, KVP_ERR_CACHE_FULL, "batch needs %lld pages, pools hold %d", (long long)pages, cache->n_pages);
+  cs->total = (int)total;
+  if ((uintptr_t)ws % 256) return fail(h, KVP_ERR_WORKSPACE, "workspace is not 256-byte aligned");
+  return KVP_OK;
+}
+
+bool ends_with(const std::string& s, const char* suf) {
+  size_t n = strlen(suf);
+  return s.size() >= n && s.compare(s.size() - n, n, suf) == 0;
+}
+
+// one base-model layer of a single-token step (shared by the first step and generation)
+void base_layer_step(kvp_handle* h, const LaunchCtx& ctx, int i, const kvp_cache* cache, const WsLayout& w, char* ws,
+                     int batch, int max_keys, bool generation) {
+  const ModelPlan& B = h->base;
+  const LayerPlan& L = B.L[i];
+  const char* P = h->packed;
+  float* xb = (float*)(ws + w.xb);
+  float* hb = (float*)(ws + w.hb);
+  float* qkvb = (float*)(ws + w.qkvb);
+  float* ab = (float*)(ws + w.ab);
+  float* actb = (float*)(ws + w.actb);
+  launch_rmsnorm(ctx, xb, (const float*)(P + L.attn_norm), B.eps, batch, B.d, hb, 0);
+  // the first step needs q only (keys and values are the predicted ones); generation needs q, k, v
+  int n_out = generation ? L.nqkv : L.dq;
+  launch_step_gemv(ctx, P + L.wqkv, B.d, n_out, B.d, hb, B.d, batch, qkvb, n_out, GEMV_STORE, 0, 0);
+  if (generation)
+    launch_step_append(ctx, qkvb, L.nq, L.nkv, L.hd, B.theta, cache->k_pools[i], cache->v_pools[i], cache->block_table,
+                       cache->max_pages_per_seq, cache->n_pages, cache->seq_lens, batch);
+  launch_step_attn(ctx, qkvb, n_out, L.nq, L.nkv, L.hd, B.theta, cache->k_pools[i], cache->v_pools[i], cache->block_table,
+                   cache->max_pages_per_seq, cache->n_pages, cache->seq_lens, generation ? 1 : 0, batch, max_keys,
+                   (float*)(ws + w.part), ab);
+  launch_step_gemv(ctx, P + L.wo, L.dq, B.d, L.dq, ab, L.dq, batch, xb, B.d, GEMV_RESID, 0, 0);
+  launch_rmsnorm(ctx, xb, (const float*)(P + L.ffn_norm), B.eps, batch, B.d, hb, 0);
+  launch_step_gemv(ctx, P + L.wgu, B.d, L.ffn, B.d, hb, B.d, batch, actb, L.ffn, GEMV_SWIGLU, L.G, L.ffn);
+  launch_step_gemv(ctx, P + L.wd, L.ffn, B.d, L.ffn, actb, L.ffn, batch, xb, B.d, GEMV_RESID, 0, 0);
+}
+
+void base_head(kvp_handle* h, const LaunchCtx& ctx, const WsLayout& w, char* ws, int batch, float* logits,
+               int32_t* token_out) {
+  const ModelPlan& B = h->base;
+  const char* P = h->packed;
+  float* xb = (float*)(ws + w.xb);
+  float* hb = (float*)(ws + w.hb);
+  launch_rmsnorm(ctx, xb, (const float*)(P + B.final_norm), B.eps, batch, B.d, hb, 0);
+  launch_step_gemv(ctx, P + B.lm_head, B.d, B.vocab, B.d, hb, B.d, batch, logits, B.vocab, GEMV_STORE, 0, 0);
+  if (token_out) launch_argmax(ctx, logits, batch, B.vocab, token_out);
+}
+
+}  // namespace
+
+// =========================================================================================
+extern "C" {
+
+kvp_status kvp_layer_map_canonical(int32_t n_base, int32_t n_aux, int32_t* out) {
+  if (!out || n_base <= 0 || n_aux <= 0 || n_aux > n_base) return KVP_ERR_INVALID_ARG;
+  int per = n_base / n_aux, more = n_base % n_aux, i = 0;
+  for (int j = 0; j < n_aux; ++j)
+    for (int c = 0; c < per + (j < more ? 1 : 0); ++c) out[i++] = j;
+  return KVP_OK;
+}
+
+kvp_status kvp_layer_map_pruned(int32_t n_base, const int32_t* retained, int32_t n_aux, int32_t* out) {
+  if (!out || !retained || n_base <= 0 || n_aux <= 0 || retained[0] != 0) return KVP_ERR_INVALID_ARG;
+  for (int j = 1; j < n_aux; ++j)
+    if (retained[j] <= retained[j - 1] || retained[j] >= n_base) return KVP_ERR_INVALID_ARG;
+  int j = 0;
+  for (int i = 0; i < n_base; ++i) {
+    while (j + 1 < n_aux && retained[j + 1] <= i) ++j;
+    out[i] = j;
+  }
+  return KVP_OK;
+}
+
+kvp_status kvp_layer_map_uniform(int32_t n_base, int32_t n_aux, int32_t* out) {
+  if (!out || n_base <= 0 || n_aux <= 0) return KVP_ERR_INVALID_ARG;
+  for (int i = 0; i < n_base; ++i) out[i] = (int32_t)(((int64_t)i * n_aux) / n_base);
+  return KVP_OK;
+}
+
+kvp_status kvp_create(const kvp_model_cfg* aux, const kvp_model_cfg* base, const int32_t* layer_map,
+                      const kvp_options* opt, kvp_handle** out) {
+  if (!out) return KVP_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!aux || !base || !layer_map || !opt) return KVP_ERR_INVALID_ARG;
+  if (validate_model(aux) || validate_model(base)) return KVP_ERR_SHAPE;
+  if (opt->dtype != KVP_F32 && opt->dtype != KVP_BF16) return KVP_ERR_INVALID_ARG;
+  if (opt->page_tokens != PAGE_TOKENS || opt->reserved != 0) return KVP_ERR_INVALID_ARG;
+  if (opt->predictor_bias != 0 && opt->predictor_bias != 1) return KVP_ERR_INVALID_ARG;
+  if (aux->vocab != base->vocab) return KVP_ERR_SHAPE;   // one token stream feeds both models
+  if (unsupported_model(aux) || unsupported_model(base)) return KVP_ERR_UNSUPPORTED;
+  int j_max = 0;
+  for (int i = 0; i < base->n_layers; ++i) {
+    if (layer_map[i] < 0 || layer_map[i] >= aux->n_layers) return KVP_ERR_INVALID_ARG;
+    if (i && layer_map[i] < layer_map[i - 1]) return KVP_ERR_INVALID_ARG;
+    j_max = std::max(j_max, layer_map[i]);
+  }
+  kvp_handle* h = new (std::nothrow) kvp_handle();
+  if (!h) return KVP_ERR_INVALID_ARG;
+  h->opt = *opt;
+  h->es = opt->dtype == KVP_BF16 ? 2 : 4;
+  h->map.assign(layer_map, layer_map + base->n_layers);
+  h->j_max = j_max;
+  h->device = 0;
+  cudaGetDevice(&h->device);
+  cudaGetLastError();
+  size_t off = 0;
+  bool bf = opt->dtype == KVP_BF16;
+  plan_model(h->aux, aux, h->es, bf, off, false);
+  plan_model(h->base, base, h->es, bf, off, true);
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  h->groups.resize(j_max + 1);
+  for (int j = 0; j <= j_max; ++j) {
+    PredGroup& g = h->groups[j];
+    g.n_seg = 0; g.col0[0] = 0; g.din = h->aux.L[j].dkv; g.fk = g.fv = g.bk = g.bv = 0;
+    for (int i = 0; i < base->n_layers; ++i) {
+      if (layer_map[i] != j) continue;
+      if (g.n_seg == MAX_PRED_SEG) { delete h; return KVP_ERR_UNSUPPORTED; }
+      g.base_layer[g.n_seg] = i;
+      g.col0[g.n_seg + 1] = g.col0[g.n_seg] + h->base.L[i].dkv;
+      ++g.n_seg;
+    }
+    int dout = g.col0[g.n_seg];
+    if (dout == 0) continue;
+    g.fk = take((size_t)dout * g.din * h->es);
+    g.fv = take((size_t)dout * g.din * h->es);
+    if (opt->predictor_bias) { g.bk = take((size_t)dout * 4); g.bv = take((size_t)dout * 4); }
+  }
+  h->packed_bytes = off;
+  add_model_slots(h, "aux", h->aux, j_max + 1, false);
+  add_model_slots(h, "base", h->base, base->n_layers, true);
+  for (int j = 0; j <= j_max; ++j) {
+    const PredGroup& g = h->groups[j];
+    for (int s = 0; s < g.n_seg; ++s) {
+      int i = g.base_layer[s], dout = g.col0[s + 1] - g.col0[s];
+      char b[64];
+      snprintf(b, sizeof b, "pred.L%d.fk", i);
+      h->slots[b] = PackSlot{g.fk + (size_t)g.col0[s] * g.din * h->es, dout, g.din, opt->dtype, RowMap{0, 0, 0, 0}};
+      snprintf(b, sizeof b, "pred.L%d.fv", i);
+      h->slots[b] = PackSlot{g.fv + (size_t)g.col0[s] * g.din * h->es, dout, g.din, opt->dtype, RowMap{0, 0, 0, 0}};
+      if (opt->predictor_bias) {
+        snprintf(b, sizeof b, "pred.L%d.bk", i);
+        h->slots[b] = PackSlot{g.bk + (size_t)g.col0[s] * 4, 1, dout, 0, RowMap{0, 0, 0, 0}};
+        snprintf(b, sizeof b, "pred.L%d.bv", i);
+        h->slots[b] = PackSlot{g.bv + (size_t)g.col0[s] * 4, 1, dout, 0, RowMap{0, 0, 0, 0}};
+      }
+    }
+  }
+  char last[32];
+  snprintf(last, sizeof last, "aux.L%d.", j_max);
+  for (auto& kv : h->slots) {
+    const std::string& n = kv.first;
+    bool is_kv = ends_with(n, ".wk") || ends_with(n, ".wv");
+    bool base_kv = n.rfind("base.L", 0) == 0 && is_kv;
+    // in the last mapped auxiliary layer only the attention norm and the K/V projections are live
+    bool aux_last_dead = n.rfind(last, 0) == 0 && !(ends_with(n, ".attn_norm") || is_kv);
+    if (aux_last_dead) continue;            // accepted if given, never required
+    (base_kv ? h->req_decode_extra : h->req_prefill).push_back(n);
+  }
+  *out = h;
+  return KVP_OK;
+}
+
+void kvp_destroy(kvp_handle* h) { delete h; }
+
+const char* kvp_last_error(const kvp_handle* h) { return h ? h->err.c_str() : "NULL handle"; }
+
+int64_t kvp_launch_count(const kvp_handle* h) { return h ? h->n_launch : 0; }
+
+kvp_status kvp_packed_weight_bytes(const kvp_handle* h, size_t* bytes) {
+  if (!h || !bytes) return KVP_ERR_INVALID_ARG;
+  *bytes = h->packed_bytes;
+  return KVP_OK;
+}
+
+kvp_status kvp_workspace_bytes(const kvp_handle* h, int32_t max_batch, int64_t max_total_tokens, size_t* bytes) {
+  if (!h || !bytes || max_batch <= 0 || max_batch > KVP_MAX_BATCH || max_total_tokens < max_batch) return KVP_ERR_INVALID_ARG;
+  *bytes = ws_layout(h, max_batch, max_total_tokens).total;
+  return KVP_OK;
+}
+
+kvp_status kvp_cache_layout(const kvp_handle* h, int32_t base_layer, size_t* bytes_per_page) {
+  if (!h || !bytes_per_page || base_layer < 0 || base_layer >= h->base.n_layers) return KVP_ERR_INVALID_ARG;
+  *bytes_per_page = (size_t)h->base.L[base_layer].dkv * PAGE_TOKENS * h->es;
+  return KVP_OK;
+}
+
+kvp_status kvp_load_weights(kvp_handle* h, const kvp_tensor* tensors, int32_t n, void* packed, size_t packed_bytes,
+                            void* stream) {
+  if (!h) return KVP_ERR_INVALID_ARG;
+  h->err.clear();
+  if (!tensors || n < 0 || !packed) return fail(h, KVP_ERR_INVALID_ARG, "NULL argument");
+  if (packed_bytes < h->packed_bytes || (uintptr_t)packed % 256)
+    return fail(h, KVP_ERR_WORKSPACE, "packed buffer needs %zu bytes, 256-byte aligned", h->packed_bytes);
+  // validate everything before launching anything
+  for (int t = 0; t < n; ++t) {
+    const kvp_tensor& T = tensors[t];
+    if (!T.name || !T.data) return fail(h, KVP_ERR_INVALID_ARG, "tensor %d has a NULL name or pointer", t);
+    auto it = h->slots.find(T.name);
+    if (it == h->slots.end()) {
+      // tensors of dead auxiliary layers / the unused auxiliary head are accepted and ignored
+      if (strncmp(T.name, "aux.", 4) == 0) continue;
+      return fail(h, KVP_ERR_SHAPE, "unknown tensor name '%s'", T.name);
+    }
+    const PackSlot& s = it->second;
+    if (T.dtype != KVP_F32 && T.dtype != KVP_BF16) return fail(h, KVP_ERR_INVALID_ARG, "tensor '%s': bad dtype", T.name);
+    bool ok = (s.rows == 1 && T.ndim == 1) ? (T.shape[0] == s.cols)
+                                           : (T.ndim == 2 && T.shape[0] == s.rows && T.shape[1] == s.cols);
+    if (!ok) return fail(h, KVP_ERR_SHAPE, "tensor '%s': expected [%d, %d]", T.name, s.rows, s.cols);
+  }
+  if (h->packed && h->packed != packed) { h->loaded.clear(); h->ready_prefill = h->ready_decode = false; }
+  h->packed = (char*)packed;
+  LaunchCtx ctx{(cudaStream_t)stream, &h->n_launch, nullptr, h->opt.dtype};
+  for (int t = 0; t < n; ++t) {
+    const kvp_tensor& T = tensors[t];
+    auto it = h->slots.find(T.name);
+    if (it == h->slots.end()) continue;
+    const PackSlot& s = it->second;
+    launch_pack_rows(ctx, T.data, T.dtype, h->packed + s.off, s.dst_dtype, s.rows, s.cols, s.map);
+    h->loaded.insert(T.name);
+  }
+  auto all = [&](const std::vector<std::string>& v) {
+    for (auto& nme : v) if (!h->loaded.count(nme)) return false;
+    return true;
+  };
+  h->ready_prefill = all(h->req_prefill);
+  h->ready_decode = h->ready_prefill && all(h->req_decode_extra);
+  return check_cuda(h, "kvp_load_weights");
+}
+
+kvp_status kvp_prefill_predict(kvp_handle* h, const int32_t* tokens, const int32_t* lengths, int32_t batch,
+                               const kvp_cache* cache, void* workspace, size_t workspace_bytes, float* logits_out,
+                               int32_t* first_token, void* stream) {
+  CallShape cs;
+  kvp_status st = common_checks(h, lengths, batch, cache, workspace, 0, &cs);
+  if (st != KVP_OK) return st;
+  if (!tokens || !logits_out) return fail(h, KVP_ERR_INVALID_ARG, "NULL argument");
+  if (!h->ready_prefill) return fail(h, KVP_ERR_NOT_LOADED, "kvp_load_weights has not supplied every required tensor");
+  WsLayout w = ws_layout(h, batch, cs.total);
+  if (workspace_bytes < w.total) return fail(h, KVP_ERR_WORKSPACE, "workspace needs %zu bytes, got %zu", w.total, workspace_bytes);
+  char* ws = (char*)workspace;
+  cudaStream_t s = (cudaStream_t)stream;
+  int* status = (int*)(ws + w.status);
+  LaunchCtx ctx{s, &h->n_launch, status, h->opt.dtype};
+  const ModelPlan& A = h->aux;
+  const char* P = h->packed;
+  const int T = cs.total, es = h->es;
+  cudaMemsetAsync(status, 0, 16, s);
+
+  int* cu_dev = (int*)(ws + w.cu);
+  int* tok_pos = (int*)(ws + w.tok_pos);
+  int* tok_slot = (int*)(ws + w.tok_slot);
+  int* last_idx = (int*)(ws + w.last_idx);
+  float* x = (float*)(ws + w.x);
+  char* hbuf = ws + w.h;
+  char* qkv = ws + w.qkv;
+  char* attn = ws + w.attn;
+  char* gu = ws + w.gu;
+  char* act = ws + w.act;
+
+  launch_build_index(ctx, cs.cu.data(), batch, T, cu_dev, tok_pos, tok_slot, last_idx, cache->block_table,
+                     cache->max_pages_per_seq, cache->n_pages, cache->seq_lens);
+  // ---- stage 1 + 2: auxiliary prefill, each layer's K/V pushed through the predictor ----
+  launch_embed(ctx, tokens, nullptr, T, P + A.embed, A.vocab, A.d, x);
+  for (int j = 0; j <= h->j_max; ++j) {
+    const LayerPlan& L = A.L[j];
+    const bool last = (j == h->j_max);   // only K and V of the last mapped layer are needed
+    launch_rmsnorm(ctx, x, (const float*)(P + L.attn_norm), A.eps, T, A.d, hbuf, h->opt.dtype);
+    GemmArgs g{};
+    g.A = hbuf; g.lda = A.d; g.M = T; g.K = A.d;
+    int col_begin = last ? L.dq : 0;
+    g.W = P + L.wqkv + (size_t)col_begin * A.d * es; g.ldw = A.d; g.N = L.nqkv - col_begin;
+    g.C = qkv + (size_t)col_begin * es; g.ldc = L.nqkv;
+    launch_gemm_simt(ctx, g, EPI_STORE);
+    launch_rope(ctx, qkv + (size_t)col_begin * es, L.nqkv, T, last ? L.nkv : L.nq + L.nkv, L.hd, tok_pos, A.theta);
+    // predictor: K_hat_i = K_A,j FK_i^T, V_hat_i = V_A,j FV_i^T for every base layer i with j_i = j
+    const PredGroup& pg = h->groups[j];
+    if (pg.n_seg > 0) {
+      for (int kv = 0; kv < 2; ++kv) {
+        GemmArgs p{};
+        p.A = qkv + (size_t)(L.dq + kv * L.dkv) * es; p.lda = L.nqkv; p.M = T; p.K = L.dkv;
+        p.W = P + (kv ? pg.fv : pg.fk); p.ldw = L.dkv; p.N = pg.col0[pg.n_seg];
+        p.paged.n_seg = pg.n_seg;
+        for (int sg = 0; sg <= pg.n_seg; ++sg) p.paged.col0[sg] = pg.col0[sg];
+        for (int sg = 0; sg < pg.n_seg; ++sg) {
+          int i = pg.base_layer[sg];
+          p.paged.n_kv[sg] = h->base.L[i].nkv;
+          p.paged.pool[sg] = kv ? cache->v_pools[i] : cache->k_pools[i];
+        }
+        p.paged.bias = h->opt.predictor_bias ? (const float*)(P + (kv ? pg.bv : pg.bk)) : nullptr;
+        p.paged.tok_slot = tok_slot;
+        p.paged.head_dim = h->base.L[0].hd;
+        launch_gemm_simt(ctx, p, EPI_PAGED);
+      }
+    }
+    if (last) break;
+    launch_attn_prefill_simt(ctx, qkv, L.nqkv, L.nq, L.nkv, L.hd, cu_dev, batch, T, attn, L.dq);
+    GemmArgs o{};
+    o.A = attn; o.lda = L.dq; o.W = P + L.wo; o.ldw = L.dq; o.M = T; o.N = A.d; o.K = L.dq; o.X = x; o.ldx = A.d;
+    launch_gemm_simt(ctx, o, EPI_RESID);
+    launch_rmsnorm(ctx, x, (const float*)(P + L.ffn_norm), A.eps, T, A.d, hbuf, h->opt.dtype);
+    GemmArgs f{};
+    f.A = hbuf; f.lda = A.d; f.W = P + L.wgu; f.ldw = A.d; f.M = T; f.N = 2 * L.ffn; f.K = A.d; f.C = gu; f.ldc = 2 * L.ffn;
+    launch_gemm_simt(ctx, f, EPI_STORE);
+    launch_swiglu(ctx, gu, T, L.ffn, L.G, act);
+    GemmArgs d{};
+    d.A = act; d.lda = L.ffn; d.W = P + L.wd; d.ldw = L.ffn; d.M = T; d.N = A.d; d.K = L.ffn; d.X = x; d.ldx = A.d;
+    launch_gemm_simt(ctx, d, EPI_RESID);
+  }
+  // ---- stage 3: one base step per sequence on its last prompt token ----
+  launch_embed(ctx, tokens, last_idx, batch, P + h->base.embed, h->base.vocab, h->base.d, (float*)(ws + w.xb));
+  for (int i = 0; i < h->base.n_layers; ++i) base_layer_step(h, ctx, i, cache, w, ws, batch, cs.max_len, false);
+  base_head(h, ctx, w, ws, batch, logits_out, first_token);
+  return check_cuda(h, "kvp_prefill_predict");
+}
+
+kvp_status kvp_prefill_predict_host(kvp_handle* h, const int32_t* tokens_host, const int32_t* lengths, int32_t batch,
+                                    const kvp_cache* cache, void* workspace, size_t workspace_bytes, float* logits_dev,
+                                    float* logits_host, int32_t* first_token_host, void* stream) {
+  CallShape cs;
+  kvp_status st = common_checks(h, lengths, batch, cache, workspace, 0, &cs);
+  if (st != KVP_OK) return st;
+  if (!tokens_host || !logits_dev || !first_token_host) return fail(h, KVP_ERR_INVALID_ARG, "NULL argument");
+  WsLayout w = ws_layout(h, batch, cs.total);
+  if (workspace_bytes < w.total) return fail(h, KVP_ERR_WORKSPACE, "workspace needs %zu bytes, got %zu", w.total, workspace_bytes);
+  char* ws = (char*)workspace;
+  cudaStream_t s = (cudaStream_t)stream;
+  int32_t* tok_dev = (int32_t*)(ws + w.tok_stage);
+  int32_t* first_dev = (int32_t*)(ws + w.first_stage);
+  if (cudaMemcpyAsync(tok_dev, tokens_host, (size_t)cs.total * 4, cudaMemcpyHostToDevice, s) != cudaSuccess)
+    return check_cuda(h, "token upload");
+  st = kvp_prefill_predict(h, tok_dev, lengths, batch, cache, workspace, workspace_bytes, logits_dev, first_dev, stream);
+  if (st != KVP_OK) return st;
+  if (logits_host)
+    cudaMemcpyAsync(logits_host, logits_dev, (size_t)batch * h->base.vocab * 4, cudaMemcpyDeviceToHost, s);
+  cudaMemcpyAsync(first_token_host, first_dev, (size_t)batch * 4, cudaMemcpyDeviceToHost, s);
+  if (cudaStreamSynchronize(s) != cudaSuccess) return check_cuda(h, "kvp_prefill_predict_host");
+  return check_cuda(h, "kvp_prefill_predict_host");
+}
+
+kvp_status kvp_decode_step(kvp_handle* h, const int32_t* tokens, const int32_t* lengths_host, int32_t batch,
+                           const kvp_cache* cache, void* workspace, size_t workspace_bytes, float* logits_out,
+                           int32_t* next_token, void* stream) {
+  CallShape cs;
+  kvp_status st = common_checks(h, lengths_host, batch, cache, workspace, 1, &cs);
+  if (st != KVP_OK) return st;
+  if (!tokens || !logits_out) return fail(h, KVP_ERR_INVALID_ARG, "NULL argument");
+  if (!h->ready_decode) return fail(h, KVP_ERR_NOT_LOADED, "kvp_load_weights has not supplied every required tensor");
+  WsLayout w = ws_layout(h, batch, batch);
+  if (workspace_bytes < w.total) return fail(h, KVP_ERR_WORKSPACE, "workspace needs %zu bytes, got %zu", w.total, workspace_bytes);
+  char* ws = (char*)workspace;
+  LaunchCtx ctx{(cudaStream_t)stream, &h->n_launch, (int*)(ws + w.status), h->opt.dtype};
+  launch_embed(ctx, tokens, nullptr, batch, h->packed + h->base.embed, h->base.vocab, h->base.d, (float*)(ws + w.xb));
+  for (int i = 0; i < h->base.n_layers; ++i) base_layer_step(h, ctx, i, cache, w, ws, batch, cs.max_len + 1, true);
+  base_head(h, ctx, w, ws, batch, logits_out, next_token);
+  launch_add_int(ctx, cache->seq_lens, batch, 1);
+  return check_cuda(h, "kvp_decode_step");
+}
+
+kvp_status kvp_poll_status(kvp_handle* h, void* workspace, void* stream) {
+  if (!h || !workspace) return KVP_ERR_INVALID_ARG;
+  h->err.clear();
+  cudaStream_t s = (cudaStream_t)stream;
+  int code = 0;
+  if (cudaStreamSynchronize(s) != cudaSuccess || cudaMemcpy(&code, workspace, 4, cudaMemcpyDeviceToHost) != cudaSuccess ||
+      cudaMemset(workspace, 0, 16) != cudaSuccess) {
+    cudaError_t e = cudaGetLastError();
+    return fail(h, KVP_ERR_CUDA, "kvp_poll_status: %s", cudaGetErrorString(e));
+  }
+  switch (code) {
+    case DEV_OK: return KVP_OK;
+    case DEV_TIMEOUT: return fail(h, KVP_ERR_TIMEOUT, "a device-side wait ran out");
+    case DEV_BAD_TOKEN: return fail(h, KVP_ERR_BAD_INDEX, "a token id was outside [0, vocab)");
+    case DEV_BAD_PAGE: return fail(h, KVP_ERR_BAD_INDEX, "a block-table entry was outside [0, n_pages)");
+    default: return fail(h, KVP_ERR_CUDA, "unknown device status %d", code);
+  }
+}
+
+}  // extern "C"

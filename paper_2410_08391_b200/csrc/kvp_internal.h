@@ -1,0 +1,66 @@
+// Host-side plan of the KV Prediction library: shapes, packed-weight offsets, workspace layout.
+#pragma once
+#include <stdint.h>
+
+#include <string>
+#include <unordered_map>
+#include <unordered_set>
+#include <vector>
+
+#include "../../include/kvp.h"
+#include "common.cuh"
+
+struct LayerPlan {
+  int nq, nkv, hd, ffn;
+  int dq, dkv, nqkv;   // nq*hd, nkv*hd, (nq + 2 nkv)*hd
+  int G;               // gate/up row interleave of the packed w_gate/w_up (0 = [gate; up])
+  size_t wqkv, wo, wgu, wd, attn_norm, ffn_norm;   // byte offsets into the packed buffer
+};
+
+struct ModelPlan {
+  int n_layers, d, vocab;
+  float theta, eps;
+  std::vector<LayerPlan> L;
+  size_t embed, final_norm, lm_head;
+  int max_nqkv, max_dq, max_ffn, max_group, max_nkv;
+};
+
+// All base layers predicted from one auxiliary layer: their FK (and FV) matrices are stored
+// one under the other so that one GEMM produces every predicted K (or V) of that group.
+struct PredGroup {
+  int n_seg;
+  int base_layer[MAX_PRED_SEG];
+  int col0[MAX_PRED_SEG + 1];
+  int din;
+  size_t fk, fv, bk, bv;
+};
+
+struct PackSlot {
+  size_t off;      // destination byte offset of row 0 / element 0
+  int rows, cols;  // expected source shape (rows = 1 for vectors)
+  int dst_dtype;   // 0 f32, 1 bf16
+  RowMap map;
+};
+
+struct WsLayout {
+  size_t status, cu, last_idx, tok_pos, tok_slot, x, h, qkv, attn, gu, act;
+  size_t xb, hb, qkvb, ab, actb, part, tok_stage, first_stage, total;
+};
+
+struct kvp_handle {
+  ModelPlan aux, base;
+  std::vector<int> map;
+  int j_max;
+  kvp_options opt;
+  int es;                               // element size of the run dtype
+  std::vector<PredGroup> groups;        // one per auxiliary layer 0..j_max
+  std::unordered_map<std::string, PackSlot> slots;
+  std::vector<std::string> req_prefill, req_decode_extra;
+  std::unordered_set<std::string> loaded;
+  bool ready_prefill = false, ready_decode = false;
+  size_t packed_bytes = 0;
+  char* packed = nullptr;
+  int device = 0;
+  int64_t n_launch = 0;
+  std::string err;
+};
