@@ -199,6 +199,23 @@ kvp_status kvp_poll_status(kvp_handle* h, void* workspace, void* stream);
 /* Number of kernels the handle launched since creation (for launch accounting). */
 int64_t kvp_launch_count(const kvp_handle* h);
 
+/* Instrumentation (not part of the method): per-kernel-class device timing.  While enabled,
+ * every kernel launch of the compute calls is bracketed by CUDA events on the call's stream.
+ * kvp_timing_read() waits for the recorded events, adds their durations per class into
+ * ms[KVP_N_CLASSES] (host) and the launch counts into launches[KVP_N_CLASSES] (host), and
+ * forgets them.  Classes: the KVP_CLASS_* constants.  Events are owned by the handle. */
+enum {
+  KVP_CLASS_AUX_GEMM = 0,   /* auxiliary QKV / O / gate-up / down projections            */
+  KVP_CLASS_AUX_ATTN = 1,   /* auxiliary causal attention                                 */
+  KVP_CLASS_PREDICTOR = 2,  /* predictor GEMM writing the paged base cache                */
+  KVP_CLASS_STEP_GEMV = 3,  /* base step: weight-streaming projections and LM head        */
+  KVP_CLASS_STEP_ATTN = 4,  /* base step: attention over the paged cache                  */
+  KVP_CLASS_OTHER = 5,      /* norms, RoPE, SwiGLU, gathers, index, argmax                */
+  KVP_N_CLASSES = 6
+};
+kvp_status kvp_timing_enable(kvp_handle* h, int32_t on);
+kvp_status kvp_timing_read(kvp_handle* h, double* ms, int64_t* launches);
+
 #ifdef __cplusplus
 }
 #endif

@@ -185,20 +185,20 @@ void base_layer_step(kvp_handle* h, const LaunchCtx& ctx, int i, const kvp_cache
   float* qkvb = (float*)(ws + w.qkvb);
   float* ab = (float*)(ws + w.ab);
   float* actb = (float*)(ws + w.actb);
-  launch_rmsnorm(ctx, xb, (const float*)(P + L.attn_norm), B.eps, batch, B.d, hb, 0);
+  KVP_TIMED(KVP_CLASS_OTHER, launch_rmsnorm(ctx, xb, (const float*)(P + L.attn_norm), B.eps, batch, B.d, hb, 0));
   // the first step needs q only (keys and values are the predicted ones); generation needs q, k, v
   int n_out = generation ? L.nqkv : L.dq;
-  launch_step_gemv(ctx, P + L.wqkv, B.d, n_out, B.d, hb, B.d, batch, qkvb, n_out, GEMV_STORE, 0, 0);
+  KVP_TIMED(KVP_CLASS_STEP_GEMV, launch_step_gemv(ctx, P + L.wqkv, B.d, n_out, B.d, hb, B.d, batch, qkvb, n_out, GEMV_STORE, 0, 0));
   if (generation)
-    launch_step_append(ctx, qkvb, L.nq, L.nkv, L.hd, B.theta, cache->k_pools[i], cache->v_pools[i], cache->block_table,
-                       cache->max_pages_per_seq, cache->n_pages, cache->seq_lens, batch);
-  launch_step_attn(ctx, qkvb, n_out, L.nq, L.nkv, L.hd, B.theta, cache->k_pools[i], cache->v_pools[i], cache->block_table,
+    KVP_TIMED(KVP_CLASS_OTHER, launch_step_append(ctx, qkvb, L.nq, L.nkv, L.hd, B.theta, cache->k_pools[i], cache->v_pools[i], cache->block_table,
+                       cache->max_pages_per_seq, cache->n_pages, cache->seq_lens, batch));
+  KVP_TIMED(KVP_CLASS_STEP_ATTN, launch_step_attn(ctx, qkvb, n_out, L.nq, L.nkv, L.hd, B.theta, cache->k_pools[i], cache->v_pools[i], cache->block_table,
                    cache->max_pages_per_seq, cache->n_pages, cache->seq_lens, generation ? 1 : 0, batch, max_keys,
-                   (float*)(ws + w.part), ab);
-  launch_step_gemv(ctx, P + L.wo, L.dq, B.d, L.dq, ab, L.dq, batch, xb, B.d, GEMV_RESID, 0, 0);
-  launch_rmsnorm(ctx, xb, (const float*)(P + L.ffn_norm), B.eps, batch, B.d, hb, 0);
-  launch_step_gemv(ctx, P + L.wgu, B.d, L.ffn, B.d, hb, B.d, batch, actb, L.ffn, GEMV_SWIGLU, L.G, L.ffn);
-  launch_step_gemv(ctx, P + L.wd, L.ffn, B.d, L.ffn, actb, L.ffn, batch, xb, B.d, GEMV_RESID, 0, 0);
+                   (float*)(ws + w.part), ab));
+  KVP_TIMED(KVP_CLASS_STEP_GEMV, launch_step_gemv(ctx, P + L.wo, L.dq, B.d, L.dq, ab, L.dq, batch, xb, B.d, GEMV_RESID, 0, 0));
+  KVP_TIMED(KVP_CLASS_OTHER, launch_rmsnorm(ctx, xb, (const float*)(P + L.ffn_norm), B.eps, batch, B.d, hb, 0));
+  KVP_TIMED(KVP_CLASS_STEP_GEMV, launch_step_gemv(ctx, P + L.wgu, B.d, L.ffn, B.d, hb, B.d, batch, actb, L.ffn, GEMV_SWIGLU, L.G, L.ffn));
+  KVP_TIMED(KVP_CLASS_STEP_GEMV, launch_step_gemv(ctx, P + L.wd, L.ffn, B.d, L.ffn, actb, L.ffn, batch, xb, B.d, GEMV_RESID, 0, 0));
 }
 
 void base_head(kvp_handle* h, const LaunchCtx& ctx, const WsLayout& w, char* ws, int batch, float* logits,
@@ -207,9 +207,9 @@ void base_head(kvp_handle* h, const LaunchCtx& ctx, const WsLayout& w, char* ws,
   const char* P = h->packed;
   float* xb = (float*)(ws + w.xb);
   float* hb = (float*)(ws + w.hb);
-  launch_rmsnorm(ctx, xb, (const float*)(P + B.final_norm), B.eps, batch, B.d, hb, 0);
-  launch_step_gemv(ctx, P + B.lm_head, B.d, B.vocab, B.d, hb, B.d, batch, logits, B.vocab, GEMV_STORE, 0, 0);
-  if (token_out) launch_argmax(ctx, logits, batch, B.vocab, token_out);
+  KVP_TIMED(KVP_CLASS_OTHER, launch_rmsnorm(ctx, xb, (const float*)(P + B.final_norm), B.eps, batch, B.d, hb, 0));
+  KVP_TIMED(KVP_CLASS_STEP_GEMV, launch_step_gemv(ctx, P + B.lm_head, B.d, B.vocab, B.d, hb, B.d, batch, logits, B.vocab, GEMV_STORE, 0, 0));
+  if (token_out) KVP_TIMED(KVP_CLASS_OTHER, launch_argmax(ctx, logits, batch, B.vocab, token_out));
 }
 
 }  // namespace
@@ -423,21 +423,21 @@ kvp_status kvp_prefill_predict(kvp_handle* h, const int32_t* tokens, const int32
   char* gu = ws + w.gu;
   char* act = ws + w.act;
 
-  launch_build_index(ctx, cs.cu.data(), batch, T, cu_dev, tok_pos, tok_slot, last_idx, cache->block_table,
-                     cache->max_pages_per_seq, cache->n_pages, cache->seq_lens);
+  KVP_TIMED(KVP_CLASS_OTHER, launch_build_index(ctx, cs.cu.data(), batch, T, cu_dev, tok_pos, tok_slot, last_idx, cache->block_table,
+                     cache->max_pages_per_seq, cache->n_pages, cache->seq_lens));
   // ---- stage 1 + 2: auxiliary prefill, each layer's K/V pushed through the predictor ----
-  launch_embed(ctx, tokens, nullptr, T, P + A.embed, A.vocab, A.d, x);
+  KVP_TIMED(KVP_CLASS_OTHER, launch_embed(ctx, tokens, nullptr, T, P + A.embed, A.vocab, A.d, x));
   for (int j = 0; j <= h->j_max; ++j) {
     const LayerPlan& L = A.L[j];
     const bool last = (j == h->j_max);   // only K and V of the last mapped layer are needed
-    launch_rmsnorm(ctx, x, (const float*)(P + L.attn_norm), A.eps, T, A.d, hbuf, h->opt.dtype);
+    KVP_TIMED(KVP_CLASS_OTHER, launch_rmsnorm(ctx, x, (const float*)(P + L.attn_norm), A.eps, T, A.d, hbuf, h->opt.dtype));
     GemmArgs g{};
     g.A = hbuf; g.lda = A.d; g.M = T; g.K = A.d;
     int col_begin = last ? L.dq : 0;
     g.W = P + L.wqkv + (size_t)col_begin * A.d * es; g.ldw = A.d; g.N = L.nqkv - col_begin;
     g.C = qkv + (size_t)col_begin * es; g.ldc = L.nqkv;
-    launch_gemm_simt(ctx, g, EPI_STORE);
-    launch_rope(ctx, qkv + (size_t)col_begin * es, L.nqkv, T, last ? L.nkv : L.nq + L.nkv, L.hd, tok_pos, A.theta);
+    KVP_TIMED(KVP_CLASS_AUX_GEMM, launch_gemm_simt(ctx, g, EPI_STORE));
+    KVP_TIMED(KVP_CLASS_OTHER, launch_rope(ctx, qkv + (size_t)col_begin * es, L.nqkv, T, last ? L.nkv : L.nq + L.nkv, L.hd, tok_pos, A.theta));
     // predictor: K_hat_i = K_A,j FK_i^T, V_hat_i = V_A,j FV_i^T for every base layer i with j_i = j
     const PredGroup& pg = h->groups[j];
     if (pg.n_seg > 0) {
@@ -455,25 +455,25 @@ kvp_status kvp_prefill_predict(kvp_handle* h, const int32_t* tokens, const int32
         p.paged.bias = h->opt.predictor_bias ? (const float*)(P + (kv ? pg.bv : pg.bk)) : nullptr;
         p.paged.tok_slot = tok_slot;
         p.paged.head_dim = h->base.L[0].hd;
-        launch_gemm_simt(ctx, p, EPI_PAGED);
+        KVP_TIMED(KVP_CLASS_PREDICTOR, launch_gemm_simt(ctx, p, EPI_PAGED));
       }
     }
     if (last) break;
-    launch_attn_prefill_simt(ctx, qkv, L.nqkv, L.nq, L.nkv, L.hd, cu_dev, batch, T, attn, L.dq);
+    KVP_TIMED(KVP_CLASS_AUX_ATTN, launch_attn_prefill_simt(ctx, qkv, L.nqkv, L.nq, L.nkv, L.hd, cu_dev, batch, T, attn, L.dq));
     GemmArgs o{};
     o.A = attn; o.lda = L.dq; o.W = P + L.wo; o.ldw = L.dq; o.M = T; o.N = A.d; o.K = L.dq; o.X = x; o.ldx = A.d;
-    launch_gemm_simt(ctx, o, EPI_RESID);
-    launch_rmsnorm(ctx, x, (const float*)(P + L.ffn_norm), A.eps, T, A.d, hbuf, h->opt.dtype);
+    KVP_TIMED(KVP_CLASS_AUX_GEMM, launch_gemm_simt(ctx, o, EPI_RESID));
+    KVP_TIMED(KVP_CLASS_OTHER, launch_rmsnorm(ctx, x, (const float*)(P + L.ffn_norm), A.eps, T, A.d, hbuf, h->opt.dtype));
     GemmArgs f{};
     f.A = hbuf; f.lda = A.d; f.W = P + L.wgu; f.ldw = A.d; f.M = T; f.N = 2 * L.ffn; f.K = A.d; f.C = gu; f.ldc = 2 * L.ffn;
-    launch_gemm_simt(ctx, f, EPI_STORE);
-    launch_swiglu(ctx, gu, T, L.ffn, L.G, act);
+    KVP_TIMED(KVP_CLASS_AUX_GEMM, launch_gemm_simt(ctx, f, EPI_STORE));
+    KVP_TIMED(KVP_CLASS_OTHER, launch_swiglu(ctx, gu, T, L.ffn, L.G, act));
     GemmArgs d{};
     d.A = act; d.lda = L.ffn; d.W = P + L.wd; d.ldw = L.ffn; d.M = T; d.N = A.d; d.K = L.ffn; d.X = x; d.ldx = A.d;
-    launch_gemm_simt(ctx, d, EPI_RESID);
+    KVP_TIMED(KVP_CLASS_AUX_GEMM, launch_gemm_simt(ctx, d, EPI_RESID));
   }
   // ---- stage 3: one base step per sequence on its last prompt token ----
-  launch_embed(ctx, tokens, last_idx, batch, P + h->base.embed, h->base.vocab, h->base.d, (float*)(ws + w.xb));
+  KVP_TIMED(KVP_CLASS_OTHER, launch_embed(ctx, tokens, last_idx, batch, P + h->base.embed, h->base.vocab, h->base.d, (float*)(ws + w.xb)));
   for (int i = 0; i < h->base.n_layers; ++i) base_layer_step(h, ctx, i, cache, w, ws, batch, cs.max_len, false);
   base_head(h, ctx, w, ws, batch, logits_out, first_token);
   return check_cuda(h, "kvp_prefill_predict");
@@ -515,11 +515,35 @@ kvp_status kvp_decode_step(kvp_handle* h, const int32_t* tokens, const int32_t* 
   if (workspace_bytes < w.total) return fail(h, KVP_ERR_WORKSPACE, "workspace needs %zu bytes, got %zu", w.total, workspace_bytes);
   char* ws = (char*)workspace;
   LaunchCtx ctx{(cudaStream_t)stream, &h->n_launch, (int*)(ws + w.status), h->opt.dtype};
-  launch_embed(ctx, tokens, nullptr, batch, h->packed + h->base.embed, h->base.vocab, h->base.d, (float*)(ws + w.xb));
+  KVP_TIMED(KVP_CLASS_OTHER, launch_embed(ctx, tokens, nullptr, batch, h->packed + h->base.embed, h->base.vocab, h->base.d, (float*)(ws + w.xb)));
   for (int i = 0; i < h->base.n_layers; ++i) base_layer_step(h, ctx, i, cache, w, ws, batch, cs.max_len + 1, true);
   base_head(h, ctx, w, ws, batch, logits_out, next_token);
-  launch_add_int(ctx, cache->seq_lens, batch, 1);
+  KVP_TIMED(KVP_CLASS_OTHER, launch_add_int(ctx, cache->seq_lens, batch, 1));
   return check_cuda(h, "kvp_decode_step");
+}
+
+kvp_status kvp_timing_enable(kvp_handle* h, int32_t on) {
+  if (!h) return KVP_ERR_INVALID_ARG;
+  h->timing = on != 0;
+  return KVP_OK;
+}
+
+kvp_status kvp_timing_read(kvp_handle* h, double* ms, int64_t* launches) {
+  if (!h || !ms || !launches) return KVP_ERR_INVALID_ARG;
+  for (int c = 0; c < KVP_N_CLASSES; ++c) { ms[c] = 0.0; launches[c] = 0; }
+  for (auto& r : h->recs) {
+    float t = 0.f;
+    if (cudaEventSynchronize(r.b) != cudaSuccess || cudaEventElapsedTime(&t, r.a, r.b) != cudaSuccess) {
+      cudaError_t e = cudaGetLastError();
+      return fail(h, KVP_ERR_CUDA, "kvp_timing_read: %s", cudaGetErrorString(e));
+    }
+    ms[r.cls] += t;
+    launches[r.cls] += r.launches;
+    h->free_events.push_back(r.a);
+    h->free_events.push_back(r.b);
+  }
+  h->recs.clear();
+  return KVP_OK;
 }
 
 kvp_status kvp_poll_status(kvp_handle* h, void* workspace, void* stream) {

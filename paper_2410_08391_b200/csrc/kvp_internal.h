@@ -63,4 +63,31 @@ struct kvp_handle {
   int device = 0;
   int64_t n_launch = 0;
   std::string err;
+  // instrumentation
+  struct TimingRec { int cls; int64_t launches; cudaEvent_t a, b; };
+  bool timing = false;
+  std::vector<TimingRec> recs;
+  std::vector<cudaEvent_t> free_events;
+  ~kvp_handle() {
+    for (auto& r : recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+    for (auto e : free_events) cudaEventDestroy(e);
+  }
 };
+
+// Brackets the launches issued by `body` with events when instrumentation is on.
+struct TimedScope {
+  kvp_handle* h; cudaStream_t st; int cls; int64_t n0; cudaEvent_t a = nullptr, b = nullptr;
+  static cudaEvent_t get(kvp_handle* h) {
+    if (!h->free_events.empty()) { cudaEvent_t e = h->free_events.back(); h->free_events.pop_back(); return e; }
+    cudaEvent_t e = nullptr;
+    cudaEventCreate(&e);
+    return e;
+  }
+  TimedScope(kvp_handle* h_, cudaStream_t s, int c) : h(h_), st(s), cls(c), n0(h_->n_launch) {
+    if (h->timing) { a = get(h); b = get(h); cudaEventRecord(a, st); }
+  }
+  ~TimedScope() {
+    if (a) { cudaEventRecord(b, st); h->recs.push_back({cls, h->n_launch - n0, a, b}); }
+  }
+};
+#define KVP_TIMED(cls, stmt) do { TimedScope _ts(h, ctx.st, cls); stmt; } while (0)

@@ -1,0 +1,185 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same
+seeded inputs, element by element.  Sizes span several tiles and ragged tails."""
+import numpy as np
+import pytest
+
+import workloads as wl
+from oracle import kvp_oracle as orc
+from parity_util import GAP, TOL, compare_prefill, make_session, rel_fro
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    import __graft_entry__ as ge
+    ge.build()
+
+
+CASES = [
+    ("c1", None, "n002"),
+    ("c1", None, "fanin"),
+    ("c1_bf16", None, "n002"),
+    ("t_small", [150, 37, 1, 64, 65], "n002"),
+    ("t_small", [150, 37, 1, 64, 65], "fanin"),
+    ("t_small_f32", [150, 37, 1, 64, 65], "fanin"),
+    ("t_small_f32", [129], "n002"),
+    ("t_hd128", [130, 70, 2], "fanin"),
+    ("t_hd128", [200], "n002"),
+    ("t_scaled", [100, 33, 257], "fanin"),
+    ("t_scaled", [100, 33, 257], "n002"),
+    ("t_bias", [40, 90], "fanin"),
+]
+
+
+@pytest.mark.parametrize("name,lens,regime", CASES, ids=lambda v: str(v).replace(" ", ""))
+def test_prefill_predict_matches_oracle(name, lens, regime):
+    pair = wl.pair(name)
+    W = wl.make_weights(pair, seed=1, regime=regime)
+    pr = wl.prompts(name, seed=1) if lens is None else wl.custom_prompts(pair.base.vocab, lens, seed=1)
+    s = make_session(pair, W, pr)
+    try:
+        ek, ev, el, n = compare_prefill(s, pair, W, pr)
+        print(f"{name} {regime}: K {ek:.2e} V {ev:.2e} logits {el:.2e} argmax compared {n}/{pr.batch}")
+    finally:
+        s.close()
+
+
+@pytest.mark.parametrize("name,regime", [("t_small", "fanin"), ("t_small_f32", "fanin"), ("c1", "n002")])
+def test_decode_steps_match_oracle(name, regime):
+    import torch
+    pair = wl.pair(name)
+    W = wl.make_weights(pair, seed=2, regime=regime)
+    lens = [70, 63, 5] if name != "c1" else [64]
+    pr = wl.custom_prompts(pair.base.vocab, lens, seed=2)
+    steps = 3
+    s = make_session(pair, W, pr, extra_len=steps)
+    tol = TOL[pair.dtype]
+    try:
+        toks = torch.from_numpy(pr.tokens).to(s.device)
+        s.prefill_predict(toks, lens)
+        s.poll()
+        ref = orc.prefill_predict(pair, W, pr)
+        caches = {b: ref[b][0] for b in range(pr.batch)}
+        cur = list(lens)
+        g = np.random.default_rng(7)
+        for step in range(steps):
+            nxt = g.integers(0, pair.base.vocab, size=pr.batch).astype(np.int32)   # same forced token on both sides
+            logits, tok = s.decode_step(torch.from_numpy(nxt).to(s.device), cur)
+            s.poll()
+            logits = logits.cpu().numpy()
+            cur = [c + 1 for c in cur]
+            assert s.cache.seq_lens[:pr.batch].cpu().tolist() == cur
+            for b in range(pr.batch):
+                ref_logits, caches[b] = orc.decode_step(pair, W, int(nxt[b]), caches[b])
+                assert rel_fro(logits[b], ref_logits) <= tol
+                if orc.top2_gap(ref_logits) > GAP:
+                    assert int(tok[b]) == orc.argmax_lowest(ref_logits)
+                for i in range(pair.base.n_layers):
+                    k, v = s.cache.gather(i, b, cur[b])
+                    assert rel_fro(k[-1], caches[b][i][0][-1]) <= tol
+                    assert rel_fro(v[-1], caches[b][i][1][-1]) <= tol
+                    assert rel_fro(k, caches[b][i][0]) <= tol
+    finally:
+        s.close()
+
+
+def test_sequence_alone_equals_sequence_in_batch():
+    import torch
+    pair = wl.pair("t_small")
+    W = wl.make_weights(pair, seed=3, regime="fanin")
+    pr = wl.custom_prompts(pair.base.vocab, [90, 200, 17], seed=3)
+    s = make_session(pair, W, pr)
+    try:
+        lens = [int(x) for x in pr.lengths]
+        logits, first = s.prefill_predict(torch.from_numpy(pr.tokens).to(s.device), lens)
+        logits = logits.cpu().numpy().copy()
+        kv = [s.cache.gather(i, 1, lens[1]) for i in range(pair.base.n_layers)]
+        alone = wl.Prompts(pr.seq(1).copy(), np.array([lens[1]], np.int32))
+        l1, _ = s.prefill_predict(torch.from_numpy(alone.tokens).to(s.device), [lens[1]])
+        s.poll()
+        for i in range(pair.base.n_layers):
+            k, v = s.cache.gather(i, 0, lens[1])
+            np.testing.assert_array_equal(k, kv[i][0])      # the prefill kernels are row-independent
+            np.testing.assert_array_equal(v, kv[i][1])
+        assert rel_fro(l1.cpu().numpy()[0], logits[1].astype(np.float64)) <= 1e-5
+    finally:
+        s.close()
+
+
+def test_host_entry_point_matches_device_entry_point():
+    import torch
+    import paper_2410_08391_b200 as kvp
+    pair = wl.pair("t_small")
+    W = wl.make_weights(pair, seed=4)
+    pr = wl.custom_prompts(pair.base.vocab, [77, 130], seed=4)
+    s = make_session(pair, W, pr)
+    try:
+        lens = [int(x) for x in pr.lengths]
+        logits, first = s.prefill_predict(torch.from_numpy(pr.tokens).to(s.device), lens)
+        a, fa = logits.cpu().numpy().copy(), first.cpu().numpy().copy()
+        th = torch.from_numpy(pr.tokens).pin_memory()
+        lh = torch.empty((2, pair.base.vocab), dtype=torch.float32).pin_memory()
+        fh = torch.empty(2, dtype=torch.int32).pin_memory()
+        kvp.kvp_prefill_predict_host(s.h, th, lens, s.cache, s.workspace, s.logits, lh, fh, s.stream)
+        np.testing.assert_array_equal(lh.numpy(), a)
+        np.testing.assert_array_equal(fh.numpy(), fa)
+    finally:
+        s.close()
+
+
+def test_error_paths_report_status_and_keep_the_context_usable():
+    import torch
+    import paper_2410_08391_b200 as kvp
+    pair = wl.pair("t_small")
+    W = wl.make_weights(pair, seed=5)
+    pr = wl.custom_prompts(pair.base.vocab, [50, 20], seed=5)
+    s = make_session(pair, W, pr)
+    try:
+        lens = [50, 20]
+        toks = torch.from_numpy(pr.tokens).to(s.device)
+        with pytest.raises(kvp.KvpError) as e:                     # prompt longer than the block table allows
+            s.prefill_predict(toks, [65, 5])
+        assert e.value.status == -5
+        with pytest.raises(kvp.KvpError) as e:
+            s.prefill_predict(toks, [50, 0])
+        assert e.value.status == -1
+        small = torch.empty(1024, dtype=torch.uint8, device=s.device)
+        with pytest.raises(kvp.KvpError) as e:
+            kvp.kvp_prefill_predict(s.h, toks, lens, s.cache, small, s.logits, s.first, s.stream)
+        assert e.value.status == -8
+        bad = toks.clone()
+        bad[3] = pair.base.vocab + 5                               # token id out of range: flagged, not dereferenced
+        s.prefill_predict(bad, lens)
+        with pytest.raises(kvp.KvpError) as e:
+            s.poll()
+        assert e.value.status == -9
+        keep = s.cache.block_table.clone()
+        s.cache.block_table[1, 0] = s.cache.n_pages + 3            # page index out of range: flagged, write skipped
+        s.prefill_predict(toks, lens)
+        with pytest.raises(kvp.KvpError) as e:
+            s.poll()
+        assert e.value.status == -9
+        s.cache.block_table.copy_(keep)
+        s.prefill_predict(toks, lens)                              # and the handle still works afterwards
+        s.poll()
+        h2 = kvp.kvp_create(pair.aux, pair.base, pair.layer_map, pair.dtype)
+        with pytest.raises(kvp.KvpError) as e:
+            kvp.kvp_prefill_predict(h2, toks, lens, s.cache, s.workspace, s.logits, s.first, s.stream)
+        assert e.value.status == -4
+        kvp.kvp_destroy(h2)
+    finally:
+        s.close()
+
+
+def test_config_2_full_size_matches_oracle():
+    """The benchmark's own workload (1.1B-shaped base, 270M-shaped aux, 1024-token prompt)."""
+    pair = wl.pair("c2")
+    W = wl.make_weights(pair, seed=0)
+    pr = wl.prompts("c2", seed=0)
+    s = make_session(pair, W, pr)
+    try:
+        ek, ev, el, n = compare_prefill(s, pair, W, pr)
+        print(f"c2: K {ek:.2e} V {ev:.2e} logits {el:.2e} argmax compared {n}")
+    finally:
+        s.close()
