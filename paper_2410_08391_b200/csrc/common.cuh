@@ -69,13 +69,19 @@ __host__ __device__ __forceinline__ int map_row(const RowMap& m, int r) {
   return 2 * blk * m.G + m.which * gb + (r - blk * m.G);
 }
 
-enum GemmEpi : int { EPI_STORE = 0, EPI_RESID = 1, EPI_PAGED = 2 };
+enum GemmEpi : int { EPI_STORE = 0, EPI_RESID = 1, EPI_PAGED = 2, EPI_STORE32 = 3 };
 
+// bf16 mode carries the K/V path in split precision: a value v travels as hi = bf16(v) and
+// lo = bf16(v - hi), and a GEMM whose A operand has a lo part accumulates A_hi W^T + A_lo W^T.
+// The predicted cache is the product of the path and the base step's logits amplify its
+// error, so the operand roundings in front of it are removed where that is cheap.
 struct GemmArgs {
   const void* A; int lda;        // [M, K] run dtype
+  const void* A2; int lda2;      // optional lo part of A (same shape), or null
+  int split_begin;               // output columns >= split_begin use A + A2 (tile granularity)
   const void* W; int ldw;        // [N, K] run dtype
   int M, N, K;
-  void* C; int ldc;              // EPI_STORE: run dtype [M, N]
+  void* C; int ldc;              // EPI_STORE: run dtype [M, N]; EPI_STORE32: fp32 [M, N]
   float* X; int ldx;             // EPI_RESID: fp32 residual, X += A W^T
   PagedOut paged;                // EPI_PAGED
 };
@@ -96,9 +102,12 @@ void launch_build_index(const LaunchCtx&, const int* cu_host /*[B+1]*/, int batc
 void launch_embed(const LaunchCtx&, const int* tokens, const int* gather_idx, int n_rows,
                   const void* table, int vocab, int d, float* x);
 void launch_rmsnorm(const LaunchCtx&, const float* x, const float* gain, float eps, int rows, int d,
-                    void* out, int out_dtype);
-void launch_rope(const LaunchCtx&, void* qkv, int ld, int rows, int n_heads_rot, int head_dim,
-                 const int* tok_pos, float theta);
+                    void* out, int out_dtype, void* out_lo = nullptr);
+// fp32 projection output [rows, n_heads*hd] -> RoPE on the first n_heads_rot heads -> run dtype
+// `out` (row stride ld_out) and, for heads >= lo_head_begin, the bf16 lo part in `out_lo`.
+void launch_rope_split(const LaunchCtx&, const float* in, int ld_in, int rows, int n_heads, int n_heads_rot,
+                       int head_dim, const int* tok_pos, float theta, void* out, int ld_out,
+                       void* out_lo, int ld_lo, int lo_head_begin);
 void launch_swiglu(const LaunchCtx&, const void* gu, int rows, int ffn, int G, void* act);
 void launch_gemm_simt(const LaunchCtx&, const GemmArgs&, int epi);
 void launch_attn_prefill_simt(const LaunchCtx&, const void* qkv, int ld, int nq, int nkv, int hd,

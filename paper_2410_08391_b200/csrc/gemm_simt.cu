@@ -14,6 +14,7 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmArgs g) {
   const T* __restrict__ A = (const T*)g.A;
   const T* __restrict__ W = (const T*)g.W;
   int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+  const T* __restrict__ A2 = (g.A2 && n0 + BN > g.split_begin) ? (const T*)g.A2 : nullptr;
   int tid = threadIdx.x;
   int tx = tid & 15, ty = tid >> 4;
   float acc[4][4] = {};
@@ -23,7 +24,9 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmArgs g) {
     for (int i = 0; i < 4; ++i) {
       int k = k0 + lk + i;
       int am = m0 + lr, wn = n0 + lr;
-      As[lk + i][lr] = (am < g.M && k < g.K) ? to_f(A[(size_t)am * g.lda + k]) : 0.f;
+      float av = (am < g.M && k < g.K) ? to_f(A[(size_t)am * g.lda + k]) : 0.f;
+      if (A2 && am < g.M && k < g.K) av += to_f(A2[(size_t)am * g.lda2 + k]);
+      As[lk + i][lr] = av;
       Ws[lk + i][lr] = (wn < g.N && k < g.K) ? to_f(W[(size_t)wn * g.ldw + k]) : 0.f;
     }
     __syncthreads();
@@ -52,6 +55,8 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmArgs g) {
       float v = acc[i][j];
       if (EPI == EPI_STORE) {
         ((T*)g.C)[(size_t)m * g.ldc + n] = from_f<T>(v);
+      } else if (EPI == EPI_STORE32) {
+        ((float*)g.C)[(size_t)m * g.ldc + n] = v;
       } else if (EPI == EPI_RESID) {
         g.X[(size_t)m * g.ldx + n] += v;
       } else {
@@ -76,9 +81,9 @@ void launch_gemm_simt(const LaunchCtx& ctx, const GemmArgs& g, int epi) {
   ++*ctx.n_launch;
 #define GO(T, E) gemm_simt_kernel<T, E><<<grid, 256, 0, ctx.st>>>(g)
   if (ctx.dtype == 0) {
-    if (epi == EPI_STORE) GO(float, EPI_STORE); else if (epi == EPI_RESID) GO(float, EPI_RESID); else GO(float, EPI_PAGED);
+    if (epi == EPI_STORE) GO(float, EPI_STORE); else if (epi == EPI_RESID) GO(float, EPI_RESID); else if (epi == EPI_STORE32) GO(float, EPI_STORE32); else GO(float, EPI_PAGED);
   } else {
-    if (epi == EPI_STORE) GO(bf16, EPI_STORE); else if (epi == EPI_RESID) GO(bf16, EPI_RESID); else GO(bf16, EPI_PAGED);
+    if (epi == EPI_STORE) GO(bf16, EPI_STORE); else if (epi == EPI_RESID) GO(bf16, EPI_RESID); else if (epi == EPI_STORE32) GO(bf16, EPI_STORE32); else GO(bf16, EPI_PAGED);
   }
 #undef GO
 }

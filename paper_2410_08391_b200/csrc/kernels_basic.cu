@@ -114,7 +114,7 @@ void launch_embed(const LaunchCtx& ctx, const int* tokens, const int* gather_idx
 // ---------------------------------------------------------------------------------------
 template <class T>
 __global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restrict__ gain, float eps, int rows,
-                               int d, T* __restrict__ out) {
+                               int d, T* __restrict__ out, T* __restrict__ out_lo) {
   int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   int lane = threadIdx.x & 31;
   if (row >= rows) return;
@@ -123,50 +123,72 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restr
   for (int c = lane; c < d; c += 32) { float v = xr[c]; ss += v * v; }
   ss = warp_sum(ss);
   float r = rsqrtf(ss / (float)d + eps);
-  for (int c = lane; c < d; c += 32) out[(size_t)row * d + c] = from_f<T>(gain[c] * xr[c] * r);
-}
-
-void launch_rmsnorm(const LaunchCtx& ctx, const float* x, const float* gain, float eps, int rows, int d, void* out,
-                    int out_dtype) {
-  if (rows == 0) return;
-  LAUNCH_COUNT(ctx);
-  int grid = (rows + 7) / 8;
-  if (out_dtype == 0) rmsnorm_kernel<float><<<grid, 256, 0, ctx.st>>>(x, gain, eps, rows, d, (float*)out);
-  else rmsnorm_kernel<bf16><<<grid, 256, 0, ctx.st>>>(x, gain, eps, rows, d, (bf16*)out);
-}
-
-// ---------------------------------------------------------------------------------------
-// RoPE (rotate-half pairing) in place on the first n_heads_rot heads of each row
-// ---------------------------------------------------------------------------------------
-template <class T>
-__global__ void rope_kernel(T* __restrict__ qkv, int ld, int rows, int n_heads_rot, int hd,
-                            const int* __restrict__ tok_pos, const __grid_constant__ InvFreq inv) {
-  int half = hd >> 1;
-  size_t n = (size_t)rows * n_heads_rot * half;
-  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
-    int c = (int)(i % half);
-    size_t rh = i / half;
-    int h = (int)(rh % n_heads_rot);
-    int r = (int)(rh / n_heads_rot);
-    float sn, cs;
-    rope_sincos(tok_pos[r], inv.f[c], &sn, &cs);
-    T* p = qkv + (size_t)r * ld + (size_t)h * hd + c;
-    float x1 = to_f(p[0]), x2 = to_f(p[half]);
-    p[0] = from_f<T>(x1 * cs - x2 * sn);
-    p[half] = from_f<T>(x2 * cs + x1 * sn);
+  for (int c = lane; c < d; c += 32) {
+    float v = gain[c] * xr[c] * r;
+    T hi = from_f<T>(v);
+    out[(size_t)row * d + c] = hi;
+    if (out_lo) out_lo[(size_t)row * d + c] = from_f<T>(v - to_f(hi));
   }
 }
 
-void launch_rope(const LaunchCtx& ctx, void* qkv, int ld, int rows, int n_heads_rot, int hd, const int* tok_pos,
-                 float theta) {
-  size_t n = (size_t)rows * n_heads_rot * (hd / 2);
+void launch_rmsnorm(const LaunchCtx& ctx, const float* x, const float* gain, float eps, int rows, int d, void* out,
+                    int out_dtype, void* out_lo) {
+  if (rows == 0) return;
+  LAUNCH_COUNT(ctx);
+  int grid = (rows + 7) / 8;
+  if (out_dtype == 0) rmsnorm_kernel<float><<<grid, 256, 0, ctx.st>>>(x, gain, eps, rows, d, (float*)out, (float*)nullptr);
+  else rmsnorm_kernel<bf16><<<grid, 256, 0, ctx.st>>>(x, gain, eps, rows, d, (bf16*)out, (bf16*)out_lo);
+}
+
+// ---------------------------------------------------------------------------------------
+// RoPE (rotate-half pairing) on an fp32 projection output, then the store in the run dtype;
+// K and V heads also leave their bf16 rounding remainder (lo part) for the predictor.
+// ---------------------------------------------------------------------------------------
+template <class T>
+__global__ void rope_split_kernel(const float* __restrict__ in, int ld_in, int rows, int n_heads, int n_heads_rot,
+                                  int hd, const int* __restrict__ tok_pos, const __grid_constant__ InvFreq inv,
+                                  T* __restrict__ out, int ld_out, T* __restrict__ out_lo, int ld_lo,
+                                  int lo_head_begin) {
+  int half = hd >> 1;
+  size_t n = (size_t)rows * n_heads * half;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+    int c = (int)(i % half);
+    size_t rh = i / half;
+    int h = (int)(rh % n_heads);
+    int r = (int)(rh / n_heads);
+    const float* p = in + (size_t)r * ld_in + (size_t)h * hd + c;
+    float y1 = p[0], y2 = p[half];
+    if (h < n_heads_rot) {
+      float sn, cs;
+      rope_sincos(tok_pos[r], inv.f[c], &sn, &cs);
+      float x1 = y1, x2 = y2;
+      y1 = x1 * cs - x2 * sn;
+      y2 = x2 * cs + x1 * sn;
+    }
+    T h1 = from_f<T>(y1), h2 = from_f<T>(y2);
+    T* o = out + (size_t)r * ld_out + (size_t)h * hd + c;
+    o[0] = h1; o[half] = h2;
+    if (out_lo && h >= lo_head_begin) {
+      T* l = out_lo + (size_t)r * ld_lo + (size_t)(h - lo_head_begin) * hd + c;
+      l[0] = from_f<T>(y1 - to_f(h1));
+      l[half] = from_f<T>(y2 - to_f(h2));
+    }
+  }
+}
+
+void launch_rope_split(const LaunchCtx& ctx, const float* in, int ld_in, int rows, int n_heads, int n_heads_rot, int hd,
+                       const int* tok_pos, float theta, void* out, int ld_out, void* out_lo, int ld_lo,
+                       int lo_head_begin) {
+  size_t n = (size_t)rows * n_heads * (hd / 2);
   if (n == 0) return;
   InvFreq inv;
   fill_inv_freq(&inv, hd, theta);
   int grid = grid_for(n, 256);
   LAUNCH_COUNT(ctx);
-  if (ctx.dtype == 0) rope_kernel<float><<<grid, 256, 0, ctx.st>>>((float*)qkv, ld, rows, n_heads_rot, hd, tok_pos, inv);
-  else rope_kernel<bf16><<<grid, 256, 0, ctx.st>>>((bf16*)qkv, ld, rows, n_heads_rot, hd, tok_pos, inv);
+  if (ctx.dtype == 0)
+    rope_split_kernel<float><<<grid, 256, 0, ctx.st>>>(in, ld_in, rows, n_heads, n_heads_rot, hd, tok_pos, inv, (float*)out, ld_out, (float*)nullptr, 0, 0);
+  else
+    rope_split_kernel<bf16><<<grid, 256, 0, ctx.st>>>(in, ld_in, rows, n_heads, n_heads_rot, hd, tok_pos, inv, (bf16*)out, ld_out, (bf16*)out_lo, ld_lo, lo_head_begin);
 }
 
 // ---------------------------------------------------------------------------------------

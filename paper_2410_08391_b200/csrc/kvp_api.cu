@@ -49,7 +49,7 @@ const char* unsupported_model(const kvp_model_cfg* m) {
 
 void plan_model(ModelPlan& p, const kvp_model_cfg* m, int es, bool bf16_mode, size_t& off, bool with_head) {
   p.n_layers = m->n_layers; p.d = m->d_model; p.vocab = m->vocab; p.theta = m->rope_theta; p.eps = m->rms_eps;
-  p.max_nqkv = p.max_dq = p.max_ffn = p.max_group = p.max_nkv = 0;
+  p.max_nqkv = p.max_dq = p.max_dkv = p.max_ffn = p.max_group = p.max_nkv = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
   p.embed = take((size_t)m->vocab * m->d_model * es);
   p.L.resize(m->n_layers);
@@ -67,7 +67,7 @@ void plan_model(ModelPlan& p, const kvp_model_cfg* m, int es, bool bf16_mode, si
     L.ffn_norm = take((size_t)p.d * 4);
     p.max_nqkv = std::max(p.max_nqkv, L.nqkv); p.max_dq = std::max(p.max_dq, L.dq);
     p.max_ffn = std::max(p.max_ffn, L.ffn); p.max_group = std::max(p.max_group, L.nq / L.nkv);
-    p.max_nkv = std::max(p.max_nkv, L.nkv);
+    p.max_nkv = std::max(p.max_nkv, L.nkv); p.max_dkv = std::max(p.max_dkv, L.dkv);
   }
   p.final_norm = p.lm_head = 0;
   if (with_head) {
@@ -111,7 +111,10 @@ WsLayout ws_layout(const kvp_handle* h, int64_t Bm, int64_t Tm) {
   w.tok_slot = take(Tm * 4);
   w.x = take(Tm * A.d * 4);
   w.h = take(Tm * A.d * es);
+  w.h_lo = take(Tm * A.d * es);
   w.qkv = take(Tm * A.max_nqkv * es);
+  w.qkv32 = take(Tm * A.max_nqkv * 4);
+  w.kv_lo = take(Tm * 2 * (size_t)A.max_dkv * es);
   w.attn = take(Tm * A.max_dq * es);
   w.gu = take(Tm * 2 * (size_t)A.max_ffn * es);
   w.act = take(Tm * (size_t)A.max_ffn * es);
@@ -419,6 +422,10 @@ kvp_status kvp_prefill_predict(kvp_handle* h, const int32_t* tokens, const int32
   float* x = (float*)(ws + w.x);
   char* hbuf = ws + w.h;
   char* qkv = ws + w.qkv;
+  const bool split = h->opt.dtype == KVP_BF16;   // K/V path in hi + lo bf16 parts
+  char* h_lo = split ? ws + w.h_lo : nullptr;
+  char* kv_lo = split ? ws + w.kv_lo : nullptr;
+  float* qkv32 = (float*)(ws + w.qkv32);
   char* attn = ws + w.attn;
   char* gu = ws + w.gu;
   char* act = ws + w.act;
@@ -430,20 +437,27 @@ kvp_status kvp_prefill_predict(kvp_handle* h, const int32_t* tokens, const int32
   for (int j = 0; j <= h->j_max; ++j) {
     const LayerPlan& L = A.L[j];
     const bool last = (j == h->j_max);   // only K and V of the last mapped layer are needed
-    KVP_TIMED(KVP_CLASS_OTHER, launch_rmsnorm(ctx, x, (const float*)(P + L.attn_norm), A.eps, T, A.d, hbuf, h->opt.dtype));
+    KVP_TIMED(KVP_CLASS_OTHER, launch_rmsnorm(ctx, x, (const float*)(P + L.attn_norm), A.eps, T, A.d, hbuf, h->opt.dtype, h_lo));
     GemmArgs g{};
     g.A = hbuf; g.lda = A.d; g.M = T; g.K = A.d;
+    g.A2 = h_lo; g.lda2 = A.d;
     int col_begin = last ? L.dq : 0;
+    g.split_begin = L.dq - col_begin;    // the K and V columns take the lo part of h as well
     g.W = P + L.wqkv + (size_t)col_begin * A.d * es; g.ldw = A.d; g.N = L.nqkv - col_begin;
-    g.C = qkv + (size_t)col_begin * es; g.ldc = L.nqkv;
-    KVP_TIMED(KVP_CLASS_AUX_GEMM, launch_gemm_simt(ctx, g, EPI_STORE));
-    KVP_TIMED(KVP_CLASS_OTHER, launch_rope(ctx, qkv + (size_t)col_begin * es, L.nqkv, T, last ? L.nkv : L.nq + L.nkv, L.hd, tok_pos, A.theta));
+    g.C = qkv32; g.ldc = g.N;
+    KVP_TIMED(KVP_CLASS_AUX_GEMM, launch_gemm_simt(ctx, g, EPI_STORE32));
+    {
+      int heads = g.N / L.hd, q_heads = last ? 0 : L.nq;
+      KVP_TIMED(KVP_CLASS_OTHER, launch_rope_split(ctx, qkv32, g.N, T, heads, q_heads + L.nkv, L.hd, tok_pos, A.theta,
+                                                   qkv + (size_t)col_begin * es, L.nqkv, kv_lo, 2 * L.dkv, q_heads));
+    }
     // predictor: K_hat_i = K_A,j FK_i^T, V_hat_i = V_A,j FV_i^T for every base layer i with j_i = j
     const PredGroup& pg = h->groups[j];
     if (pg.n_seg > 0) {
       for (int kv = 0; kv < 2; ++kv) {
         GemmArgs p{};
         p.A = qkv + (size_t)(L.dq + kv * L.dkv) * es; p.lda = L.nqkv; p.M = T; p.K = L.dkv;
+        if (split) { p.A2 = kv_lo + (size_t)(kv * L.dkv) * es; p.lda2 = 2 * L.dkv; p.split_begin = 0; }
         p.W = P + (kv ? pg.fv : pg.fk); p.ldw = L.dkv; p.N = pg.col0[pg.n_seg];
         p.paged.n_seg = pg.n_seg;
         for (int sg = 0; sg <= pg.n_seg; ++sg) p.paged.col0[sg] = pg.col0[sg];

@@ -22,7 +22,7 @@ struct ModelPlan {
   float theta, eps;
   std::vector<LayerPlan> L;
   size_t embed, final_norm, lm_head;
-  int max_nqkv, max_dq, max_ffn, max_group, max_nkv;
+  int max_nqkv, max_dq, max_dkv, max_ffn, max_group, max_nkv;
 };
 
 // All base layers predicted from one auxiliary layer: their FK (and FV) matrices are stored
@@ -43,7 +43,7 @@ struct PackSlot {
 };
 
 struct WsLayout {
-  size_t status, cu, last_idx, tok_pos, tok_slot, x, h, qkv, attn, gu, act;
+  size_t status, cu, last_idx, tok_pos, tok_slot, x, h, h_lo, qkv, qkv32, kv_lo, attn, gu, act;
   size_t xb, hb, qkvb, ab, actb, part, tok_stage, first_stage, total;
 };
 
