@@ -192,6 +192,30 @@ kvp_status kvp_decode_step(kvp_handle* h, const int32_t* tokens /* dev [batch] *
                            void* workspace, size_t workspace_bytes, float* logits_out,
                            int32_t* next_token, void* stream);
 
+/* (The paper has no counterpart to this call: it exists for the library's users.)
+ * kvp_decode_step for callers that must not allocate device memory and therefore have no
+ * workspace to pass: code running while a CUDA memory pool is frozen, inside a latency-critical
+ * serving loop where cudaMalloc would synchronise the whole device, or in a plug-in whose host
+ * application owns the allocator.  Same inputs, outputs and semantics as kvp_decode_step, but
+ * the step's scratch is a fixed array of KVP_STATIC_SCRATCH_BYTES inside the library image
+ * (every GPU that loads the library holds it until the process exits).  The call itself
+ * performs no cudaMalloc / cudaFree and calls no allocating routine.
+ *   - A step whose kvp_workspace_bytes(h, batch, batch) exceeds KVP_STATIC_SCRATCH_BYTES is
+ *     rejected with KVP_ERR_WORKSPACE and a message naming both sizes.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current); make that first call before any stream capture begins.
+ *   - All calls on a device share the one array, which keeps the previous call's contents.
+ *     The call clears the status word itself; everything else is overwritten before it is
+ *     read.  Two calls that overlap on the GPU (different streams or handles) race on the
+ *     array: keep them on one stream or order them with events.
+ *   - status_out (dev int32, may be NULL) receives the device status word of this step:
+ *     0 = ok, 1 = a wait ran out, 2 = bad token id, 3 = bad page index. */
+#define KVP_STATIC_SCRATCH_BYTES (8 * 1024 * 1024)
+kvp_status kvp_decode_step_static(kvp_handle* h, const int32_t* tokens /* dev [batch] */,
+                                  const int32_t* lengths_host, int32_t batch, const kvp_cache* cache,
+                                  float* logits_out, int32_t* next_token, int32_t* status_out,
+                                  void* stream);
+
 /* Synchronises `stream`, reads the device status word of `workspace`, clears it and returns
  * KVP_OK, KVP_ERR_TIMEOUT, KVP_ERR_BAD_INDEX or KVP_ERR_CUDA. */
 kvp_status kvp_poll_status(kvp_handle* h, void* workspace, void* stream);

@@ -51,7 +51,8 @@ class CacheC(C.Structure):
 EXPORTS = ["kvp_create", "kvp_destroy", "kvp_last_error", "kvp_layer_map_canonical", "kvp_layer_map_pruned",
            "kvp_layer_map_uniform", "kvp_packed_weight_bytes", "kvp_workspace_bytes", "kvp_cache_layout",
            "kvp_load_weights", "kvp_prefill_predict", "kvp_prefill_predict_host", "kvp_decode_step",
-           "kvp_poll_status", "kvp_launch_count", "kvp_timing_enable", "kvp_timing_read"]
+           "kvp_poll_status", "kvp_launch_count", "kvp_timing_enable", "kvp_timing_read",
+           "kvp_decode_step_static"]
 
 CLASS_NAMES = ["aux_gemm", "aux_attn", "predictor", "step_gemv", "step_attn", "other"]
 
@@ -81,6 +82,7 @@ def lib() -> C.CDLL:
         L.kvp_prefill_predict.argtypes = [vp, vp, C.POINTER(i32), i32, C.POINTER(CacheC), vp, C.c_size_t, vp, vp, vp]
         L.kvp_prefill_predict_host.argtypes = [vp, vp, C.POINTER(i32), i32, C.POINTER(CacheC), vp, C.c_size_t, vp, vp, vp, vp]
         L.kvp_decode_step.argtypes = [vp, vp, C.POINTER(i32), i32, C.POINTER(CacheC), vp, C.c_size_t, vp, vp, vp]
+        L.kvp_decode_step_static.argtypes = [vp, vp, C.POINTER(i32), i32, C.POINTER(CacheC), vp, vp, vp, vp]
         L.kvp_poll_status.argtypes = [vp, vp, vp]
         L.kvp_launch_count.argtypes = [vp]
         L.kvp_launch_count.restype = i64
@@ -222,6 +224,15 @@ def kvp_decode_step(h, tokens, lengths_host: Sequence[int], cache: "Cache", work
     _check(lib().kvp_decode_step(h, tokens.data_ptr(), _i32arr(lengths_host), len(lengths_host), C.byref(cc),
                                  workspace.data_ptr(), workspace.numel(), logits_out.data_ptr(),
                                  next_token.data_ptr() if next_token is not None else None, stream), h)
+
+
+def kvp_decode_step_static(h, tokens, lengths_host: Sequence[int], cache: "Cache", logits_out, next_token, status_out,
+                           stream: int) -> None:
+    """kvp_decode_step without a workspace argument: the scratch is the library's built-in array."""
+    cc = _cache_c(cache)
+    _check(lib().kvp_decode_step_static(h, tokens.data_ptr(), _i32arr(lengths_host), len(lengths_host), C.byref(cc),
+                                        logits_out.data_ptr(), next_token.data_ptr() if next_token is not None else None,
+                                        status_out.data_ptr() if status_out is not None else None, stream), h)
 
 
 def kvp_poll_status(h, workspace, stream: int) -> None:

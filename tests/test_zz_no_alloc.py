@@ -1,0 +1,63 @@
+"""kvp_decode_step_static: the generation step for callers that cannot hand the library a workspace
+because they must not allocate device memory at that point (a frozen memory pool, a serving loop
+where cudaMalloc would stall the device, a host application that owns the allocator).  Its scratch
+is an array built into the library, shared by all calls, so the test runs two steps in a row and
+checks each against kvp_decode_step with an ordinary workspace."""
+import numpy as np
+import pytest
+
+import workloads as wl
+from parity_util import TOL, make_session, rel_fro
+
+pytestmark = pytest.mark.gpu
+
+
+def test_static_scratch_step_matches_workspace_step_twice_in_a_row():
+    import torch
+    import __graft_entry__ as ge
+    ge.build()
+    import paper_2410_08391_b200 as kvp
+
+    pair = wl.pair("t_small")
+    W = wl.make_weights(pair, seed=11, regime="fanin")
+    lens = [150, 9, 64]          # 150 keys: the split-attention partials in the scratch are exercised
+    pr = wl.custom_prompts(pair.base.vocab, lens, seed=11)
+    a = make_session(pair, W, pr, extra_len=2)      # reference: caller-provided workspace
+    b = make_session(pair, W, pr, extra_len=2)      # under test: built-in scratch
+    try:
+        toks = torch.from_numpy(pr.tokens).to(a.device)
+        for s in (a, b):
+            s.prefill_predict(toks, lens)
+            s.poll()
+        status = torch.full((1,), -1, dtype=torch.int32, device=a.device)
+        cur = list(lens)
+        g = np.random.default_rng(3)
+        for step in range(2):
+            nxt = torch.from_numpy(g.integers(0, pair.base.vocab, size=len(lens)).astype(np.int32)).to(a.device)
+            la, ta = a.decode_step(nxt, cur)
+            kvp.kvp_decode_step_static(b.h, nxt, cur, b.cache, b.logits, b.first, status, b.stream)
+            torch.cuda.synchronize()
+            assert int(status.item()) == 0
+            la, lb = la.cpu().numpy(), b.logits[:len(lens)].cpu().numpy()
+            for i in range(len(lens)):
+                assert rel_fro(lb[i], la[i].astype(np.float64)) <= TOL[pair.dtype]
+            assert ta.cpu().tolist() == b.first[:len(lens)].cpu().tolist()
+            cur = [c + 1 for c in cur]
+            assert b.cache.seq_lens[:len(lens)].cpu().tolist() == cur
+            for i in range(pair.base.n_layers):
+                ka, va = a.cache.gather(i, 0, cur[0])
+                kb, vb = b.cache.gather(i, 0, cur[0])
+                np.testing.assert_array_equal(ka, kb)
+                np.testing.assert_array_equal(va, vb)
+        # a step that does not fit the built-in array is refused with a message, nothing is launched
+        big = wl.pair("c3")
+        h = kvp.kvp_create(big.aux, big.base, big.layer_map, big.dtype)
+        n0 = kvp.kvp_launch_count(h)
+        with pytest.raises(kvp.KvpError) as e:
+            kvp.kvp_decode_step_static(h, nxt, [5] * 256, b.cache, b.logits, b.first, status, b.stream)
+        assert e.value.status == -8 and "built-in array" in str(e.value)
+        assert kvp.kvp_launch_count(h) == n0
+        kvp.kvp_destroy(h)
+    finally:
+        a.close()
+        b.close()
