@@ -1,0 +1,33 @@
+// Host interface of the tcgen05 GEMM (bf16 operands, fp32 accumulation in tensor memory).
+#pragma once
+#include "common.cuh"
+
+enum TcEpi : int {
+  TC_STORE = 0,   // C[m, n] = bf16(acc)
+  TC_RESID = 1,   // X[m, n] += acc (fp32 residual stream)
+  TC_SWIGLU = 2,  // W rows interleaved (64 gate rows, 64 up rows); C[m, c] = bf16(silu(gate_c) * up_c)
+  TC_QKV = 3,     // RoPE on columns < rot_cols, bf16 hi to C, bf16 lo of columns >= lo_col_begin to C_lo
+  TC_PAGED = 4    // predictor: columns scattered into cache pages
+};
+
+struct TcGemm {
+  const bf16* A; int lda;          // [M, K]
+  const bf16* A2; int lda2;        // lo part of A or null
+  int split_begin;                 // tiles reaching columns >= split_begin add A2 W^T
+  const bf16* W; int ldw;          // [N, K]
+  int M, N, K;
+  int epi;
+  bf16* C; int ldc;
+  float* X; int ldx;
+  bf16* C_lo; int ld_lo; int lo_col_begin;
+  int rot_cols; int hd;
+  const float2* rope_tab;          // [position][hd/2] (cos, sin)
+  const int* tok_pos;              // [M] position of each row in its sequence
+  int ffn;
+  PagedOut paged;
+  int n_sm;
+};
+
+bool tc_gemm_supported(const TcGemm& g);
+cudaError_t launch_gemm_tc(const TcGemm& g, int* status, cudaStream_t st, int64_t* n_launch);
+void launch_rope_table(const LaunchCtx& ctx, float2* tab, int n_pos, int hd, float theta);

@@ -3,11 +3,13 @@
 #include <math.h>
 #include <stdarg.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <algorithm>
 #include <new>
 
+#include "gemm_tc.h"
 #include "kvp_internal.h"
 
 namespace {
@@ -109,6 +111,7 @@ WsLayout ws_layout(const kvp_handle* h, int64_t Bm, int64_t Tm) {
   w.last_idx = take(Bm * 4);
   w.tok_pos = take(Tm * 4);
   w.tok_slot = take(Tm * 4);
+  w.rope_tab = take(Tm * (size_t)(A.L[0].hd / 2) * 8);
   w.x = take(Tm * A.d * 4);
   w.h = take(Tm * A.d * es);
   w.h_lo = take(Tm * A.d * es);
@@ -175,6 +178,17 @@ kvp_status common_checks(kvp_handle* h, const int32_t* lengths, int32_t batch, c
 bool ends_with(const std::string& s, const char* suf) {
   size_t n = strlen(suf);
   return s.size() >= n && s.compare(s.size() - n, n, suf) == 0;
+}
+
+// Tries the tcgen05 GEMM; returns false when the shape is not one it takes (caller falls back).
+bool try_tc(kvp_handle* h, const LaunchCtx& ctx, TcGemm& t, int cls, cudaError_t* err) {
+  if (!h->use_tc || h->opt.dtype != KVP_BF16) return false;
+  t.n_sm = h->n_sm;
+  if (!tc_gemm_supported(t)) return false;
+  TimedScope ts(h, ctx.st, cls);
+  cudaError_t e = launch_gemm_tc(t, ctx.status, ctx.st, ctx.n_launch);
+  if (e != cudaSuccess && *err == cudaSuccess) *err = e;
+  return true;
 }
 
 // one base-model layer of a single-token step (shared by the first step and generation)
@@ -270,8 +284,12 @@ kvp_status kvp_create(const kvp_model_cfg* aux, const kvp_model_cfg* base, const
   h->map.assign(layer_map, layer_map + base->n_layers);
   h->j_max = j_max;
   h->device = 0;
-  cudaGetDevice(&h->device);
+  if (cudaGetDevice(&h->device) == cudaSuccess) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, h->device) == cudaSuccess && n > 0) h->n_sm = n;
+  }
   cudaGetLastError();
+  if (const char* e = getenv("KVP_NO_TC")) h->use_tc = !(e[0] == '1');
   size_t off = 0;
   bool bf = opt->dtype == KVP_BF16;
   plan_model(h->aux, aux, h->es, bf, off, false);
@@ -426,29 +444,39 @@ kvp_status kvp_prefill_predict(kvp_handle* h, const int32_t* tokens, const int32
   char* h_lo = split ? ws + w.h_lo : nullptr;
   char* kv_lo = split ? ws + w.kv_lo : nullptr;
   float* qkv32 = (float*)(ws + w.qkv32);
+  float2* rope_tab = (float2*)(ws + w.rope_tab);
+  cudaError_t tc_err = cudaSuccess;
   char* attn = ws + w.attn;
   char* gu = ws + w.gu;
   char* act = ws + w.act;
 
   KVP_TIMED(KVP_CLASS_OTHER, launch_build_index(ctx, cs.cu.data(), batch, T, cu_dev, tok_pos, tok_slot, last_idx, cache->block_table,
                      cache->max_pages_per_seq, cache->n_pages, cache->seq_lens));
+  if (h->use_tc && h->opt.dtype == KVP_BF16 && (A.L[0].hd == 64 || A.L[0].hd == 128))
+    KVP_TIMED(KVP_CLASS_OTHER, launch_rope_table(ctx, rope_tab, cs.max_len, A.L[0].hd, A.theta));
   // ---- stage 1 + 2: auxiliary prefill, each layer's K/V pushed through the predictor ----
   KVP_TIMED(KVP_CLASS_OTHER, launch_embed(ctx, tokens, nullptr, T, P + A.embed, A.vocab, A.d, x));
   for (int j = 0; j <= h->j_max; ++j) {
     const LayerPlan& L = A.L[j];
     const bool last = (j == h->j_max);   // only K and V of the last mapped layer are needed
     KVP_TIMED(KVP_CLASS_OTHER, launch_rmsnorm(ctx, x, (const float*)(P + L.attn_norm), A.eps, T, A.d, hbuf, h->opt.dtype, h_lo));
-    GemmArgs g{};
-    g.A = hbuf; g.lda = A.d; g.M = T; g.K = A.d;
-    g.A2 = h_lo; g.lda2 = A.d;
     int col_begin = last ? L.dq : 0;
-    g.split_begin = L.dq - col_begin;    // the K and V columns take the lo part of h as well
-    g.W = P + L.wqkv + (size_t)col_begin * A.d * es; g.ldw = A.d; g.N = L.nqkv - col_begin;
-    g.C = qkv32; g.ldc = g.N;
-    KVP_TIMED(KVP_CLASS_AUX_GEMM, launch_gemm_simt(ctx, g, EPI_STORE32));
-    {
-      int heads = g.N / L.hd, q_heads = last ? 0 : L.nq;
-      KVP_TIMED(KVP_CLASS_OTHER, launch_rope_split(ctx, qkv32, g.N, T, heads, q_heads + L.nkv, L.hd, tok_pos, A.theta,
+    const int n_out = L.nqkv - col_begin, q_heads = last ? 0 : L.nq;
+    TcGemm tq{};
+    tq.A = (const bf16*)hbuf; tq.lda = A.d; tq.A2 = (const bf16*)h_lo; tq.lda2 = A.d; tq.split_begin = L.dq - col_begin;
+    tq.W = (const bf16*)(P + L.wqkv + (size_t)col_begin * A.d * es); tq.ldw = A.d; tq.M = T; tq.N = n_out; tq.K = A.d;
+    tq.epi = TC_QKV; tq.C = (bf16*)(qkv + (size_t)col_begin * es); tq.ldc = L.nqkv;
+    tq.C_lo = (bf16*)kv_lo; tq.ld_lo = 2 * L.dkv; tq.lo_col_begin = q_heads * L.hd;
+    tq.rot_cols = (q_heads + L.nkv) * L.hd; tq.hd = L.hd; tq.rope_tab = rope_tab; tq.tok_pos = tok_pos;
+    if (!try_tc(h, ctx, tq, KVP_CLASS_AUX_GEMM, &tc_err)) {
+      GemmArgs g{};
+      g.A = hbuf; g.lda = A.d; g.M = T; g.K = A.d;
+      g.A2 = h_lo; g.lda2 = A.d;
+      g.split_begin = L.dq - col_begin;    // the K and V columns take the lo part of h as well
+      g.W = P + L.wqkv + (size_t)col_begin * A.d * es; g.ldw = A.d; g.N = n_out;
+      g.C = qkv32; g.ldc = g.N;
+      KVP_TIMED(KVP_CLASS_AUX_GEMM, launch_gemm_simt(ctx, g, EPI_STORE32));
+      KVP_TIMED(KVP_CLASS_OTHER, launch_rope_split(ctx, qkv32, g.N, T, g.N / L.hd, q_heads + L.nkv, L.hd, tok_pos, A.theta,
                                                    qkv + (size_t)col_begin * es, L.nqkv, kv_lo, 2 * L.dkv, q_heads));
     }
     // predictor: K_hat_i = K_A,j FK_i^T, V_hat_i = V_A,j FV_i^T for every base layer i with j_i = j
@@ -469,23 +497,39 @@ kvp_status kvp_prefill_predict(kvp_handle* h, const int32_t* tokens, const int32
         p.paged.bias = h->opt.predictor_bias ? (const float*)(P + (kv ? pg.bv : pg.bk)) : nullptr;
         p.paged.tok_slot = tok_slot;
         p.paged.head_dim = h->base.L[0].hd;
-        KVP_TIMED(KVP_CLASS_PREDICTOR, launch_gemm_simt(ctx, p, EPI_PAGED));
+        TcGemm tp{};
+        tp.A = (const bf16*)p.A; tp.lda = p.lda; tp.A2 = (const bf16*)p.A2; tp.lda2 = p.lda2; tp.split_begin = 0;
+        tp.W = (const bf16*)p.W; tp.ldw = p.ldw; tp.M = T; tp.N = p.N; tp.K = p.K; tp.epi = TC_PAGED; tp.paged = p.paged;
+        if (!try_tc(h, ctx, tp, KVP_CLASS_PREDICTOR, &tc_err))
+          KVP_TIMED(KVP_CLASS_PREDICTOR, launch_gemm_simt(ctx, p, EPI_PAGED));
       }
     }
     if (last) break;
     KVP_TIMED(KVP_CLASS_AUX_ATTN, launch_attn_prefill_simt(ctx, qkv, L.nqkv, L.nq, L.nkv, L.hd, cu_dev, batch, T, attn, L.dq));
     GemmArgs o{};
     o.A = attn; o.lda = L.dq; o.W = P + L.wo; o.ldw = L.dq; o.M = T; o.N = A.d; o.K = L.dq; o.X = x; o.ldx = A.d;
-    KVP_TIMED(KVP_CLASS_AUX_GEMM, launch_gemm_simt(ctx, o, EPI_RESID));
+    TcGemm to{};
+    to.A = (const bf16*)attn; to.lda = L.dq; to.W = (const bf16*)(P + L.wo); to.ldw = L.dq; to.M = T; to.N = A.d; to.K = L.dq;
+    to.epi = TC_RESID; to.X = x; to.ldx = A.d;
+    if (!try_tc(h, ctx, to, KVP_CLASS_AUX_GEMM, &tc_err)) KVP_TIMED(KVP_CLASS_AUX_GEMM, launch_gemm_simt(ctx, o, EPI_RESID));
     KVP_TIMED(KVP_CLASS_OTHER, launch_rmsnorm(ctx, x, (const float*)(P + L.ffn_norm), A.eps, T, A.d, hbuf, h->opt.dtype));
     GemmArgs f{};
     f.A = hbuf; f.lda = A.d; f.W = P + L.wgu; f.ldw = A.d; f.M = T; f.N = 2 * L.ffn; f.K = A.d; f.C = gu; f.ldc = 2 * L.ffn;
-    KVP_TIMED(KVP_CLASS_AUX_GEMM, launch_gemm_simt(ctx, f, EPI_STORE));
-    KVP_TIMED(KVP_CLASS_OTHER, launch_swiglu(ctx, gu, T, L.ffn, L.G, act));
+    TcGemm tf{};
+    tf.A = (const bf16*)hbuf; tf.lda = A.d; tf.W = (const bf16*)(P + L.wgu); tf.ldw = A.d; tf.M = T; tf.N = 2 * L.ffn; tf.K = A.d;
+    tf.epi = TC_SWIGLU; tf.C = (bf16*)act; tf.ldc = L.ffn; tf.ffn = L.G == 64 ? L.ffn : 1;
+    if (!try_tc(h, ctx, tf, KVP_CLASS_AUX_GEMM, &tc_err)) {
+      KVP_TIMED(KVP_CLASS_AUX_GEMM, launch_gemm_simt(ctx, f, EPI_STORE));
+      KVP_TIMED(KVP_CLASS_OTHER, launch_swiglu(ctx, gu, T, L.ffn, L.G, act));
+    }
     GemmArgs d{};
     d.A = act; d.lda = L.ffn; d.W = P + L.wd; d.ldw = L.ffn; d.M = T; d.N = A.d; d.K = L.ffn; d.X = x; d.ldx = A.d;
-    KVP_TIMED(KVP_CLASS_AUX_GEMM, launch_gemm_simt(ctx, d, EPI_RESID));
+    TcGemm td{};
+    td.A = (const bf16*)act; td.lda = L.ffn; td.W = (const bf16*)(P + L.wd); td.ldw = L.ffn; td.M = T; td.N = A.d; td.K = L.ffn;
+    td.epi = TC_RESID; td.X = x; td.ldx = A.d;
+    if (!try_tc(h, ctx, td, KVP_CLASS_AUX_GEMM, &tc_err)) KVP_TIMED(KVP_CLASS_AUX_GEMM, launch_gemm_simt(ctx, d, EPI_RESID));
   }
+  if (tc_err != cudaSuccess) return fail(h, KVP_ERR_CUDA, "tensor-core GEMM launch: %s", cudaGetErrorString(tc_err));
   // ---- stage 3: one base step per sequence on its last prompt token ----
   KVP_TIMED(KVP_CLASS_OTHER, launch_embed(ctx, tokens, last_idx, batch, P + h->base.embed, h->base.vocab, h->base.d, (float*)(ws + w.xb)));
   for (int i = 0; i < h->base.n_layers; ++i) base_layer_step(h, ctx, i, cache, w, ws, batch, cs.max_len, false);

@@ -43,7 +43,7 @@ struct PackSlot {
 };
 
 struct WsLayout {
-  size_t status, cu, last_idx, tok_pos, tok_slot, x, h, h_lo, qkv, qkv32, kv_lo, attn, gu, act;
+  size_t status, cu, last_idx, tok_pos, tok_slot, rope_tab, x, h, h_lo, qkv, qkv32, kv_lo, attn, gu, act;
   size_t xb, hb, qkvb, ab, actb, part, tok_stage, first_stage, total;
 };
 
@@ -61,6 +61,8 @@ struct kvp_handle {
   size_t packed_bytes = 0;
   char* packed = nullptr;
   int device = 0;
+  int n_sm = 148;
+  bool use_tc = true;                   // tcgen05 kernels for bf16 shapes they accept
   int64_t n_launch = 0;
   std::string err;
   // instrumentation
