@@ -9,6 +9,7 @@
 #include <algorithm>
 #include <new>
 
+#include "attn_tc.h"
 #include "gemm_tc.h"
 #include "kvp_internal.h"
 
@@ -505,7 +506,14 @@ kvp_status kvp_prefill_predict(kvp_handle* h, const int32_t* tokens, const int32
       }
     }
     if (last) break;
-    KVP_TIMED(KVP_CLASS_AUX_ATTN, launch_attn_prefill_simt(ctx, qkv, L.nqkv, L.nq, L.nkv, L.hd, cu_dev, batch, T, attn, L.dq));
+    if (h->use_tc && split && attn_tc_supported(L.hd, L.nqkv, qkv, L.dq, attn)) {
+      TimedScope ts(h, ctx.st, KVP_CLASS_AUX_ATTN);
+      cudaError_t e = launch_attn_tc((const bf16*)qkv, L.nqkv, T, L.nq, L.nkv, L.hd, cu_dev, batch, (bf16*)attn, L.dq,
+                                     ctx.status, ctx.st, ctx.n_launch);
+      if (e != cudaSuccess && tc_err == cudaSuccess) tc_err = e;
+    } else {
+      KVP_TIMED(KVP_CLASS_AUX_ATTN, launch_attn_prefill_simt(ctx, qkv, L.nqkv, L.nq, L.nkv, L.hd, cu_dev, batch, T, attn, L.dq));
+    }
     GemmArgs o{};
     o.A = attn; o.lda = L.dq; o.W = P + L.wo; o.ldw = L.dq; o.M = T; o.N = A.d; o.K = L.dq; o.X = x; o.ldx = A.d;
     TcGemm to{};
