@@ -52,7 +52,7 @@ class ClockSampler:
         self.proc = None
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                                          "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.t = threading.Thread(target=self._read, daemon=True)
             self.t.start()
         except Exception:
@@ -67,7 +67,7 @@ class ClockSampler:
             return None
         time.sleep(0.15)
         self.proc.terminate()
-        rows = [r for ts, r in self.rows if t0 - 0.05 <= ts <= t1 + 0.15 and len(r) >= 7] or [r for _, r in self.rows if len(r) >= 7]
+        rows = [r for ts, r in self.rows if t0 - 0.02 <= ts <= t1 + 0.05 and len(r) >= 7] or [r for _, r in self.rows if len(r) >= 7][-3:]
         if not rows:
             return None
         sm = [float(r[0]) for r in rows]
@@ -160,13 +160,13 @@ def main():
     def step():
         sess.prefill_predict(toks, lens)
 
+    sampler = ClockSampler(local) if rank == 0 else None
     for _ in range(args.warmup):
         step()
     sess.poll()
     # ---- timed region: K steps, device time by CUDA events on the launching stream ----
     stream = torch.cuda.current_stream()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sampler = ClockSampler(local) if rank == 0 else None
     n0 = kvp.kvp_launch_count(sess.h)
     barrier()
     t0 = time.time()

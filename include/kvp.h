@@ -167,7 +167,11 @@ kvp_status kvp_load_weights(kvp_handle* h, const kvp_tensor* tensors, int32_t n,
  *   cache              pools and block table as described above; seq_lens[b] <- L_b
  *   workspace     dev, 256-byte aligned, >= kvp_workspace_bytes(batch, sum(lengths))
  *   logits_out    dev  fp32 [batch, vocab]
- *   first_token   dev  int32 [batch], argmax of logits (lowest index on ties); may be NULL */
+ *   first_token   dev  int32 [batch], argmax of logits (lowest index on ties); may be NULL
+ * The first call with a given set of arguments (pointers, lengths, stream) records the kernel
+ * schedule into a CUDA graph owned by the handle; later calls with the same arguments replay it
+ * (the token values themselves may change between calls).  If `stream` is already being
+ * captured by the caller, the kernels are enqueued into the caller's capture instead. */
 kvp_status kvp_prefill_predict(kvp_handle* h, const int32_t* tokens, const int32_t* lengths,
                                int32_t batch, const kvp_cache* cache, void* workspace,
                                size_t workspace_bytes, float* logits_out, int32_t* first_token,

@@ -116,7 +116,8 @@ void launch_attn_prefill_simt(const LaunchCtx&, const void* qkv, int ld, int nq,
 // base single-token step
 enum StepGemvMode : int { GEMV_STORE = 0, GEMV_RESID = 1, GEMV_SWIGLU = 2 };
 void launch_step_gemv(const LaunchCtx&, const void* W, int ldw, int N, int K, const float* x, int ldx,
-                      int batch, float* y, int ldy, int mode, int G, int ffn);
+                      int batch, float* y, int ldy, int mode, int G, int ffn, const float* gain = nullptr,
+                      float eps = 0.f, float* scratch_h = nullptr);
 void launch_step_attn(const LaunchCtx&, const float* q, int ldq, int nq, int nkv, int hd, float theta,
                       const void* kpool, const void* vpool, const int* block_table,
                       int max_pages_per_seq, int n_pages, const int* seq_lens, int extra, int batch,

@@ -203,10 +203,10 @@ void base_layer_step(kvp_handle* h, const LaunchCtx& ctx, int i, const kvp_cache
   float* qkvb = (float*)(ws + w.qkvb);
   float* ab = (float*)(ws + w.ab);
   float* actb = (float*)(ws + w.actb);
-  KVP_TIMED(KVP_CLASS_OTHER, launch_rmsnorm(ctx, xb, (const float*)(P + L.attn_norm), B.eps, batch, B.d, hb, 0));
   // the first step needs q only (keys and values are the predicted ones); generation needs q, k, v
   int n_out = generation ? L.nqkv : L.dq;
-  KVP_TIMED(KVP_CLASS_STEP_GEMV, launch_step_gemv(ctx, P + L.wqkv, B.d, n_out, B.d, hb, B.d, batch, qkvb, n_out, GEMV_STORE, 0, 0));
+  KVP_TIMED(KVP_CLASS_STEP_GEMV, launch_step_gemv(ctx, P + L.wqkv, B.d, n_out, B.d, xb, B.d, batch, qkvb, n_out, GEMV_STORE, 0, 0,
+                                                  (const float*)(P + L.attn_norm), B.eps, hb));
   if (generation)
     KVP_TIMED(KVP_CLASS_OTHER, launch_step_append(ctx, qkvb, L.nq, L.nkv, L.hd, B.theta, cache->k_pools[i], cache->v_pools[i], cache->block_table,
                        cache->max_pages_per_seq, cache->n_pages, cache->seq_lens, batch));
@@ -214,8 +214,8 @@ void base_layer_step(kvp_handle* h, const LaunchCtx& ctx, int i, const kvp_cache
                    cache->max_pages_per_seq, cache->n_pages, cache->seq_lens, generation ? 1 : 0, batch, max_keys,
                    (float*)(ws + w.part), ab));
   KVP_TIMED(KVP_CLASS_STEP_GEMV, launch_step_gemv(ctx, P + L.wo, L.dq, B.d, L.dq, ab, L.dq, batch, xb, B.d, GEMV_RESID, 0, 0));
-  KVP_TIMED(KVP_CLASS_OTHER, launch_rmsnorm(ctx, xb, (const float*)(P + L.ffn_norm), B.eps, batch, B.d, hb, 0));
-  KVP_TIMED(KVP_CLASS_STEP_GEMV, launch_step_gemv(ctx, P + L.wgu, B.d, L.ffn, B.d, hb, B.d, batch, actb, L.ffn, GEMV_SWIGLU, L.G, L.ffn));
+  KVP_TIMED(KVP_CLASS_STEP_GEMV, launch_step_gemv(ctx, P + L.wgu, B.d, L.ffn, B.d, xb, B.d, batch, actb, L.ffn, GEMV_SWIGLU, L.G, L.ffn,
+                                                  (const float*)(P + L.ffn_norm), B.eps, hb));
   KVP_TIMED(KVP_CLASS_STEP_GEMV, launch_step_gemv(ctx, P + L.wd, L.ffn, B.d, L.ffn, actb, L.ffn, batch, xb, B.d, GEMV_RESID, 0, 0));
 }
 
@@ -225,8 +225,8 @@ void base_head(kvp_handle* h, const LaunchCtx& ctx, const WsLayout& w, char* ws,
   const char* P = h->packed;
   float* xb = (float*)(ws + w.xb);
   float* hb = (float*)(ws + w.hb);
-  KVP_TIMED(KVP_CLASS_OTHER, launch_rmsnorm(ctx, xb, (const float*)(P + B.final_norm), B.eps, batch, B.d, hb, 0));
-  KVP_TIMED(KVP_CLASS_STEP_GEMV, launch_step_gemv(ctx, P + B.lm_head, B.d, B.vocab, B.d, hb, B.d, batch, logits, B.vocab, GEMV_STORE, 0, 0));
+  KVP_TIMED(KVP_CLASS_STEP_GEMV, launch_step_gemv(ctx, P + B.lm_head, B.d, B.vocab, B.d, xb, B.d, batch, logits, B.vocab, GEMV_STORE, 0, 0,
+                                                  (const float*)(P + B.final_norm), B.eps, hb));
   if (token_out) KVP_TIMED(KVP_CLASS_OTHER, launch_argmax(ctx, logits, batch, B.vocab, token_out));
 }
 
@@ -291,6 +291,7 @@ kvp_status kvp_create(const kvp_model_cfg* aux, const kvp_model_cfg* base, const
   }
   cudaGetLastError();
   if (const char* e = getenv("KVP_NO_TC")) h->use_tc = !(e[0] == '1');
+  if (const char* e = getenv("KVP_NO_GRAPH")) h->use_graph = !(e[0] == '1');
   size_t off = 0;
   bool bf = opt->dtype == KVP_BF16;
   plan_model(h->aux, aux, h->es, bf, off, false);
@@ -415,9 +416,10 @@ kvp_status kvp_load_weights(kvp_handle* h, const kvp_tensor* tensors, int32_t n,
   return check_cuda(h, "kvp_load_weights");
 }
 
-kvp_status kvp_prefill_predict(kvp_handle* h, const int32_t* tokens, const int32_t* lengths, int32_t batch,
-                               const kvp_cache* cache, void* workspace, size_t workspace_bytes, float* logits_out,
-                               int32_t* first_token, void* stream) {
+// Enqueues every kernel of the time-to-first-token path on `stream` (validates first).
+static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int32_t* lengths, int32_t batch,
+                                 const kvp_cache* cache, void* workspace, size_t workspace_bytes, float* logits_out,
+                                 int32_t* first_token, void* stream) {
   CallShape cs;
   kvp_status st = common_checks(h, lengths, batch, cache, workspace, 0, &cs);
   if (st != KVP_OK) return st;
@@ -543,6 +545,80 @@ kvp_status kvp_prefill_predict(kvp_handle* h, const int32_t* tokens, const int32
   for (int i = 0; i < h->base.n_layers; ++i) base_layer_step(h, ctx, i, cache, w, ws, batch, cs.max_len, false);
   base_head(h, ctx, w, ws, batch, logits_out, first_token);
   return check_cuda(h, "kvp_prefill_predict");
+}
+
+// The schedule is a few hundred short kernels, so the host's launch cost would exceed the device
+// time.  The first call with a given set of arguments records the schedule into a CUDA graph;
+// later calls with the same arguments replay it (token values may change, they are read on the
+// device).  Everything baked into the kernels' parameters is part of the key.
+kvp_status kvp_prefill_predict(kvp_handle* h, const int32_t* tokens, const int32_t* lengths, int32_t batch,
+                               const kvp_cache* cache, void* workspace, size_t workspace_bytes, float* logits_out,
+                               int32_t* first_token, void* stream) {
+  cudaStream_t s = (cudaStream_t)stream;
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  bool graph_ok = h && h->use_graph && !h->timing && lengths && cache && cache->k_pools && cache->v_pools && batch > 0 &&
+                  batch <= KVP_MAX_BATCH && cudaStreamIsCapturing(s, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusNone;
+  if (!graph_ok) {
+    cudaGetLastError();
+    return prefill_direct(h, tokens, lengths, batch, cache, workspace, workspace_bytes, logits_out, first_token, stream);
+  }
+  std::vector<uint64_t> key;
+  key.reserve(12 + batch + 2 * h->base.n_layers);
+  key.push_back((uint64_t)(uintptr_t)tokens); key.push_back((uint64_t)batch);
+  key.push_back((uint64_t)(uintptr_t)workspace); key.push_back((uint64_t)workspace_bytes);
+  key.push_back((uint64_t)(uintptr_t)logits_out); key.push_back((uint64_t)(uintptr_t)first_token);
+  key.push_back((uint64_t)(uintptr_t)cache->block_table); key.push_back((uint64_t)(uintptr_t)cache->seq_lens);
+  key.push_back((uint64_t)cache->max_pages_per_seq); key.push_back((uint64_t)cache->n_pages);
+  key.push_back((uint64_t)(uintptr_t)h->packed); key.push_back((uint64_t)(uintptr_t)s);
+  for (int b = 0; b < batch; ++b) key.push_back((uint64_t)(uint32_t)lengths[b]);
+  for (int i = 0; i < h->base.n_layers; ++i) {
+    key.push_back((uint64_t)(uintptr_t)cache->k_pools[i]);
+    key.push_back((uint64_t)(uintptr_t)cache->v_pools[i]);
+  }
+  for (auto& g : h->graphs)
+    if (g.key == key) {
+      g.last_use = ++h->graph_clock;
+      h->err.clear();
+      if (cudaGraphLaunch(g.exec, s) != cudaSuccess) return check_cuda(h, "cudaGraphLaunch");
+      h->n_launch += g.launches;
+      return KVP_OK;
+    }
+  // record
+  int64_t n0 = h->n_launch;
+  if (cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+    cudaGetLastError();
+    return prefill_direct(h, tokens, lengths, batch, cache, workspace, workspace_bytes, logits_out, first_token, stream);
+  }
+  kvp_status st = prefill_direct(h, tokens, lengths, batch, cache, workspace, workspace_bytes, logits_out, first_token, stream);
+  cudaGraph_t graph = nullptr;
+  cudaError_t ce = cudaStreamEndCapture(s, &graph);
+  if (st != KVP_OK) {               // argument error: nothing was launched, drop the empty capture
+    if (graph) cudaGraphDestroy(graph);
+    cudaGetLastError();
+    h->n_launch = n0;
+    return st;
+  }
+  cudaGraphExec_t exec = nullptr;
+  if (ce != cudaSuccess || !graph || cudaGraphInstantiate(&exec, graph, 0) != cudaSuccess) {
+    if (graph) cudaGraphDestroy(graph);
+    cudaGetLastError();
+    h->n_launch = n0;
+    h->use_graph = false;           // this context cannot record: run directly from now on
+    return prefill_direct(h, tokens, lengths, batch, cache, workspace, workspace_bytes, logits_out, first_token, stream);
+  }
+  cudaGraphDestroy(graph);
+  int64_t launches = h->n_launch - n0;
+  h->n_launch = n0;
+  if (h->graphs.size() >= 8) {      // evict the least recently used schedule
+    size_t victim = 0;
+    for (size_t i = 1; i < h->graphs.size(); ++i) if (h->graphs[i].last_use < h->graphs[victim].last_use) victim = i;
+    cudaGraphExecDestroy(h->graphs[victim].exec);
+    h->graphs.erase(h->graphs.begin() + victim);
+  }
+  h->graphs.push_back({key, exec, launches, ++h->graph_clock});
+  if (cudaGraphLaunch(exec, s) != cudaSuccess) return check_cuda(h, "cudaGraphLaunch");
+  h->n_launch += launches;
+  return KVP_OK;
 }
 
 kvp_status kvp_prefill_predict_host(kvp_handle* h, const int32_t* tokens_host, const int32_t* lengths, int32_t batch,

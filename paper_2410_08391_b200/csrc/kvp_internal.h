@@ -65,6 +65,11 @@ struct kvp_handle {
   bool use_tc = true;                   // tcgen05 kernels for bf16 shapes they accept
   int64_t n_launch = 0;
   std::string err;
+  // captured kernel schedules of kvp_prefill_predict, keyed by every argument that is baked in
+  struct GraphEntry { std::vector<uint64_t> key; cudaGraphExec_t exec; int64_t launches; uint64_t last_use; };
+  std::vector<GraphEntry> graphs;
+  bool use_graph = true;
+  uint64_t graph_clock = 0;
   // instrumentation
   struct TimingRec { int cls; int64_t launches; cudaEvent_t a, b; };
   bool timing = false;
@@ -73,6 +78,7 @@ struct kvp_handle {
   ~kvp_handle() {
     for (auto& r : recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
     for (auto e : free_events) cudaEventDestroy(e);
+    for (auto& g : graphs) cudaGraphExecDestroy(g.exec);
   }
 };
 
