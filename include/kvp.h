@@ -239,7 +239,8 @@ enum {
   KVP_CLASS_STEP_GEMV = 3,  /* base step: weight-streaming projections and LM head        */
   KVP_CLASS_STEP_ATTN = 4,  /* base step: attention over the paged cache                  */
   KVP_CLASS_OTHER = 5,      /* norms, RoPE, SwiGLU, gathers, index, argmax                */
-  KVP_N_CLASSES = 6
+  KVP_CLASS_STEP_FUSED = 6, /* base step as one persistent kernel (batch <= 4)            */
+  KVP_N_CLASSES = 7
 };
 kvp_status kvp_timing_enable(kvp_handle* h, int32_t on);
 kvp_status kvp_timing_read(kvp_handle* h, double* ms, int64_t* launches);

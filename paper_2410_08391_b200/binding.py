@@ -54,7 +54,7 @@ EXPORTS = ["kvp_create", "kvp_destroy", "kvp_last_error", "kvp_layer_map_canonic
            "kvp_poll_status", "kvp_launch_count", "kvp_timing_enable", "kvp_timing_read",
            "kvp_decode_step_static"]
 
-CLASS_NAMES = ["aux_gemm", "aux_attn", "predictor", "step_gemv", "step_attn", "other"]
+CLASS_NAMES = ["aux_gemm", "aux_attn", "predictor", "step_gemv", "step_attn", "other", "step_fused"]
 
 _lib = None
 

@@ -12,6 +12,7 @@
 #include "attn_tc.h"
 #include "gemm_tc.h"
 #include "kvp_internal.h"
+#include "step_mega.h"
 
 namespace {
 
@@ -107,7 +108,7 @@ WsLayout ws_layout(const kvp_handle* h, int64_t Bm, int64_t Tm) {
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
   const ModelPlan &A = h->aux, &B = h->base;
   size_t es = h->es;
-  w.status = take(256);
+  w.status = take(16384);     // status word, barrier counter, argmax slots; from byte 256: optional phase trace
   w.cu = take((Bm + 1) * 4);
   w.last_idx = take(Bm * 4);
   w.tok_pos = take(Tm * 4);
@@ -219,6 +220,45 @@ void base_layer_step(kvp_handle* h, const LaunchCtx& ctx, int i, const kvp_cache
   KVP_TIMED(KVP_CLASS_STEP_GEMV, launch_step_gemv(ctx, P + L.wd, L.ffn, B.d, L.ffn, actb, L.ffn, batch, xb, B.d, GEMV_RESID, 0, 0));
 }
 
+// The whole base step (all layers, LM head, argmax) as one persistent kernel; false = not applicable.
+bool base_step_fused(kvp_handle* h, const LaunchCtx& ctx, const kvp_cache* cache, const WsLayout& w, char* ws, int batch,
+                     int max_keys, bool generation, const int* tokens, const int* gather_idx, float* logits,
+                     int32_t* token_out, cudaError_t* err) {
+  const ModelPlan& B = h->base;
+  int k_max = std::max(B.d, std::max(B.max_dq, B.max_ffn));
+  if (!h->use_mega || B.n_layers > MEGA_MAX_LAYERS || !step_mega_supported(batch, B.L[0].hd, k_max, B.max_group, h->es)) return false;
+  // bulk copies need 16-byte rows: every projection's row length must be a multiple of 16 bytes
+  for (int i = 0; i < B.n_layers; ++i)
+    if ((B.d * h->es) % 16 || (B.L[i].dq * h->es) % 16 || (B.L[i].ffn * h->es) % 16) return false;
+  const char* P = h->packed;
+  MegaParams p{};
+  p.n_layers = B.n_layers; p.d = B.d; p.vocab = B.vocab; p.hd = B.L[0].hd; p.batch = batch; p.generation = generation ? 1 : 0;
+  p.eps = B.eps;
+  fill_inv_freq(&p.inv, p.hd, B.theta);
+  p.tokens = tokens; p.gather_idx = gather_idx;
+  p.embed = P + B.embed; p.final_norm = (const float*)(P + B.final_norm); p.lm_head = P + B.lm_head;
+  p.block_table = cache->block_table; p.mpps = cache->max_pages_per_seq; p.n_pages = cache->n_pages; p.seq_lens = cache->seq_lens;
+  p.xb = (float*)(ws + w.xb); p.qkvb = (float*)(ws + w.qkvb); p.ab = (float*)(ws + w.ab); p.actb = (float*)(ws + w.actb);
+  p.part = (float*)(ws + w.part);
+  p.logits = logits; p.token_out = token_out; p.status = ctx.status;
+  p.trace = getenv("KVP_MEGA_TRACE") ? (long long*)((char*)ctx.status + 256) : nullptr;
+  int min_nkv = B.L[0].nkv;
+  for (int i = 0; i < B.n_layers; ++i) {
+    const LayerPlan& L = B.L[i];
+    MegaLayer& m = p.layers[i];
+    m.wqkv = P + L.wqkv; m.wo = P + L.wo; m.wgu = P + L.wgu; m.wd = P + L.wd;
+    m.attn_norm = (const float*)(P + L.attn_norm); m.ffn_norm = (const float*)(P + L.ffn_norm);
+    m.kpool = cache->k_pools[i]; m.vpool = cache->v_pools[i];
+    m.nq = L.nq; m.nkv = L.nkv; m.dq = L.dq; m.nqkv = L.nqkv; m.ffn = L.ffn; m.G = L.G;
+    min_nkv = std::min(min_nkv, L.nkv);
+  }
+  p.n_split = step_attn_splits(batch, min_nkv, max_keys);   // sized for the layer with the fewest kv heads
+  TimedScope ts(h, ctx.st, KVP_CLASS_STEP_FUSED);
+  cudaError_t e = launch_step_mega(p, h->opt.dtype, k_max, h->n_sm, ctx.st, ctx.n_launch);
+  if (e != cudaSuccess && *err == cudaSuccess) *err = e;
+  return true;
+}
+
 void base_head(kvp_handle* h, const LaunchCtx& ctx, const WsLayout& w, char* ws, int batch, float* logits,
                int32_t* token_out) {
   const ModelPlan& B = h->base;
@@ -292,6 +332,7 @@ kvp_status kvp_create(const kvp_model_cfg* aux, const kvp_model_cfg* base, const
   cudaGetLastError();
   if (const char* e = getenv("KVP_NO_TC")) h->use_tc = !(e[0] == '1');
   if (const char* e = getenv("KVP_NO_GRAPH")) h->use_graph = !(e[0] == '1');
+  if (const char* e = getenv("KVP_NO_MEGA")) h->use_mega = !(e[0] == '1');
   size_t off = 0;
   bool bf = opt->dtype == KVP_BF16;
   plan_model(h->aux, aux, h->es, bf, off, false);
@@ -541,9 +582,12 @@ static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int
   }
   if (tc_err != cudaSuccess) return fail(h, KVP_ERR_CUDA, "tensor-core GEMM launch: %s", cudaGetErrorString(tc_err));
   // ---- stage 3: one base step per sequence on its last prompt token ----
-  KVP_TIMED(KVP_CLASS_OTHER, launch_embed(ctx, tokens, last_idx, batch, P + h->base.embed, h->base.vocab, h->base.d, (float*)(ws + w.xb)));
-  for (int i = 0; i < h->base.n_layers; ++i) base_layer_step(h, ctx, i, cache, w, ws, batch, cs.max_len, false);
-  base_head(h, ctx, w, ws, batch, logits_out, first_token);
+  if (!base_step_fused(h, ctx, cache, w, ws, batch, cs.max_len, false, tokens, last_idx, logits_out, first_token, &tc_err)) {
+    KVP_TIMED(KVP_CLASS_OTHER, launch_embed(ctx, tokens, last_idx, batch, P + h->base.embed, h->base.vocab, h->base.d, (float*)(ws + w.xb)));
+    for (int i = 0; i < h->base.n_layers; ++i) base_layer_step(h, ctx, i, cache, w, ws, batch, cs.max_len, false);
+    base_head(h, ctx, w, ws, batch, logits_out, first_token);
+  }
+  if (tc_err != cudaSuccess) return fail(h, KVP_ERR_CUDA, "base step launch: %s", cudaGetErrorString(tc_err));
   return check_cuda(h, "kvp_prefill_predict");
 }
 
@@ -657,6 +701,12 @@ kvp_status kvp_decode_step(kvp_handle* h, const int32_t* tokens, const int32_t* 
   if (workspace_bytes < w.total) return fail(h, KVP_ERR_WORKSPACE, "workspace needs %zu bytes, got %zu", w.total, workspace_bytes);
   char* ws = (char*)workspace;
   LaunchCtx ctx{(cudaStream_t)stream, &h->n_launch, (int*)(ws + w.status), h->opt.dtype};
+  cudaError_t mega_err = cudaSuccess;
+  cudaMemsetAsync((int*)(ws + w.status) + 1, 0, 4, ctx.st);     // barrier counter of the persistent kernel
+  if (base_step_fused(h, ctx, cache, w, ws, batch, cs.max_len + 1, true, tokens, nullptr, logits_out, next_token, &mega_err)) {
+    if (mega_err != cudaSuccess) return fail(h, KVP_ERR_CUDA, "base step launch: %s", cudaGetErrorString(mega_err));
+    return check_cuda(h, "kvp_decode_step");
+  }
   KVP_TIMED(KVP_CLASS_OTHER, launch_embed(ctx, tokens, nullptr, batch, h->packed + h->base.embed, h->base.vocab, h->base.d, (float*)(ws + w.xb)));
   for (int i = 0; i < h->base.n_layers; ++i) base_layer_step(h, ctx, i, cache, w, ws, batch, cs.max_len + 1, true);
   base_head(h, ctx, w, ws, batch, logits_out, next_token);

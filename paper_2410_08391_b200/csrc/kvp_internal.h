@@ -69,6 +69,7 @@ struct kvp_handle {
   struct GraphEntry { std::vector<uint64_t> key; cudaGraphExec_t exec; int64_t launches; uint64_t last_use; };
   std::vector<GraphEntry> graphs;
   bool use_graph = true;
+  bool use_mega = true;                 // persistent kernel for the base step when it applies
   uint64_t graph_clock = 0;
   // instrumentation
   struct TimingRec { int cls; int64_t launches; cudaEvent_t a, b; };

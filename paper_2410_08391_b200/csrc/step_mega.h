@@ -1,0 +1,31 @@
+// Host interface of the persistent single-token step kernel.
+#pragma once
+#include "common.cuh"
+
+constexpr int MEGA_MAX_LAYERS = 64;
+
+struct MegaLayer {
+  const void *wqkv, *wo, *wgu, *wd;      // packed weights of the layer (run dtype)
+  const float *attn_norm, *ffn_norm;
+  void *kpool, *vpool;                   // cache pools of the layer
+  int nq, nkv, dq, nqkv, ffn, G;
+};
+
+struct MegaParams {
+  int n_layers, d, vocab, hd, batch, generation, n_split;
+  float eps;
+  InvFreq inv;
+  const int* tokens; const int* gather_idx;      // token of row b = tokens[gather_idx ? gather_idx[b] : b]
+  const void* embed; const float* final_norm; const void* lm_head;
+  const int* block_table; int mpps, n_pages;
+  int* seq_lens;
+  float *xb, *qkvb, *ab, *actb, *part;           // workspace: residual, projections, attention out, FFN act, partials
+  float* logits; int* token_out;
+  int stage_bytes, slot_bytes;                   // shared-memory plan (set by the launcher)
+  long long* trace;                              // optional: clock64 of CTA 0 around every barrier (debugging aid)
+  int* status;                                   // [0] status word, [1] barrier counter, +64 bytes: argmax slots
+  MegaLayer layers[MEGA_MAX_LAYERS];
+};
+
+bool step_mega_supported(int batch, int hd, int k_max, int max_group, int es);
+cudaError_t launch_step_mega(MegaParams p, int dtype, int k_max, int n_sm, cudaStream_t st, int64_t* n_launch);
