@@ -134,11 +134,19 @@ __device__ __forceinline__ void stream_fill(const MegaParams& p, WarpStream& ws,
   }
 }
 
+// Staged activations are stored permuted so that a warp's reads are bank-conflict free: within
+// every group of 256 elements, lane l's elements 8l..8l+3 sit at [4l, 4l+4) and 8l+4..8l+7 at
+// [128 + 4l, 128 + 4l + 4).  (Shared-memory bandwidth, not HBM, bounds these phases otherwise.)
+__device__ __forceinline__ int xs_index(int k) {
+  return (k & ~255) + ((k & 4) << 5) + (((k & 255) >> 3) << 2) + (k & 3);
+}
+__device__ __forceinline__ int xs_stride(int K) { return (K + 255) & ~255; }
+
 // 8 consecutive weights (16 bytes for bf16, 32 for fp32) times 8 activations, two partial sums
 template <class T> __device__ __forceinline__ float dot_w8(const unsigned char* w, const float* x);
 template <> __device__ __forceinline__ float dot_w8<bf16>(const unsigned char* w, const float* x) {
   const uint4 u = *reinterpret_cast<const uint4*>(w);
-  const float4 x0 = *reinterpret_cast<const float4*>(x), x1 = *reinterpret_cast<const float4*>(x + 4);
+  const float4 x0 = *reinterpret_cast<const float4*>(x), x1 = *reinterpret_cast<const float4*>(x + 128);
   float a = __uint_as_float(u.x << 16) * x0.x;
   float b = __uint_as_float(u.x & 0xffff0000u) * x0.y;
   a = fmaf(__uint_as_float(u.y << 16), x0.z, a);
@@ -151,7 +159,7 @@ template <> __device__ __forceinline__ float dot_w8<bf16>(const unsigned char* w
 }
 template <> __device__ __forceinline__ float dot_w8<float>(const unsigned char* w, const float* x) {
   const float4 w0 = *reinterpret_cast<const float4*>(w), w1 = *reinterpret_cast<const float4*>(w + 16);
-  const float4 x0 = *reinterpret_cast<const float4*>(x), x1 = *reinterpret_cast<const float4*>(x + 4);
+  const float4 x0 = *reinterpret_cast<const float4*>(x), x1 = *reinterpret_cast<const float4*>(x + 128);
   float a = w0.x * x0.x, b = w0.y * x0.y;
   a = fmaf(w0.z, x0.z, a); b = fmaf(w0.w, x0.w, b);
   a = fmaf(w1.x, x1.x, a); b = fmaf(w1.y, x1.y, b);
@@ -171,6 +179,7 @@ __device__ __forceinline__ void gemv_phase(const MegaParams& p, const GemvDesc g
   const int R = g.mode == GEMV_SWIGLU ? 2 : 1;
   const bool vec = (K % 8 == 0);
   const int slot_elems = ws.slot_bytes / (int)sizeof(T);
+  const int KS = xs_stride(K);
   float acc[BB], accu[BB];
 #pragma unroll
   for (int b = 0; b < BB; ++b) { acc[b] = 0.f; accu[b] = 0.f; }
@@ -195,16 +204,16 @@ __device__ __forceinline__ void gemv_phase(const MegaParams& p, const GemvDesc g
           float* a = which ? accu : acc;
           if (vec) {
 #pragma unroll 4
-            for (int e = lane * 8; e < ne; e += 256) {
+            for (int e = lane * 8; e < ne; e += 256) {   // k0 and e - 8 lane are multiples of 256
 #pragma unroll
-              for (int b = 0; b < BB; ++b) a[b] += dot_w8<T>(sp + (size_t)e * sizeof(T), xs + b * K + k0 + e);
+              for (int b = 0; b < BB; ++b) a[b] += dot_w8<T>(sp + (size_t)e * sizeof(T), xs + b * KS + k0 + (e - lane * 8) + lane * 4);
             }
           } else {
             const T* wp = reinterpret_cast<const T*>(sp);
             for (int e = lane; e < ne; e += 32) {
               float wv = to_f(wp[e]);
 #pragma unroll
-              for (int b = 0; b < BB; ++b) a[b] = fmaf(wv, xs[b * K + k0 + e], a[b]);
+              for (int b = 0; b < BB; ++b) a[b] = fmaf(wv, xs[b * KS + xs_index(k0 + e)], a[b]);
             }
           }
         }
@@ -243,6 +252,7 @@ template <int BB>
 __device__ __noinline__ void stage_x(const float* x, int ldx, int K, int batch, const float* gain, float eps, float* xs,
                                      float* red) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int KS = xs_stride(K);
   if (gain && K <= 8 * NT) {
     float v[BB][8];
     float ss[BB];
@@ -268,7 +278,7 @@ __device__ __noinline__ void stage_x(const float* x, int ldx, int K, int batch, 
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
         int k = tid + j * NT;
-        if (k < K) xs[b * K + k] = gain[k] * v[b][j] * r;
+        if (k < K) xs[b * KS + xs_index(k)] = gain[k] * v[b][j] * r;
       }
     }
   } else {
@@ -298,7 +308,7 @@ __device__ __noinline__ void stage_x(const float* x, int ldx, int K, int batch, 
     for (int k = tid; k < K; k += NT) {
       float g = gain ? gain[k] : 1.f;
 #pragma unroll
-      for (int b = 0; b < BB; ++b) xs[b * K + k] = b < batch ? g * __ldcg(x + (size_t)b * ldx + k) * r[b] : 0.f;
+      for (int b = 0; b < BB; ++b) xs[b * KS + xs_index(k)] = b < batch ? g * __ldcg(x + (size_t)b * ldx + k) * r[b] : 0.f;
     }
   }
   __syncthreads();
@@ -576,7 +586,7 @@ constexpr int SMEM_LIMIT = 227 * 1024 - 2048;   // dynamic shared memory we allo
 
 size_t stage_region_bytes(int batch, int hd, int k_max, int es) {
   int bb = batch <= 1 ? 1 : (batch == 2 ? 2 : 4);
-  size_t xs = (size_t)bb * k_max * 4;
+  size_t xs = (size_t)bb * ((k_max + 255) / 256 * 256) * 4;
   size_t at = (size_t)2 * PAGE_TOKENS * (hd * es + 16) + (size_t)(MAXG * hd + MAXG * PAGE_TOKENS + 3 * MAXG) * 4;
   size_t r = xs > at ? xs : at;
   return (r + 127) / 128 * 128;
@@ -609,7 +619,7 @@ cudaError_t launch_step_mega(MegaParams p, int dtype, int k_max, int n_sm, cudaS
   const int es = dtype == 0 ? 4 : 2;
   size_t stage = stage_region_bytes(p.batch, p.hd, k_max, es);
   int slot = (int)((SMEM_LIMIT - stage) / (NW * NSLOT));
-  slot = slot / 256 * 256;
+  slot = slot / 1024 * 1024;      // whole 256-element groups of either element size
   if (slot > 8192) slot = 8192;
   p.stage_bytes = (int)stage;
   p.slot_bytes = slot;
