@@ -1,12 +1,19 @@
 // Tensor-core GEMM for sm_100a:  D[M,N] = A[M,K] W[N,K]^T (+ A_lo W^T on split tiles), bf16
 // operands, fp32 accumulation in tensor memory.
 //
-// One persistent CTA per SM walks output tiles of 128 x 128.  Warp 0 feeds a 6-stage ring of
-// shared-memory operand tiles with TMA (128-byte swizzle, 64 k-elements per stage); warp 1
-// issues tcgen05.mma (one elected thread) into one of two 128-column accumulators in tensor
-// memory; warps 2-5 drain the other accumulator with tcgen05.ld and run the fused epilogue
+// One persistent CTA per SM walks output tiles of 128 x BN (BN = 256, or 128 when the problem
+// has too few wide tiles to fill the SMs).  Operand tiles travel through a ring of shared-
+// memory stages (128-byte swizzle, 64 k-elements per stage) filled by TMA.  A thread that
+// issues a tensor copy is held for a few hundred cycles per copy, which caps one issuing thread
+// at about 120 GB/s; a 128 x 256 tile needs 48 KiB per 512 tensor-pipe cycles (about 180 GB/s),
+// so the A and the W tile of a stage are issued by two different warps (0 and 2).  Warp 1
+// issues tcgen05.mma (one elected thread) into one of two BN-column accumulators in tensor
+// memory; warps 3-6 drain the other accumulator with tcgen05.ld and run the fused epilogue
 // (bf16 store / fp32 residual add / RoPE + hi-lo split / SwiGLU / scatter into cache pages),
 // so the epilogue of tile i overlaps the main loop of tile i+1.
+// Tiles are visited in groups of 16 row blocks so that a wave's A and W tiles stay in L2.
+// The residual GEMMs (x += A W^T) add with red.global, so when they have fewer tiles than
+// two per SM their k loops are cut into equal contiguous shares, one per CTA (stream-K).
 // Every mbarrier wait is bounded: on expiry the kernel records DEV_TIMEOUT, all roles leave
 // their loops, in-flight copies are given time to land, tensor memory is freed.
 #include <cuda.h>
@@ -18,11 +25,15 @@
 
 namespace {
 
-constexpr int BM = 128, BN = 128, BK = 64;
-constexpr int STAGES = 6;
-constexpr int STAGE_BYTES = (BM + BN) * BK * 2;          // 32 KiB
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
-constexpr int N_THREADS = 192;
+constexpr int BM = 128, BK = 64;
+constexpr int GROUP_M = 16;                                // row blocks per rasterisation group
+constexpr int N_THREADS = 224;                             // warps: 0 A loads, 1 MMA, 2 W loads, 3-6 epilogue
+template <int BN> struct Tile {
+  static constexpr int STAGES = BN == 256 ? 4 : 6;
+  static constexpr int A_BYTES = BM * BK * 2, W_BYTES = BN * BK * 2;
+  static constexpr int STAGE_BYTES = A_BYTES + W_BYTES;    // 48 KiB / 32 KiB
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+};
 constexpr uint32_t SPIN_LIMIT = 20u * 1000u * 1000u;      // ~1-2 s of polling
 
 // ---- PTX wrappers -------------------------------------------------------------------------
@@ -134,6 +145,7 @@ struct Params {
   int M, N, K;
   int split_begin;       // tiles with n0 + BN > split_begin run the k loop a second time over A2
   int has_a2;
+  int stream_k;          // residual GEMM only: CTAs take equal shares of all k blocks
   int* status;
   // epilogue
   bf16* C; int ldc;
@@ -145,8 +157,56 @@ struct Params {
   PagedOut paged;
 };
 
+// ---- work list: every role of a CTA walks the same sequence of (tile, k-block range) ---------
+struct Work { int m0, n0, kb0, kb1; };
+
+template <int BN>
+struct Sched {
+  int tiles_m, tiles_n, n_tiles, num_kb;
+  int tile;                 // tile mode: next tile of this CTA
+  long long g, g_end;       // stream-K mode: this CTA's share of the global k-block sequence
+  const Params& p;
+  __device__ __forceinline__ explicit Sched(const Params& p_) : p(p_) {
+    tiles_m = (p.M + BM - 1) / BM; tiles_n = (p.N + BN - 1) / BN;
+    n_tiles = tiles_m * tiles_n;
+    num_kb = (p.K + BK - 1) / BK;
+    tile = blockIdx.x;
+    long long total = (long long)n_tiles * num_kb;
+    g = total * blockIdx.x / gridDim.x;
+    g_end = total * (blockIdx.x + 1) / gridDim.x;
+  }
+  __device__ __forceinline__ void coords(int t, Work& w) const {
+    const int per_group = GROUP_M * tiles_n;
+    const int grp = t / per_group, r = t - grp * per_group;
+    const int gm = min(GROUP_M, tiles_m - grp * GROUP_M);
+    w.m0 = (grp * GROUP_M + r % gm) * BM;
+    w.n0 = (r / gm) * BN;
+  }
+  __device__ __forceinline__ bool next(Work& w) {
+    if (p.stream_k) {
+      if (g >= g_end) return false;
+      const int t = (int)(g / num_kb);
+      coords(t, w);
+      w.kb0 = (int)(g - (long long)t * num_kb);
+      w.kb1 = (int)min((long long)num_kb, w.kb0 + (g_end - g));
+      g += w.kb1 - w.kb0;
+      return true;
+    }
+    if (tile >= n_tiles) return false;
+    coords(tile, w);
+    w.kb0 = 0;
+    w.kb1 = ((p.has_a2 && w.n0 + BN > p.split_begin) ? 2 : 1) * num_kb;
+    tile += gridDim.x;
+    return true;
+  }
+};
+
+__device__ __forceinline__ void red_add4(float* dst, float a, float b, float c, float d) {
+  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+
 // ---- epilogues: one thread owns one output row of the tile ---------------------------------
-template <int EPI>
+template <int EPI, int BN>
 __device__ __forceinline__ void epilogue_tile(const Params& p, uint32_t tmem_acc, int m, int n0, bool row_ok) {
   // tmem_acc already carries this warp's lane quarter in its upper half
   if (EPI == TC_STORE || EPI == TC_RESID || EPI == TC_PAGED) {
@@ -154,23 +214,20 @@ __device__ __forceinline__ void epilogue_tile(const Params& p, uint32_t tmem_acc
     if (EPI == TC_PAGED && row_ok) slot = p.paged.tok_slot[m];
 #pragma unroll 1
     for (int c = 0; c < BN; c += 32) {
+      int n = n0 + c;
+      int n_valid = p.N - n;
+      if (n_valid <= 0) break;           // uniform over the warp
       float v[32];
       tmem_ld32(tmem_acc + c, v);
       tmem_ld_wait();
-      int n = n0 + c;
-      int n_valid = p.N - n;
-      if (!row_ok || n_valid <= 0) continue;
+      if (!row_ok) continue;
       if (EPI == TC_STORE) {
         store32_bf16(p.C + (size_t)m * p.ldc + n, v, n_valid);
       } else if (EPI == TC_RESID) {
-        float4* x = reinterpret_cast<float4*>(p.X + (size_t)m * p.ldx + n);
+        float* x = p.X + (size_t)m * p.ldx + n;
 #pragma unroll
         for (int g = 0; g < 8; ++g)
-          if (g * 4 < n_valid) {
-            float4 t = x[g];
-            t.x += v[4 * g]; t.y += v[4 * g + 1]; t.z += v[4 * g + 2]; t.w += v[4 * g + 3];
-            x[g] = t;
-          }
+          if (g * 4 < n_valid) red_add4(x + 4 * g, v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
       } else {
         if (slot < 0) continue;
         const PagedOut& q = p.paged;
@@ -188,18 +245,20 @@ __device__ __forceinline__ void epilogue_tile(const Params& p, uint32_t tmem_acc
       }
     }
   } else if (EPI == TC_SWIGLU) {
-    // columns [0, 64) of the tile are gate rows, [64, 128) the matching up rows
+    // every 128 columns of the tile: [0, 64) gate rows, [64, 128) the matching up rows
 #pragma unroll 1
-    for (int c = 0; c < 64; c += 32) {
-      float g[32], u[32];
-      tmem_ld32(tmem_acc + c, g);
-      tmem_ld32(tmem_acc + 64 + c, u);
-      tmem_ld_wait();
-      int n = (n0 >> 1) + c;
+    for (int c = 0; c < BN / 2; c += 32) {
+      int grp = c >> 6, cc = c & 63;
+      int n = ((n0 + grp * 128) >> 1) + cc;
       int n_valid = p.ffn - n;
-      if (!row_ok || n_valid <= 0) continue;
+      if (n_valid <= 0) break;
+      float g[32], u[32];
+      tmem_ld32(tmem_acc + grp * 128 + cc, g);
+      tmem_ld32(tmem_acc + grp * 128 + 64 + cc, u);
+      tmem_ld_wait();
+      if (!row_ok) continue;
 #pragma unroll
-      for (int i = 0; i < 32; ++i) g[i] = g[i] / (1.f + __expf(-g[i])) * u[i];
+      for (int i = 0; i < 32; ++i) g[i] = __fdividef(g[i], 1.f + __expf(-g[i])) * u[i];
       store32_bf16(p.C + (size_t)m * p.ldc + n, g, n_valid);
     }
   } else {  // TC_QKV: RoPE on columns < rot_cols, hi part to C, lo part of columns >= lo_col_begin to C_lo
@@ -207,6 +266,7 @@ __device__ __forceinline__ void epilogue_tile(const Params& p, uint32_t tmem_acc
     const float2* tab = row_ok ? p.rope_tab + (size_t)p.tok_pos[m] * half : nullptr;
 #pragma unroll 1
     for (int h0 = 0; h0 < BN; h0 += p.hd) {
+      if (n0 + h0 >= p.N) break;
 #pragma unroll 1
       for (int j = 0; j < half; j += 32) {
         float a[32], b[32];
@@ -214,7 +274,7 @@ __device__ __forceinline__ void epilogue_tile(const Params& p, uint32_t tmem_acc
         tmem_ld32(tmem_acc + h0 + half + j, b);
         tmem_ld_wait();
         int n = n0 + h0 + j;
-        if (!row_ok || n >= p.N) continue;
+        if (!row_ok) continue;
         if (n < p.rot_cols) {
 #pragma unroll
           for (int i = 0; i < 32; i += 2) {
@@ -241,10 +301,12 @@ __device__ __forceinline__ void epilogue_tile(const Params& p, uint32_t tmem_acc
   }
 }
 
-template <int EPI>
+template <int EPI, int BN>
 __global__ void __launch_bounds__(N_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_a2,
                const __grid_constant__ CUtensorMap map_w, const Params p) {
+  using T = Tile<BN>;
+  constexpr int STAGES = T::STAGES, STAGE_BYTES = T::STAGE_BYTES;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
@@ -259,12 +321,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int tiles_m = (p.M + BM - 1) / BM, tiles_n = (p.N + BN - 1) / BN;
-  const int n_tiles = tiles_m * tiles_n;
-  const int num_kb = (p.K + BK - 1) / BK;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 2); mbar_init(empty_bar(s), 1); }   // two loaders per stage
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -277,23 +336,29 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  const int num_kb = (p.K + BK - 1) / BK;
 
-  if (warp == 0) {
-    // ---------------- TMA producer ----------------
+  if (warp == 0 || warp == 2) {
+    // ---------------- TMA producers: warp 0 loads the A tile of every stage, warp 2 the W tile ----------------
     if (lane == 0) {
+      const bool is_a = warp == 0;
+      Sched<BN> sched(p);
+      Work w;
       int stage = 0; uint32_t phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-        int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
-        int passes = (p.has_a2 && n0 + BN > p.split_begin) ? 2 : 1;
-        for (int it = 0; it < passes * num_kb && ok; ++it) {
+      while (ok && sched.next(w)) {
+        for (int it = w.kb0; it < w.kb1 && ok; ++it) {
           ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status);
           if (!ok) break;
-          int kb = it < num_kb ? it : it - num_kb;
-          uint32_t sa = smem_base + stage * STAGE_BYTES, sb = sa + BM * BK * 2;
-          mbar_expect_tx(full_bar(stage), STAGE_BYTES);
-          tma_load_2d(sa, it < num_kb ? &map_a : &map_a2, kb * BK, m0, full_bar(stage));
-          tma_load_2d(sb, &map_w, kb * BK, n0, full_bar(stage));
+          const int kb = it < num_kb ? it : it - num_kb;
+          const uint32_t sa = smem_base + stage * STAGE_BYTES;
+          if (is_a) {
+            mbar_expect_tx(full_bar(stage), T::A_BYTES);
+            tma_load_2d(sa, it < num_kb ? &map_a : &map_a2, kb * BK, w.m0, full_bar(stage));
+          } else {
+            mbar_expect_tx(full_bar(stage), T::W_BYTES);
+            tma_load_2d(sa + T::A_BYTES, &map_w, kb * BK, w.n0, full_bar(stage));
+          }
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
       }
@@ -305,25 +370,25 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      Sched<BN> sched(p);
+      Work w;
       int stage = 0; uint32_t phase = 0;
       int acc = 0; uint32_t acc_phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-        int n0 = (tile / tiles_m) * BN;
-        int passes = (p.has_a2 && n0 + BN > p.split_begin) ? 2 : 1;
+      while (ok && sched.next(w)) {
         ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.status);
         if (!ok) break;
         tc_fence_after();
-        uint32_t d_tmem = tmem_base + acc * BN;
-        for (int it = 0; it < passes * num_kb && ok; ++it) {
+        const uint32_t d_tmem = tmem_base + acc * BN;
+        for (int it = w.kb0; it < w.kb1 && ok; ++it) {
           ok = mbar_wait(full_bar(stage), phase, abort_flag, p.status);
           if (!ok) break;
           tc_fence_after();
-          uint32_t sa = smem_base + stage * STAGE_BYTES, sb = sa + BM * BK * 2;
-          uint64_t da = make_desc(sa), db = make_desc(sb);
+          const uint32_t sa = smem_base + stage * STAGE_BYTES, sb = sa + T::A_BYTES;
+          const uint64_t da = make_desc(sa), db = make_desc(sb);
 #pragma unroll
           for (int k = 0; k < BK / 16; ++k)
-            tc_mma_bf16(d_tmem, da + 2u * k, db + 2u * k, idesc, (it > 0 || k > 0) ? 1u : 0u);
+            tc_mma_bf16(d_tmem, da + 2u * k, db + 2u * k, idesc, (it > w.kb0 || k > 0) ? 1u : 0u);
           tc_commit(empty_bar(stage));        // the slot is free once these MMAs have read it
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -337,17 +402,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   } else {
     // ---------------- epilogue: 4 warps, each owns the 32 tensor-memory lanes of its quarter ----------------
     const int quarter = warp & 3;
+    Sched<BN> sched(p);
+    Work w;
     int acc = 0; uint32_t acc_phase = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-      int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
+    while (sched.next(w)) {
       ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      int m = m0 + quarter * 32 + lane;
-      uint32_t tmem_acc = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
-      epilogue_tile<EPI>(p, tmem_acc, m, n0, m < p.M);
+      const int m = w.m0 + quarter * 32 + lane;
+      const uint32_t tmem_acc = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
+      epilogue_tile<EPI, BN>(p, tmem_acc, m, w.n0, m < p.M);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar(acc));
@@ -374,11 +440,11 @@ bool get_encode() {
   return true;
 }
 
-// bf16 [rows, cols] row-major with row stride ld elements; box = 64 columns x 128 rows, 128B swizzle
-bool make_map(CUtensorMap* m, const void* base, int rows, int cols, int ld) {
+// bf16 [rows, cols] row-major with row stride ld elements; box = 64 columns x box_rows rows, 128B swizzle
+bool make_map(CUtensorMap* m, const void* base, int rows, int cols, int ld, int box_rows) {
   cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
-  cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)BM};
+  cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
   CUresult r = g_encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -386,16 +452,38 @@ bool make_map(CUtensorMap* m, const void* base, int rows, int cols, int ld) {
   return r == CUDA_SUCCESS;
 }
 
-template <int EPI>
+template <int EPI, int BN>
 cudaError_t go(const CUtensorMap& a, const CUtensorMap& a2, const CUtensorMap& w, const Params& p, int grid, cudaStream_t st) {
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<EPI, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Tile<BN>::SMEM_BYTES);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  gemm_tc_kernel<EPI><<<grid, N_THREADS, SMEM_BYTES, st>>>(a, a2, w, p);
+  gemm_tc_kernel<EPI, BN><<<grid, N_THREADS, Tile<BN>::SMEM_BYTES, st>>>(a, a2, w, p);
   return cudaGetLastError();
+}
+
+template <int BN>
+cudaError_t go_epi(int epi, const CUtensorMap& a, const CUtensorMap& a2, const CUtensorMap& w, const Params& p, int grid, cudaStream_t st) {
+  switch (epi) {
+    case TC_STORE: return go<TC_STORE, BN>(a, a2, w, p, grid, st);
+    case TC_RESID: return go<TC_RESID, BN>(a, a2, w, p, grid, st);
+    case TC_SWIGLU: return go<TC_SWIGLU, BN>(a, a2, w, p, grid, st);
+    case TC_QKV: return go<TC_QKV, BN>(a, a2, w, p, grid, st);
+    default: return go<TC_PAGED, BN>(a, a2, w, p, grid, st);
+  }
+}
+
+// Relative time of a launch with tile width bn on n_sm SMs: waves of tiles, each tile costing
+// the larger of its tensor-pipe time and its operand-feed time (two issuing threads deliver
+// about 100 bytes per cycle).
+double tile_cost(const TcGemm& g, int bn, bool stream_k) {
+  const double tiles = (double)((g.M + BM - 1) / BM) * ((g.N + bn - 1) / bn);
+  const double mma = 2.0 * bn, feed = (BM + bn) * 128.0 / 100.0;      // cycles per k block
+  const double per_tile = mma > feed ? mma : feed;
+  const double waves = stream_k ? tiles / g.n_sm : (double)(((long long)tiles + g.n_sm - 1) / g.n_sm);
+  return waves * per_tile;
 }
 
 }  // namespace
@@ -424,25 +512,25 @@ bool tc_gemm_supported(const TcGemm& g) {
 
 cudaError_t launch_gemm_tc(const TcGemm& g, int* status, cudaStream_t st, int64_t* n_launch) {
   if (!get_encode()) return cudaErrorNotSupported;
+  const int tiles128 = ((g.M + BM - 1) / BM) * ((g.N + 127) / 128);
+  const bool stream_k = g.epi == TC_RESID && !g.A2 && tiles128 < 2 * g.n_sm;
+  int bn = g.bn;
+  if (bn != 128 && bn != 256) bn = tile_cost(g, 256, stream_k) <= tile_cost(g, 128, stream_k) ? 256 : 128;
   CUtensorMap ma, ma2, mw;
-  if (!make_map(&ma, g.A, g.M, g.K, g.lda)) return cudaErrorInvalidValue;
-  if (!make_map(&mw, g.W, g.N, g.K, g.ldw)) return cudaErrorInvalidValue;
-  if (g.A2) { if (!make_map(&ma2, g.A2, g.M, g.K, g.lda2)) return cudaErrorInvalidValue; }
+  if (!make_map(&ma, g.A, g.M, g.K, g.lda, BM)) return cudaErrorInvalidValue;
+  if (!make_map(&mw, g.W, g.N, g.K, g.ldw, bn)) return cudaErrorInvalidValue;
+  if (g.A2) { if (!make_map(&ma2, g.A2, g.M, g.K, g.lda2, BM)) return cudaErrorInvalidValue; }
   else ma2 = ma;
   Params p{};
   p.M = g.M; p.N = g.N; p.K = g.K; p.split_begin = g.split_begin; p.has_a2 = g.A2 != nullptr; p.status = status;
+  p.stream_k = stream_k ? 1 : 0;
   p.C = g.C; p.ldc = g.ldc; p.X = g.X; p.ldx = g.ldx; p.C_lo = g.C_lo; p.ld_lo = g.ld_lo; p.lo_col_begin = g.lo_col_begin;
   p.rot_cols = g.rot_cols; p.hd = g.hd; p.rope_tab = g.rope_tab; p.tok_pos = g.tok_pos; p.ffn = g.ffn; p.paged = g.paged;
-  int tiles = ((g.M + BM - 1) / BM) * ((g.N + BN - 1) / BN);
-  int grid = tiles < g.n_sm ? tiles : g.n_sm;
+  const int tiles = ((g.M + BM - 1) / BM) * ((g.N + bn - 1) / bn);
+  const long long kblocks = (long long)tiles * ((g.K + BK - 1) / BK);
+  int grid = stream_k ? (int)(kblocks < g.n_sm ? kblocks : g.n_sm) : (tiles < g.n_sm ? tiles : g.n_sm);
   ++*n_launch;
-  switch (g.epi) {
-    case TC_STORE: return go<TC_STORE>(ma, ma2, mw, p, grid, st);
-    case TC_RESID: return go<TC_RESID>(ma, ma2, mw, p, grid, st);
-    case TC_SWIGLU: return go<TC_SWIGLU>(ma, ma2, mw, p, grid, st);
-    case TC_QKV: return go<TC_QKV>(ma, ma2, mw, p, grid, st);
-    default: return go<TC_PAGED>(ma, ma2, mw, p, grid, st);
-  }
+  return bn == 256 ? go_epi<256>(g.epi, ma, ma2, mw, p, grid, st) : go_epi<128>(g.epi, ma, ma2, mw, p, grid, st);
 }
 
 // ---- RoPE table: tab[pos][c] = (cos, sin)(pos * theta^(-2c/hd)) -----------------------------

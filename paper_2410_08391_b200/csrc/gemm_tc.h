@@ -26,6 +26,7 @@ struct TcGemm {
   int ffn;
   PagedOut paged;
   int n_sm;
+  int bn;                          // tile width: 128, 256, or 0 = chosen by the launcher
 };
 
 bool tc_gemm_supported(const TcGemm& g);
