@@ -13,6 +13,7 @@
 #include "gemm_tc.h"
 #include "kvp_internal.h"
 #include "step_mega.h"
+#include "step_tc.h"
 
 namespace {
 
@@ -131,6 +132,11 @@ WsLayout ws_layout(const kvp_handle* h, int64_t Bm, int64_t Tm) {
   w.part = take((size_t)(2 * 148 + Bm * B.max_nkv) * B.max_group * (B.L[0].hd + 2) * 4);
   w.tok_stage = take(Tm * 4);
   w.first_stage = take(Bm * 4);
+  // tensor-core step projections: operand rows (hi + lo) of the widest input, fp32 gate/up outputs
+  const int64_t Bp = step_tc_rows((int)Bm);
+  const int64_t k_max = std::max((int64_t)B.d, std::max((int64_t)B.max_dq, (int64_t)B.max_ffn));
+  w.xbt = take(2 * Bp * k_max * 2);
+  w.gub = take(Bm * 2 * (size_t)B.max_ffn * 4);
   w.total = off;
   return w;
 }
@@ -193,9 +199,31 @@ bool try_tc(kvp_handle* h, const LaunchCtx& ctx, TcGemm& t, int cls, cudaError_t
   return true;
 }
 
+// Are the step's projections run on the tensor cores (batches the CUDA-core kernels are too slow for)?
+bool step_uses_tc(const kvp_handle* h, int batch) {
+  if (!h->use_tc || h->opt.dtype != KVP_BF16 || batch <= 4 || step_tc_rows(batch) > 128) return false;
+  const ModelPlan& B = h->base;
+  if (B.d % 8) return false;
+  for (int i = 0; i < B.n_layers; ++i)
+    if (B.L[i].dq % 8 || B.L[i].ffn % 8) return false;
+  return true;
+}
+
+// y += W x on the tensor cores: operand rows from `src` (RMS-normalised with `gain`, or SwiGLU of a
+// gate/up row, or as they are), output cleared first unless it is the residual stream.
+void step_proj_tc(kvp_handle* h, const LaunchCtx& ctx, const WsLayout& w, char* ws, int mode, const float* src, int ld_src,
+                  int K, int batch, const float* gain, int G, const void* W, int N, float* Y, int ldy, bool clear,
+                  cudaError_t* err) {
+  bf16* XB = (bf16*)(ws + w.xbt);
+  KVP_TIMED(KVP_CLASS_STEP_GEMV, launch_step_prep(ctx, mode, src, ld_src, K, batch, gain, h->base.eps, G, XB, clear ? Y : nullptr, ldy, N));
+  TimedScope ts(h, ctx.st, KVP_CLASS_STEP_GEMV);
+  cudaError_t e = launch_step_gemm_tc((const bf16*)W, K, N, K, XB, batch, Y, ldy, h->n_sm, ctx.status, ctx.st, ctx.n_launch);
+  if (e != cudaSuccess && *err == cudaSuccess) *err = e;
+}
+
 // one base-model layer of a single-token step (shared by the first step and generation)
 void base_layer_step(kvp_handle* h, const LaunchCtx& ctx, int i, const kvp_cache* cache, const WsLayout& w, char* ws,
-                     int batch, int max_keys, bool generation) {
+                     int batch, int max_keys, bool generation, cudaError_t* err) {
   const ModelPlan& B = h->base;
   const LayerPlan& L = B.L[i];
   const char* P = h->packed;
@@ -206,14 +234,25 @@ void base_layer_step(kvp_handle* h, const LaunchCtx& ctx, int i, const kvp_cache
   float* actb = (float*)(ws + w.actb);
   // the first step needs q only (keys and values are the predicted ones); generation needs q, k, v
   int n_out = generation ? L.nqkv : L.dq;
-  KVP_TIMED(KVP_CLASS_STEP_GEMV, launch_step_gemv(ctx, P + L.wqkv, B.d, n_out, B.d, xb, B.d, batch, qkvb, n_out, GEMV_STORE, 0, 0,
-                                                  (const float*)(P + L.attn_norm), B.eps, hb));
+  const bool tc = step_uses_tc(h, batch);
+  if (tc)
+    step_proj_tc(h, ctx, w, ws, PREP_NORM, xb, B.d, B.d, batch, (const float*)(P + L.attn_norm), 0, P + L.wqkv, n_out, qkvb, n_out, true, err);
+  else
+    KVP_TIMED(KVP_CLASS_STEP_GEMV, launch_step_gemv(ctx, P + L.wqkv, B.d, n_out, B.d, xb, B.d, batch, qkvb, n_out, GEMV_STORE, 0, 0,
+                                                    (const float*)(P + L.attn_norm), B.eps, hb));
   if (generation)
     KVP_TIMED(KVP_CLASS_OTHER, launch_step_append(ctx, qkvb, L.nq, L.nkv, L.hd, B.theta, cache->k_pools[i], cache->v_pools[i], cache->block_table,
                        cache->max_pages_per_seq, cache->n_pages, cache->seq_lens, batch));
   KVP_TIMED(KVP_CLASS_STEP_ATTN, launch_step_attn(ctx, qkvb, n_out, L.nq, L.nkv, L.hd, B.theta, cache->k_pools[i], cache->v_pools[i], cache->block_table,
                    cache->max_pages_per_seq, cache->n_pages, cache->seq_lens, generation ? 1 : 0, batch, max_keys,
                    (float*)(ws + w.part), ab));
+  if (tc) {
+    float* gub = (float*)(ws + w.gub);
+    step_proj_tc(h, ctx, w, ws, PREP_PLAIN, ab, L.dq, L.dq, batch, nullptr, 0, P + L.wo, B.d, xb, B.d, false, err);
+    step_proj_tc(h, ctx, w, ws, PREP_NORM, xb, B.d, B.d, batch, (const float*)(P + L.ffn_norm), 0, P + L.wgu, 2 * L.ffn, gub, 2 * L.ffn, true, err);
+    step_proj_tc(h, ctx, w, ws, PREP_SWIGLU, gub, 2 * L.ffn, L.ffn, batch, nullptr, L.G, P + L.wd, B.d, xb, B.d, false, err);
+    return;
+  }
   KVP_TIMED(KVP_CLASS_STEP_GEMV, launch_step_gemv(ctx, P + L.wo, L.dq, B.d, L.dq, ab, L.dq, batch, xb, B.d, GEMV_RESID, 0, 0));
   KVP_TIMED(KVP_CLASS_STEP_GEMV, launch_step_gemv(ctx, P + L.wgu, B.d, L.ffn, B.d, xb, B.d, batch, actb, L.ffn, GEMV_SWIGLU, L.G, L.ffn,
                                                   (const float*)(P + L.ffn_norm), B.eps, hb));
@@ -260,11 +299,14 @@ bool base_step_fused(kvp_handle* h, const LaunchCtx& ctx, const kvp_cache* cache
 }
 
 void base_head(kvp_handle* h, const LaunchCtx& ctx, const WsLayout& w, char* ws, int batch, float* logits,
-               int32_t* token_out) {
+               int32_t* token_out, cudaError_t* err) {
   const ModelPlan& B = h->base;
   const char* P = h->packed;
   float* xb = (float*)(ws + w.xb);
   float* hb = (float*)(ws + w.hb);
+  if (step_uses_tc(h, batch))
+    step_proj_tc(h, ctx, w, ws, PREP_NORM, xb, B.d, B.d, batch, (const float*)(P + B.final_norm), 0, P + B.lm_head, B.vocab, logits, B.vocab, true, err);
+  else
   KVP_TIMED(KVP_CLASS_STEP_GEMV, launch_step_gemv(ctx, P + B.lm_head, B.d, B.vocab, B.d, xb, B.d, batch, logits, B.vocab, GEMV_STORE, 0, 0,
                                                   (const float*)(P + B.final_norm), B.eps, hb));
   if (token_out) KVP_TIMED(KVP_CLASS_OTHER, launch_argmax(ctx, logits, batch, B.vocab, token_out));
@@ -584,8 +626,8 @@ static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int
   // ---- stage 3: one base step per sequence on its last prompt token ----
   if (!base_step_fused(h, ctx, cache, w, ws, batch, cs.max_len, false, tokens, last_idx, logits_out, first_token, &tc_err)) {
     KVP_TIMED(KVP_CLASS_OTHER, launch_embed(ctx, tokens, last_idx, batch, P + h->base.embed, h->base.vocab, h->base.d, (float*)(ws + w.xb)));
-    for (int i = 0; i < h->base.n_layers; ++i) base_layer_step(h, ctx, i, cache, w, ws, batch, cs.max_len, false);
-    base_head(h, ctx, w, ws, batch, logits_out, first_token);
+    for (int i = 0; i < h->base.n_layers; ++i) base_layer_step(h, ctx, i, cache, w, ws, batch, cs.max_len, false, &tc_err);
+    base_head(h, ctx, w, ws, batch, logits_out, first_token, &tc_err);
   }
   if (tc_err != cudaSuccess) return fail(h, KVP_ERR_CUDA, "base step launch: %s", cudaGetErrorString(tc_err));
   return check_cuda(h, "kvp_prefill_predict");
@@ -708,9 +750,10 @@ kvp_status kvp_decode_step(kvp_handle* h, const int32_t* tokens, const int32_t* 
     return check_cuda(h, "kvp_decode_step");
   }
   KVP_TIMED(KVP_CLASS_OTHER, launch_embed(ctx, tokens, nullptr, batch, h->packed + h->base.embed, h->base.vocab, h->base.d, (float*)(ws + w.xb)));
-  for (int i = 0; i < h->base.n_layers; ++i) base_layer_step(h, ctx, i, cache, w, ws, batch, cs.max_len + 1, true);
-  base_head(h, ctx, w, ws, batch, logits_out, next_token);
+  for (int i = 0; i < h->base.n_layers; ++i) base_layer_step(h, ctx, i, cache, w, ws, batch, cs.max_len + 1, true, &mega_err);
+  base_head(h, ctx, w, ws, batch, logits_out, next_token, &mega_err);
   KVP_TIMED(KVP_CLASS_OTHER, launch_add_int(ctx, cache->seq_lens, batch, 1));
+  if (mega_err != cudaSuccess) return fail(h, KVP_ERR_CUDA, "base step launch: %s", cudaGetErrorString(mega_err));
   return check_cuda(h, "kvp_decode_step");
 }
 

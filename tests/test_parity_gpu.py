@@ -29,6 +29,9 @@ CASES = [
     ("t_scaled", [100, 33, 257], "fanin"),
     ("t_scaled", [100, 33, 257], "n002"),
     ("t_bias", [40, 90], "fanin"),
+    # more than 4 sequences: the step's projections run on the tensor cores (operand rows padded to 16, 24)
+    ("t_hd128", [40, 9, 130, 17, 64, 65, 3, 90, 128], "fanin"),
+    ("t_scaled", [20, 33, 5, 64, 65, 1, 40, 41, 42, 43, 44, 45, 46, 47, 48, 49, 50], "fanin"),
 ]
 
 
@@ -45,12 +48,13 @@ def test_prefill_predict_matches_oracle(name, lens, regime):
         s.close()
 
 
-@pytest.mark.parametrize("name,regime", [("t_small", "fanin"), ("t_small_f32", "fanin"), ("c1", "n002")])
-def test_decode_steps_match_oracle(name, regime):
+@pytest.mark.parametrize("name,regime,lens", [("t_small", "fanin", [70, 63, 5]), ("t_small_f32", "fanin", [70, 63, 5]),
+                                              ("c1", "n002", [64]), ("t_small", "n002", [70, 63, 5, 64, 1, 30])],
+                         ids=lambda v: str(v).replace(" ", ""))
+def test_decode_steps_match_oracle(name, regime, lens):
     import torch
     pair = wl.pair(name)
     W = wl.make_weights(pair, seed=2, regime=regime)
-    lens = [70, 63, 5] if name != "c1" else [64]
     pr = wl.custom_prompts(pair.base.vocab, lens, seed=2)
     steps = 3
     s = make_session(pair, W, pr, extra_len=steps)
