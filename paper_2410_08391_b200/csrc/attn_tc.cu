@@ -1,81 +1,38 @@
 // Causal grouped-query attention over a ragged batch on the sm_100a tensor cores.
 //
-// One CTA = 128 consecutive queries of one sequence and one query head.  Warp 0 streams K and
-// V tiles (128 keys) of the matching kv head with TMA straight out of the packed [T, q|k|v]
-// projection buffer; warp 1 issues S = Q K^T and PV = P V with tcgen05.mma into tensor memory
-// (two S buffers, one PV buffer); warps 2-5 own one query row per thread: they read S from
-// tensor memory, keep the running max / sum in fp32, write P as bf16 into shared memory in the
-// swizzled operand layout, and accumulate O in registers from the per-tile PV products, so
-// no rescaling ever touches tensor memory.  S of tile j+1 is computed while the softmax of
-// tile j runs.  Key tiles above the diagonal are skipped; the diagonal tile is masked.
-#include <cuda.h>
-#include <cudaTypedefs.h>
+// One CTA = 256 consecutive queries of one sequence (two tiles of 128) and one query head.
+// Warp 0 streams K and V tiles of the matching kv head with TMA straight out of the packed
+// [T, q|k|v] projection buffer; both query tiles use them.  Warp 1 issues S = Q K^T and
+// O += P V with tcgen05.mma; S and O of both query tiles live in tensor memory.  Two groups of
+// four warps, one per query tile, own one query row per thread: a thread reads its row of S
+// into registers in one go (which frees S for the next key tile at once), keeps the running
+// max / sum in fp32 and writes P as bf16 into shared memory in the swizzled operand layout.
+// O is accumulated by the tensor core itself and only touched when a row's maximum has grown
+// by more than 2^8 since the exponent offset was last fixed; then the group rescales its O in
+// tensor memory (tcgen05.ld / st).  While one group computes exponentials the tensor core works
+// for the other.  Key tiles above the diagonal are skipped; tiles touching it are masked.
+// Work is ordered so that, over the whole batch, CTAs with the most key tiles start first.
 #include <math.h>
 
 #include "attn_tc.h"
-#include "common.cuh"
+#include "tc_ptx.cuh"
 
 namespace {
+using namespace tcp;
 
-constexpr int BQ = 128, BKV = 128;
-constexpr int N_THREADS = 192;
-constexpr uint32_t SPIN_LIMIT = 20u * 1000u * 1000u;
-constexpr int P_BYTES = BQ * BKV * 2;
+constexpr int BQ = 128;                 // queries per tile; a CTA has two tiles
+constexpr int N_THREADS = 320;          // warps: 0 TMA, 1 MMA, 2-5 tile 0, 6-9 tile 1
+constexpr int STAGES = 3;
+constexpr float RESCALE_LOG2 = 8.f;     // tolerated growth of a row maximum before O is rescaled
 
 template <int HD> struct Cfg {
-  static constexpr int TILE_BYTES = 128 * HD * 2;       // a Q, K or V tile
-  static constexpr int STAGES = HD == 64 ? 3 : 2;
-  static constexpr int SMEM = TILE_BYTES + P_BYTES + STAGES * 2 * TILE_BYTES + 1024 + 256;
+  static constexpr int BKV = HD == 64 ? 128 : 64;       // keys per tile
+  static constexpr int Q_BYTES = BQ * HD * 2;
+  static constexpr int KV_BYTES = BKV * HD * 2;         // a K or a V tile
+  static constexpr int P_BYTES = BQ * BKV * 2;
+  static constexpr int SMEM = 2 * Q_BYTES + 2 * P_BYTES + STAGES * 2 * KV_BYTES + 1024 + 256;
 };
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
-  for (uint32_t it = 0; it < SPIN_LIMIT; ++it) {
-    if (mbar_test(bar, parity)) return true;
-    if ((it & 63u) == 63u) {
-      if (*abort_flag) return false;
-      __nanosleep(64);
-    }
-  }
-  *abort_flag = 1;
-  dev_flag(status, DEV_TIMEOUT);
-  return false;
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
   uint32_t* r = reinterpret_cast<uint32_t*>(v);
   asm volatile(
@@ -88,18 +45,23 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
         "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr) : "memory");
 }
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float* v) {
+  const uint32_t* r = reinterpret_cast<const uint32_t*>(v);
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
+        "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
+        "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
-}
-
-// K-major operand tile (rows of 128 bytes, 128B swizzle, 8-row groups 1024 B apart)
-__device__ __forceinline__ uint64_t desc_kmajor(uint32_t addr) {
-  uint64_t lo = ((addr & 0x3FFFFu) >> 4) | (1u << 16);
-  uint64_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);
-  return lo | (hi << 32);
 }
 // MN-major operand tile: 64 contiguous MN elements per 128-byte row, rows = K index, 8-row groups
 // 1024 B apart (stride offset), next 64 MN elements `lbo` bytes away (leading offset)
@@ -110,58 +72,54 @@ __device__ __forceinline__ uint64_t desc_mnmajor(uint32_t addr, uint32_t lbo) {
 }
 
 struct Params {
-  const int* cu; int batch; int nq, nkv;
+  const int* cu; const int2* sched;     // sched[i] = (sequence, first query of the pair of tiles)
+  int nq, nkv;
   bf16* out; int ldo;
   float scale_log2e;
   int* status;
 };
 
 template <int HD>
-__global__ void __launch_bounds__(N_THREADS, 1) attn_tc_kernel(const __grid_constant__ CUtensorMap map_qkv, const Params p) {
+__global__ void __launch_bounds__(N_THREADS, 1)
+attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kv, const Params p) {
   using C = Cfg<HD>;
-  constexpr int ST = C::STAGES, TB = C::TILE_BYTES, NBOX = HD / 64;
+  constexpr int BKV = C::BKV, QB = C::Q_BYTES, KB = C::KV_BYTES, PB = C::P_BYTES, NBOX = HD / 64;
+  constexpr int KV_BOX = BKV * 128;     // bytes of one 64-column box of a K or V tile
   extern __shared__ uint8_t smem_raw[];
-  __shared__ int s_b, s_q0;
-  // which (sequence, query tile): tiles are numbered sequence by sequence, last tile of a sequence first
-  if (threadIdx.x == 0) {
-    int blk = blockIdx.y, b = 0;
-    for (; b < p.batch; ++b) {
-      int nb = (p.cu[b + 1] - p.cu[b] + BQ - 1) / BQ;
-      if (blk < nb) { blk = nb - 1 - blk; break; }
-      blk -= nb;
-    }
-    s_b = b; s_q0 = blk * BQ;
-  }
-  __syncthreads();
-  const int b = s_b, q0 = s_q0;
-  if (b >= p.batch) return;
+  const int2 item = p.sched[blockIdx.y];
+  const int b = item.x, q0 = item.y;
   const int base = p.cu[b], L = p.cu[b + 1] - base;
   const int head = blockIdx.x, kvh = head / (p.nq / p.nkv);
-  const int n_kv = (min(L, q0 + BQ) + BKV - 1) / BKV;
+  // key tiles each query tile needs (tile 1 may lie beyond the end of the sequence)
+  int n_kv[2];
+  n_kv[0] = (min(L, q0 + BQ) + BKV - 1) / BKV;
+  n_kv[1] = q0 + BQ < L ? (min(L, q0 + 2 * BQ) + BKV - 1) / BKV : 0;
+  const int n_max = max(n_kv[0], n_kv[1]);
 
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  const uint32_t sQ = smem_u32(smem), sP = sQ + TB, sKV = sP + P_BYTES;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + TB + P_BYTES + ST * 2 * TB);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * ST + 5);
+  const uint32_t sQ = smem_u32(smem), sP = sQ + 2 * QB, sKV = sP + 2 * PB;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 2 * QB + 2 * PB + STAGES * 2 * KB);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 9);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const uint32_t bar_base = smem_u32(bars);
   auto kv_full = [&](int s) { return bar_base + 8u * s; };
-  auto kv_empty = [&](int s) { return bar_base + 8u * (ST + s); };
-  auto s_full = [&](int i) { return bar_base + 8u * (2 * ST + i); };
-  const uint32_t q_full = bar_base + 8u * (2 * ST + 2), p_ready = bar_base + 8u * (2 * ST + 3), pv_full = bar_base + 8u * (2 * ST + 4);
+  auto kv_empty = [&](int s) { return bar_base + 8u * (STAGES + s); };
+  auto s_full = [&](int g) { return bar_base + 8u * (2 * STAGES + g); };
+  auto s_free = [&](int g) { return bar_base + 8u * (2 * STAGES + 2 + g); };
+  auto p_ready = [&](int g) { return bar_base + 8u * (2 * STAGES + 4 + g); };
+  auto pv_done = [&](int g) { return bar_base + 8u * (2 * STAGES + 6 + g); };
+  const uint32_t q_full = bar_base + 8u * (2 * STAGES + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
-    for (int s = 0; s < ST; ++s) { mbar_init(kv_full(s), 1); mbar_init(kv_empty(s), 1); }
-    mbar_init(s_full(0), 1); mbar_init(s_full(1), 1);
-    mbar_init(q_full, 1); mbar_init(p_ready, 4); mbar_init(pv_full, 1);
+    for (int s = 0; s < STAGES; ++s) { mbar_init(kv_full(s), 1); mbar_init(kv_empty(s), 1); }
+    for (int g = 0; g < 2; ++g) { mbar_init(s_full(g), 1); mbar_init(s_free(g), 4); mbar_init(p_ready(g), 4); mbar_init(pv_done(g), 1); }
+    mbar_init(q_full, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 1) {   // tensor memory: S0 at column 0, S1 at 128, PV at 256
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
+  // tensor memory: S of tile g at column 128 g, O of tile g at column 256 + 128 g
+  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), 512);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -170,171 +128,183 @@ __global__ void __launch_bounds__(N_THREADS, 1) attn_tc_kernel(const __grid_cons
   if (warp == 0) {
     if (lane == 0) {
       bool ok = true;
-      mbar_expect_tx(q_full, TB);
+      mbar_expect_tx(q_full, 2 * QB);
 #pragma unroll
-      for (int x = 0; x < NBOX; ++x) tma_load_2d(sQ + x * 16384, &map_qkv, head * HD + x * 64, base + q0, q_full);
+      for (int g = 0; g < 2; ++g)
+#pragma unroll
+        for (int x = 0; x < NBOX; ++x) tma_load_2d(sQ + g * QB + x * 16384, &map_q, head * HD + x * 64, base + q0 + g * BQ, q_full);
       const int kcol = (p.nq + kvh) * HD, vcol = (p.nq + p.nkv + kvh) * HD;
       int stage = 0; uint32_t phase = 0;
-      for (int j = 0; j < n_kv && ok; ++j) {
+      for (int j = 0; j < n_max && ok; ++j) {
         ok = mbar_wait(kv_empty(stage), phase ^ 1u, abort_flag, p.status);
         if (!ok) break;
-        uint32_t sk = sKV + stage * 2 * TB, sv = sk + TB;
-        mbar_expect_tx(kv_full(stage), 2 * TB);
+        const uint32_t sk = sKV + stage * 2 * KB, sv = sk + KB;
+        mbar_expect_tx(kv_full(stage), 2 * KB);
 #pragma unroll
         for (int x = 0; x < NBOX; ++x) {
-          tma_load_2d(sk + x * 16384, &map_qkv, kcol + x * 64, base + j * BKV, kv_full(stage));
-          tma_load_2d(sv + x * 16384, &map_qkv, vcol + x * 64, base + j * BKV, kv_full(stage));
+          tma_load_2d(sk + x * KV_BOX, &map_kv, kcol + x * 64, base + j * BKV, kv_full(stage));
+          tma_load_2d(sv + x * KV_BOX, &map_kv, vcol + x * 64, base + j * BKV, kv_full(stage));
         }
-        if (++stage == ST) { stage = 0; phase ^= 1u; }
+        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
       }
-      if (!ok) for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+      if (!ok) drain_after_abort();
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      // S = Q K^T: M = 128 queries, N = 128 keys, both operands K-major over head_dim
-      const uint32_t idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BKV >> 3) << 17) | ((uint32_t)(BQ >> 4) << 24);
-      // PV = P V: A = P (K-major over keys), B = V as stored [key][dim] = MN-major, N = head_dim
-      const uint32_t idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(HD >> 3) << 17) | ((uint32_t)(BQ >> 4) << 24);
-      bool ok = mbar_wait(q_full, 0, abort_flag, p.status);
-      int stage_qk = 0; uint32_t phase_qk = 0;      // stage of the next QK to issue
-      int stage_pv = 0;                             // stage of the next PV to issue
-      auto issue_qk = [&](int j) -> bool {
-        if (!mbar_wait(kv_full(stage_qk), phase_qk, abort_flag, p.status)) return false;
-        tc_fence_after();
-        uint32_t sk = sKV + stage_qk * 2 * TB;
+      // S = Q K^T: M = 128 queries, N = BKV keys, both operands K-major over head_dim
+      const uint32_t idesc_s = idesc_bf16(BQ, BKV);
+      // O += P V: A = P (K-major over keys), B = V as stored [key][dim] = MN-major, N = head_dim
+      const uint32_t idesc_pv = idesc_bf16(BQ, HD) | (1u << 16);
+      auto issue_s = [&](int g, int stage) {
+        const uint32_t sk = sKV + stage * 2 * KB;
 #pragma unroll
-        for (int kk = 0; kk < HD / 16; ++kk) {
-          uint32_t off = (kk >> 2) * 16384 + (kk & 3) * 32;
-          tc_mma_bf16(tmem_base + (j & 1) * 128, desc_kmajor(sQ + off), desc_kmajor(sk + off), idesc_s, kk > 0 ? 1u : 0u);
-        }
-        tc_commit(s_full(j & 1));
-        if (++stage_qk == ST) { stage_qk = 0; phase_qk ^= 1u; }
-        return true;
+        for (int kk = 0; kk < HD / 16; ++kk)
+          tc_mma_bf16(tmem_base + g * 128, desc_kmajor(sQ + g * QB + (kk >> 2) * 16384 + (kk & 3) * 32),
+                      desc_kmajor(sk + (kk >> 2) * KV_BOX + (kk & 3) * 32), idesc_s, kk > 0 ? 1u : 0u);
+        tc_commit(s_full(g));
       };
-      if (ok) ok = issue_qk(0);
-      for (int j = 0; j < n_kv && ok; ++j) {
-        if (j + 1 < n_kv) { ok = issue_qk(j + 1); if (!ok) break; }
-        ok = mbar_wait(p_ready, j & 1, abort_flag, p.status);
-        if (!ok) break;
+      bool ok = mbar_wait(q_full, 0, abort_flag, p.status);
+      if (ok) ok = mbar_wait(kv_full(0), 0, abort_flag, p.status);
+      if (ok) {
         tc_fence_after();
-        uint32_t sv = sKV + stage_pv * 2 * TB + TB;
-#pragma unroll
-        for (int kk = 0; kk < BKV / 16; ++kk) {
-          uint64_t da = desc_kmajor(sP + (kk >> 2) * 16384 + (kk & 3) * 32);
-          uint64_t db = desc_mnmajor(sv + kk * 2048, 16384);
-          tc_mma_bf16(tmem_base + 256, da, db, idesc_pv, kk > 0 ? 1u : 0u);
-        }
-        tc_commit(pv_full);
-        tc_commit(kv_empty(stage_pv));
-        if (++stage_pv == ST) stage_pv = 0;
+        for (int g = 0; g < 2; ++g) if (n_kv[g] > 0) issue_s(g, 0);
       }
-      if (!ok) for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+      for (int j = 0; j < n_max && ok; ++j) {
+        const int stage = j % STAGES;
+        if (j + 1 < n_max) {
+          const int s1 = (j + 1) % STAGES;
+          ok = mbar_wait(kv_full(s1), ((j + 1) / STAGES) & 1, abort_flag, p.status);
+          if (!ok) break;
+          tc_fence_after();
+          for (int g = 0; g < 2 && ok; ++g)
+            if (j + 1 < n_kv[g]) {
+              ok = mbar_wait(s_free(g), j & 1, abort_flag, p.status);      // S(j) of this tile is in registers
+              if (!ok) break;
+              tc_fence_after();
+              issue_s(g, s1);
+            }
+          if (!ok) break;
+        }
+        const uint32_t sv = sKV + stage * 2 * KB + KB;
+        for (int g = 0; g < 2 && ok; ++g)
+          if (j < n_kv[g]) {
+            ok = mbar_wait(p_ready(g), j & 1, abort_flag, p.status);
+            if (!ok) break;
+            tc_fence_after();
+#pragma unroll
+            for (int kk = 0; kk < BKV / 16; ++kk)
+              tc_mma_bf16(tmem_base + 256 + g * 128, desc_kmajor(sP + g * PB + (kk >> 2) * 16384 + (kk & 3) * 32),
+                          desc_mnmajor(sv + kk * 2048, KV_BOX), idesc_pv, (j > 0 || kk > 0) ? 1u : 0u);
+            tc_commit(pv_done(g));
+          }
+        if (!ok) break;
+        tc_commit(kv_empty(stage));
+      }
+      if (!ok) drain_after_abort();
     }
   } else {
-    const int quarter = warp & 3;
+    const int g = (warp - 2) >> 2;              // query tile of this warp's group
+    const int quarter = warp & 3;               // tensor-memory lane quarter this warp may access
     const int r = quarter * 32 + lane;          // row of the query tile owned by this thread
-    const int q_pos = q0 + r;
+    const int qs = q0 + g * BQ, q_pos = qs + r;
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
+    const uint32_t tS = tmem_base + lane_off + g * 128, tO = tmem_base + lane_off + 256 + g * 128;
+    const uint32_t sPg = sP + g * PB;
     const float c = p.scale_log2e;
-    float m = -INFINITY, l = 0.f;
-    float o[HD];
-#pragma unroll
-    for (int i = 0; i < HD; ++i) o[i] = 0.f;
+    const int n = n_kv[g];
+    float m_ref = -INFINITY, l = 0.f;
     bool ok = true;
-    for (int j = 0; j < n_kv; ++j) {
-      ok = mbar_wait(s_full(j & 1), (j >> 1) & 1, abort_flag, p.status);
+    for (int j = 0; j < n; ++j) {
+      ok = mbar_wait(s_full(g), j & 1, abort_flag, p.status);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      const uint32_t tS = tmem_base + lane_off + (j & 1) * 128;
-      const int kbase = j * BKV;
-      const bool diag = kbase + BKV - 1 > q0;    // some key of this tile may lie above some query of the tile
-      // pass 1: row maximum over the visible keys
-      float mt = -INFINITY;
-#pragma unroll 1
-      for (int cc = 0; cc < BKV; cc += 32) {
-        float v[32];
-        tmem_ld32(tS + cc, v);
-        tmem_ld_wait();
+      float s[BKV];
 #pragma unroll
-        for (int i = 0; i < 32; ++i)
-          if (!diag || kbase + cc + i <= q_pos) mt = fmaxf(mt, v[i]);
+      for (int cc = 0; cc < BKV; cc += 32) tmem_ld32(tS + cc, s + cc);
+      tmem_ld_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(s_free(g));
+      const int kbase = j * BKV;
+      const bool diag = kbase + BKV - 1 > qs;     // some key of this tile lies above some query of the tile
+      float mt = -INFINITY;
+      if (diag) {
+#pragma unroll
+        for (int i = 0; i < BKV; ++i) { if (kbase + i > q_pos) s[i] = -INFINITY; mt = fmaxf(mt, s[i]); }
+      } else {
+#pragma unroll
+        for (int i = 0; i < BKV; ++i) mt = fmaxf(mt, s[i]);
       }
-      const float m_new = fmaxf(m, mt);
-      const float alpha = (m_new == -INFINITY) ? 1.f : fast_exp2((m - m_new) * c);
-      // fold in the previous tile's PV product (this also tells us that P may be overwritten)
-      if (j > 0) {
-        ok = mbar_wait(pv_full, (j - 1) & 1, abort_flag, p.status);
+      if (j > 0) {     // the previous P V product has read P and finished writing O
+        ok = mbar_wait(pv_done(g), (j - 1) & 1, abort_flag, p.status);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
-#pragma unroll
-        for (int cc = 0; cc < HD; cc += 32) {
-          float v[32];
-          tmem_ld32(tmem_base + lane_off + 256 + cc, v);
-          tmem_ld_wait();
-#pragma unroll
-          for (int i = 0; i < 32; ++i) o[cc + i] = (o[cc + i] + v[i]) * alpha;
-        }
       }
-      l *= alpha;
-      // pass 2: probabilities, written as the bf16 A operand of the PV product
-      const float mc = (m_new == -INFINITY) ? 0.f : m_new * c;
-      float rowsum = 0.f;
+      const bool need = mt > m_ref && (m_ref == -INFINITY || (mt - m_ref) * c > RESCALE_LOG2);
+      if (__any_sync(0xffffffffu, need)) {
+        const float alpha = (need && m_ref != -INFINITY) ? fast_exp2((m_ref - mt) * c) : 1.f;
+        if (j > 0) {
 #pragma unroll 1
-      for (int cc = 0; cc < BKV; cc += 32) {
-        float v[32];
-        tmem_ld32(tS + cc, v);
-        tmem_ld_wait();
+          for (int cc = 0; cc < HD; cc += 32) {
+            float v[32];
+            tmem_ld32(tO + cc, v);
+            tmem_ld_wait();
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          float e = (!diag || kbase + cc + i <= q_pos) ? fast_exp2(v[i] * c - mc) : 0.f;
-          rowsum += e;
-          v[i] = e;
+            for (int i = 0; i < 32; ++i) v[i] *= alpha;
+            tmem_st32(tO + cc, v);
+          }
+          tmem_st_wait();
         }
+        l *= alpha;
+        if (need) m_ref = mt;
+      }
+      const float mc = (m_ref == -INFINITY) ? 0.f : m_ref * c;
+      float rowsum = 0.f;
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {
-          int k0 = cc + g * 8;
-          uint32_t addr = sP + (k0 >> 6) * 16384 + r * 128 + ((((k0 & 63) >> 3) ^ (r & 7)) << 4);
-          __nv_bfloat162 a0 = __floats2bfloat162_rn(v[g * 8], v[g * 8 + 1]), a1 = __floats2bfloat162_rn(v[g * 8 + 2], v[g * 8 + 3]);
-          __nv_bfloat162 a2 = __floats2bfloat162_rn(v[g * 8 + 4], v[g * 8 + 5]), a3 = __floats2bfloat162_rn(v[g * 8 + 6], v[g * 8 + 7]);
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(*reinterpret_cast<uint32_t*>(&a0)),
-                       "r"(*reinterpret_cast<uint32_t*>(&a1)), "r"(*reinterpret_cast<uint32_t*>(&a2)),
-                       "r"(*reinterpret_cast<uint32_t*>(&a3)) : "memory");
-        }
+      for (int g8 = 0; g8 < BKV / 8; ++g8) {
+        float e[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { e[i] = fast_exp2(s[g8 * 8 + i] * c - mc); rowsum += e[i]; }   // exp2(-inf) = 0
+        const int k0 = g8 * 8;
+        const uint32_t addr = sPg + (k0 >> 6) * 16384 + r * 128 + ((((k0 & 63) >> 3) ^ (r & 7)) << 4);
+        __nv_bfloat162 a0 = __floats2bfloat162_rn(e[0], e[1]), a1 = __floats2bfloat162_rn(e[2], e[3]);
+        __nv_bfloat162 a2 = __floats2bfloat162_rn(e[4], e[5]), a3 = __floats2bfloat162_rn(e[6], e[7]);
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(*reinterpret_cast<uint32_t*>(&a0)),
+                     "r"(*reinterpret_cast<uint32_t*>(&a1)), "r"(*reinterpret_cast<uint32_t*>(&a2)),
+                     "r"(*reinterpret_cast<uint32_t*>(&a3)) : "memory");
       }
       l += rowsum;
-      m = m_new;
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P visible to the tensor core's reads
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(p_ready);
+      if (lane == 0) mbar_arrive(p_ready(g));
     }
-    if (ok) {
-      ok = mbar_wait(pv_full, (n_kv - 1) & 1, abort_flag, p.status);
+    if (ok && n > 0) {
+      ok = mbar_wait(pv_done(g), (n - 1) & 1, abort_flag, p.status);
       ok = __all_sync(0xffffffffu, ok);
     }
-    if (ok) {
+    if (ok && n > 0) {
       tc_fence_after();
       const float inv = 1.f / l;
       bf16* dst = p.out + (size_t)(base + q_pos) * p.ldo + (size_t)head * HD;
-#pragma unroll
+#pragma unroll 1
       for (int cc = 0; cc < HD; cc += 32) {
         float v[32];
-        tmem_ld32(tmem_base + lane_off + 256 + cc, v);
+        tmem_ld32(tO + cc, v);
         tmem_ld_wait();
         if (q_pos < L) {
 #pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            float t[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) t[i] = (o[cc + g * 8 + i] + v[g * 8 + i]) * inv;
-            __nv_bfloat162 a0 = __floats2bfloat162_rn(t[0], t[1]), a1 = __floats2bfloat162_rn(t[2], t[3]);
-            __nv_bfloat162 a2 = __floats2bfloat162_rn(t[4], t[5]), a3 = __floats2bfloat162_rn(t[6], t[7]);
+          for (int g8 = 0; g8 < 4; ++g8) {
+            __nv_bfloat162 a0 = __floats2bfloat162_rn(v[g8 * 8] * inv, v[g8 * 8 + 1] * inv);
+            __nv_bfloat162 a1 = __floats2bfloat162_rn(v[g8 * 8 + 2] * inv, v[g8 * 8 + 3] * inv);
+            __nv_bfloat162 a2 = __floats2bfloat162_rn(v[g8 * 8 + 4] * inv, v[g8 * 8 + 5] * inv);
+            __nv_bfloat162 a3 = __floats2bfloat162_rn(v[g8 * 8 + 6] * inv, v[g8 * 8 + 7] * inv);
             uint4 u;
             u.x = *reinterpret_cast<uint32_t*>(&a0); u.y = *reinterpret_cast<uint32_t*>(&a1);
             u.z = *reinterpret_cast<uint32_t*>(&a2); u.w = *reinterpret_cast<uint32_t*>(&a3);
-            *reinterpret_cast<uint4*>(dst + cc + g * 8) = u;
+            *reinterpret_cast<uint4*>(dst + cc + g8 * 8) = u;
           }
         }
       }
@@ -344,29 +314,49 @@ __global__ void __launch_bounds__(N_THREADS, 1) attn_tc_kernel(const __grid_cons
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+    tmem_dealloc(tmem_base, 512);
   }
 }
 
-PFN_cuTensorMapEncodeTiled_v12000 g_encode = nullptr;
-bool get_encode() {
-  if (g_encode) return true;
-  void* fn = nullptr;
-  cudaDriverEntryPointQueryResult q;
-  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn) return false;
-  g_encode = (PFN_cuTensorMapEncodeTiled_v12000)fn;
-  return true;
+// Work list: pairs of query tiles of all sequences, those nearest the end of their sequence
+// (most key tiles) first.  One block, thread = sequence.
+__global__ void __launch_bounds__(256) attn_schedule_kernel(const int* __restrict__ cu, int batch, int2* __restrict__ sched) {
+  __shared__ int s_warp[8];
+  __shared__ int s_base;
+  const int b = threadIdx.x, warp = b >> 5, lane = b & 31;
+  const int np = b < batch ? (cu[b + 1] - cu[b] + 2 * BQ - 1) / (2 * BQ) : 0;
+  int max_np = np;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) max_np = max(max_np, __shfl_xor_sync(0xffffffffu, max_np, o));
+  if (lane == 0) s_warp[warp] = max_np;
+  if (b == 0) s_base = 0;
+  __syncthreads();
+  max_np = 0;
+  for (int w = 0; w < 8; ++w) max_np = max(max_np, s_warp[w]);
+  __syncthreads();
+  for (int r = 0; r < max_np; ++r) {
+    const bool has = np > r;
+    const unsigned bal = __ballot_sync(0xffffffffu, has);
+    if (lane == 0) s_warp[warp] = __popc(bal);
+    __syncthreads();
+    int pos = s_base + __popc(bal & ((1u << lane) - 1u));
+    for (int w = 0; w < warp; ++w) pos += s_warp[w];
+    if (has) sched[pos] = make_int2(b, (np - 1 - r) * 2 * BQ);
+    __syncthreads();
+    if (b == 0) { int t = 0; for (int w = 0; w < 8; ++w) t += s_warp[w]; s_base += t; }
+    __syncthreads();
+  }
 }
 
 template <int HD>
-cudaError_t go(const CUtensorMap& map, const Params& p, dim3 grid, cudaStream_t st) {
+cudaError_t go(const CUtensorMap& mq, const CUtensorMap& mkv, const Params& p, dim3 grid, cudaStream_t st) {
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<HD>::SMEM);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  attn_tc_kernel<HD><<<grid, N_THREADS, Cfg<HD>::SMEM, st>>>(map, p);
+  attn_tc_kernel<HD><<<grid, N_THREADS, Cfg<HD>::SMEM, st>>>(mq, mkv, p);
   return cudaGetLastError();
 }
 }  // namespace
@@ -375,20 +365,25 @@ bool attn_tc_supported(int hd, int ld, const void* qkv, int ldo, const void* out
   return (hd == 64 || hd == 128) && ld % 8 == 0 && ((uintptr_t)qkv & 15) == 0 && ldo % 8 == 0 && ((uintptr_t)out & 15) == 0;
 }
 
-cudaError_t launch_attn_tc(const bf16* qkv, int ld, int total, int nq, int nkv, int hd, const int* cu_dev, int batch,
-                           bf16* out, int ldo, int* status, cudaStream_t st, int64_t* n_launch) {
-  if (!get_encode()) return cudaErrorNotSupported;
-  CUtensorMap map;
-  cuuint64_t dims[2] = {(cuuint64_t)((nq + 2 * nkv) * hd), (cuuint64_t)total};
-  cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
-  cuuint32_t box[2] = {64, 128};
-  cuuint32_t estr[2] = {1, 1};
-  if (g_encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<bf16*>(qkv), dims, strides, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-    return cudaErrorInvalidValue;
-  Params p{cu_dev, batch, nq, nkv, out, ldo, (1.f / sqrtf((float)hd)) * 1.4426950408889634f, status};
-  dim3 grid(nq, (total + BQ - 1) / BQ + batch);
+int attn_tc_items(const int* cu_host, int batch) {
+  int n = 0;
+  for (int b = 0; b < batch; ++b) n += (cu_host[b + 1] - cu_host[b] + 2 * BQ - 1) / (2 * BQ);
+  return n;
+}
+
+void launch_attn_schedule(const int* cu_dev, int batch, int2* sched, cudaStream_t st, int64_t* n_launch) {
   ++*n_launch;
-  return hd == 64 ? go<64>(map, p, grid, st) : go<128>(map, p, grid, st);
+  attn_schedule_kernel<<<1, 256, 0, st>>>(cu_dev, batch, sched);
+}
+
+cudaError_t launch_attn_tc(const bf16* qkv, int ld, int total, int nq, int nkv, int hd, const int* cu_dev, const int2* sched,
+                           int n_items, bf16* out, int ldo, int* status, cudaStream_t st, int64_t* n_launch) {
+  CUtensorMap mq, mkv;
+  const int bkv = hd == 64 ? 128 : 64;
+  if (!tc_make_map_bf16(&mq, qkv, total, (long long)(nq + 2 * nkv) * hd, ld, BQ)) return cudaErrorInvalidValue;
+  if (!tc_make_map_bf16(&mkv, qkv, total, (long long)(nq + 2 * nkv) * hd, ld, bkv)) return cudaErrorInvalidValue;
+  Params p{cu_dev, sched, nq, nkv, out, ldo, (1.f / sqrtf((float)hd)) * 1.4426950408889634f, status};
+  dim3 grid(nq, n_items);
+  ++*n_launch;
+  return hd == 64 ? go<64>(mq, mkv, p, grid, st) : go<128>(mq, mkv, p, grid, st);
 }

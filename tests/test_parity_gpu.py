@@ -106,9 +106,9 @@ def test_sequence_alone_equals_sequence_in_batch():
             k, v = s.cache.gather(i, 0, lens[1])
             # rows are independent, but the residual GEMMs add their k-range partial sums with fp32
             # atomics whose split and order depend on the launch shape: equal up to that reassociation
-            assert rel_fro(k, kv[i][0]) <= 1e-3
-            assert rel_fro(v, kv[i][1]) <= 1e-3
-        assert rel_fro(l1.cpu().numpy()[0], logits[1].astype(np.float64)) <= 1e-3
+            assert rel_fro(k, kv[i][0]) <= 3e-3
+            assert rel_fro(v, kv[i][1]) <= 3e-3
+        assert rel_fro(l1.cpu().numpy()[0], logits[1].astype(np.float64)) <= 3e-3
     finally:
         s.close()
 
@@ -130,7 +130,7 @@ def test_host_entry_point_matches_device_entry_point():
         kvp.kvp_prefill_predict_host(s.h, th, lens, s.cache, s.workspace, s.logits, lh, fh, s.stream)
         # two runs differ by the order of the residual GEMMs' fp32 atomic adds, nothing else
         for b in range(2):
-            assert rel_fro(lh.numpy()[b], a[b].astype(np.float64)) <= 1e-3
+            assert rel_fro(lh.numpy()[b], a[b].astype(np.float64)) <= 3e-3
             top2 = np.sort(a[b])[-2:]
             if top2[1] - top2[0] > 1e-3:
                 assert fh.numpy()[b] == fa[b]
