@@ -228,14 +228,16 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       if (lane == 0) mbar_arrive(s_free(g));
       const int kbase = j * BKV;
       const bool diag = kbase + BKV - 1 > qs;     // some key of this tile lies above some query of the tile
-      float mt = -INFINITY;
       if (diag) {
 #pragma unroll
-        for (int i = 0; i < BKV; ++i) { if (kbase + i > q_pos) s[i] = -INFINITY; mt = fmaxf(mt, s[i]); }
-      } else {
-#pragma unroll
-        for (int i = 0; i < BKV; ++i) mt = fmaxf(mt, s[i]);
+        for (int i = 0; i < BKV; ++i) if (kbase + i > q_pos) s[i] = -INFINITY;
       }
+      float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};    // four chains instead of one of length BKV
+#pragma unroll
+      for (int i = 0; i < BKV; i += 4) {
+        mx[0] = fmaxf(mx[0], s[i]); mx[1] = fmaxf(mx[1], s[i + 1]); mx[2] = fmaxf(mx[2], s[i + 2]); mx[3] = fmaxf(mx[3], s[i + 3]);
+      }
+      const float mt = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
       if (j > 0) {     // the previous P V product has read P and finished writing O
         ok = mbar_wait(pv_done(g), (j - 1) & 1, abort_flag, p.status);
         ok = __all_sync(0xffffffffu, ok);
@@ -261,12 +263,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         if (need) m_ref = mt;
       }
       const float mc = (m_ref == -INFINITY) ? 0.f : m_ref * c;
-      float rowsum = 0.f;
+      float rs[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int g8 = 0; g8 < BKV / 8; ++g8) {
         float e[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) { e[i] = fast_exp2(s[g8 * 8 + i] * c - mc); rowsum += e[i]; }   // exp2(-inf) = 0
+        for (int i = 0; i < 8; ++i) { e[i] = fast_exp2(s[g8 * 8 + i] * c - mc); rs[i & 3] += e[i]; }   // exp2(-inf) = 0
         const int k0 = g8 * 8;
         const uint32_t addr = sPg + (k0 >> 6) * 16384 + r * 128 + ((((k0 & 63) >> 3) ^ (r & 7)) << 4);
         __nv_bfloat162 a0 = __floats2bfloat162_rn(e[0], e[1]), a1 = __floats2bfloat162_rn(e[2], e[3]);
@@ -275,7 +277,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                      "r"(*reinterpret_cast<uint32_t*>(&a1)), "r"(*reinterpret_cast<uint32_t*>(&a2)),
                      "r"(*reinterpret_cast<uint32_t*>(&a3)) : "memory");
       }
-      l += rowsum;
+      l += (rs[0] + rs[1]) + (rs[2] + rs[3]);
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P visible to the tensor core's reads
       tc_fence_before();
       __syncwarp();
