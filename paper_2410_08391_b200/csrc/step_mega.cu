@@ -539,17 +539,24 @@ __global__ void __launch_bounds__(NT, 1) step_mega_kernel(const __grid_constant_
         float mm = -INFINITY;
         for (int s = lane; s < p.n_split; s += 32) mm = fmaxf(mm, __ldcg(pr + (size_t)s * ldr + p.hd));
         mm = warp_max(mm);
-        for (int c = lane; c < p.hd; c += 32) {
-          float ll = 0.f, oo = 0.f;
-          for (int s = 0; s < p.n_split; ++s) {
-            const float* r = pr + (size_t)s * ldr;
-            float ms = __ldcg(r + p.hd);
-            float f = (ms == -INFINITY) ? 0.f : __expf(ms - mm);
-            ll += __ldcg(r + p.hd + 1) * f;
-            oo += __ldcg(r + c) * f;
-          }
-          p.ab[(size_t)it * p.hd + c] = oo / ll;
+        // the loads of different splits do not depend on one another: unrolled, they are in flight together
+        float ll = 0.f, o0 = 0.f, o1 = 0.f, o2 = 0.f, o3 = 0.f;
+#pragma unroll 8
+        for (int s = 0; s < p.n_split; ++s) {
+          const float* r = pr + (size_t)s * ldr;
+          const float ms = __ldcg(r + p.hd);
+          const float f = (ms == -INFINITY) ? 0.f : __expf(ms - mm);
+          ll = fmaf(__ldcg(r + p.hd + 1), f, ll);
+          if (lane < p.hd) o0 = fmaf(__ldcg(r + lane), f, o0);
+          if (lane + 32 < p.hd) o1 = fmaf(__ldcg(r + lane + 32), f, o1);
+          if (lane + 64 < p.hd) o2 = fmaf(__ldcg(r + lane + 64), f, o2);
+          if (lane + 96 < p.hd) o3 = fmaf(__ldcg(r + lane + 96), f, o3);
         }
+        float* dst = p.ab + (size_t)it * p.hd;
+        if (lane < p.hd) dst[lane] = o0 / ll;
+        if (lane + 32 < p.hd) dst[lane + 32] = o1 / ll;
+        if (lane + 64 < p.hd) dst[lane + 64] = o2 / ll;
+        if (lane + 96 < p.hd) dst[lane + 96] = o3 / ll;
       }
       BARRIER();
     }
