@@ -589,6 +589,14 @@ void launch_step_attn(const LaunchCtx& ctx, const float* q, int ldq, int nq, int
   fill_inv_freq(&inv, hd, theta);
   int n_split = step_attn_splits(batch, nkv, max_keys);
   dim3 grid(n_split, nkv, batch);
+  if (step_attn_ring_supported(ctx.dtype, nq, nkv, hd, kpool, vpool)) {
+    launch_step_attn_ring(ctx, q, ldq, nq, nkv, hd, theta, kpool, vpool, block_table, mpps, n_pages, seq_lens, extra, batch, n_split, part, out);
+    if (n_split > 1) {
+      ++*ctx.n_launch;
+      step_attn_merge_kernel<<<dim3(nq, batch), 64, 0, ctx.st>>>(part, nq, hd, n_split, out);
+    }
+    return;
+  }
   ++*ctx.n_launch;
   if (hd == 16 || hd == 32 || hd == 64 || hd == 128) {
     int es = ctx.dtype == 0 ? 4 : 2;
