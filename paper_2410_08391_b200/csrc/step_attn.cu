@@ -136,7 +136,7 @@ __global__ void __launch_bounds__(512) step_attn_ring_kernel(const float* __rest
     const unsigned char* Vs = Ks + PAGE_BYTES;
     // ---- scores
     {
-      float sc = 0.f;
+      float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;     // four short chains instead of one of HD steps
       const unsigned char* kr = Ks + key * (HD * 2);
       const float* qh = qs + h * HD;
 #pragma unroll 4
@@ -144,12 +144,12 @@ __global__ void __launch_bounds__(512) step_attn_ring_kernel(const float* __rest
         const int c = (i + key) & (CH - 1);
         const uint4 u = *reinterpret_cast<const uint4*>(kr + c * 16);
         const float4 q0 = *reinterpret_cast<const float4*>(qh + c * 8), q1 = *reinterpret_cast<const float4*>(qh + c * 8 + 4);
-        sc = fmaf(__uint_as_float(u.x << 16), q0.x, sc); sc = fmaf(__uint_as_float(u.x & 0xffff0000u), q0.y, sc);
-        sc = fmaf(__uint_as_float(u.y << 16), q0.z, sc); sc = fmaf(__uint_as_float(u.y & 0xffff0000u), q0.w, sc);
-        sc = fmaf(__uint_as_float(u.z << 16), q1.x, sc); sc = fmaf(__uint_as_float(u.z & 0xffff0000u), q1.y, sc);
-        sc = fmaf(__uint_as_float(u.w << 16), q1.z, sc); sc = fmaf(__uint_as_float(u.w & 0xffff0000u), q1.w, sc);
+        s0 = fmaf(__uint_as_float(u.x << 16), q0.x, s0); s1 = fmaf(__uint_as_float(u.x & 0xffff0000u), q0.y, s1);
+        s2 = fmaf(__uint_as_float(u.y << 16), q0.z, s2); s3 = fmaf(__uint_as_float(u.y & 0xffff0000u), q0.w, s3);
+        s0 = fmaf(__uint_as_float(u.z << 16), q1.x, s0); s1 = fmaf(__uint_as_float(u.z & 0xffff0000u), q1.y, s1);
+        s2 = fmaf(__uint_as_float(u.w << 16), q1.z, s2); s3 = fmaf(__uint_as_float(u.w & 0xffff0000u), q1.w, s3);
       }
-      ps[h * PAGE_TOKENS + key] = key < nk ? sc : -INFINITY;
+      ps[h * PAGE_TOKENS + key] = key < nk ? (s0 + s1) + (s2 + s3) : -INFINITY;
     }
     __syncthreads();
     // ---- running softmax statistics, one warp per head
@@ -172,23 +172,34 @@ __global__ void __launch_bounds__(512) step_attn_ring_kernel(const float* __rest
     {
       const float a = alpha[h];
       const float* pr = ps + h * PAGE_TOKENS;
+      // keys beyond nk carry p = 0 but their rows are not initialised memory: they are not read
       if (DP == 2) {
-        float a0 = acc[0] * a, a1 = acc[DP - 1] * a;
+        float a0 = acc[0] * a, a1 = acc[DP - 1] * a, b0 = 0.f, b1 = 0.f;
         const uint32_t* vr = reinterpret_cast<const uint32_t*>(Vs) + key;
-#pragma unroll 8
-        for (int s = 0; s < nk; ++s) {
-          const uint32_t u = vr[s * (HD / 2)];
-          const float pv = pr[s];
-          a0 = fmaf(pv, __uint_as_float(u << 16), a0);
-          a1 = fmaf(pv, __uint_as_float(u & 0xffff0000u), a1);
+        int s = 0;
+#pragma unroll 4
+        for (; s + 2 <= nk; s += 2) {
+          const uint32_t u = vr[s * (HD / 2)], w = vr[(s + 1) * (HD / 2)];
+          const float pu = pr[s], pw = pr[s + 1];
+          a0 = fmaf(pu, __uint_as_float(u << 16), a0); a1 = fmaf(pu, __uint_as_float(u & 0xffff0000u), a1);
+          b0 = fmaf(pw, __uint_as_float(w << 16), b0); b1 = fmaf(pw, __uint_as_float(w & 0xffff0000u), b1);
         }
-        acc[0] = a0; acc[DP - 1] = a1;
+        if (s < nk) {
+          const uint32_t u = vr[s * (HD / 2)];
+          a0 = fmaf(pr[s], __uint_as_float(u << 16), a0); a1 = fmaf(pr[s], __uint_as_float(u & 0xffff0000u), a1);
+        }
+        acc[0] = a0 + b0; acc[DP - 1] = a1 + b1;
       } else {
-        float a0 = acc[0] * a;
+        float a0 = acc[0] * a, b0 = 0.f, c0 = 0.f, d0 = 0.f;
         const bf16* vr = reinterpret_cast<const bf16*>(Vs) + key;
-#pragma unroll 8
-        for (int s = 0; s < nk; ++s) a0 = fmaf(pr[s], __bfloat162float(vr[s * HD]), a0);
-        acc[0] = a0;
+        int s = 0;
+#pragma unroll 2
+        for (; s + 4 <= nk; s += 4) {
+          a0 = fmaf(pr[s], __bfloat162float(vr[s * HD]), a0); b0 = fmaf(pr[s + 1], __bfloat162float(vr[(s + 1) * HD]), b0);
+          c0 = fmaf(pr[s + 2], __bfloat162float(vr[(s + 2) * HD]), c0); d0 = fmaf(pr[s + 3], __bfloat162float(vr[(s + 3) * HD]), d0);
+        }
+        for (; s < nk; ++s) a0 = fmaf(pr[s], __bfloat162float(vr[s * HD]), a0);
+        acc[0] = (a0 + b0) + (c0 + d0);
       }
     }
   }

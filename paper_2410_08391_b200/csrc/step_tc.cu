@@ -171,23 +171,34 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
   }
 }
 
-// One CTA per operand row (pad rows included).
+// grid (operand row incl. pad rows, chunk of PREP_CHUNK elements); 8 elements per thread and step.
+// Every CTA of a row recomputes the row's sum of squares (the row is a few KB in L2), so the
+// chunks need no second kernel.
+constexpr int PREP_CHUNK = 2048;
+
 __global__ void __launch_bounds__(256) step_prep_kernel(int mode, const float* __restrict__ x, int ldx, int K, int batch, int Bp,
                                                         const float* __restrict__ gain, float eps, RowMap mg, RowMap mu,
                                                         bf16* __restrict__ XB, float* zero_ptr, int zero_ld, int zero_n) {
   __shared__ float red[8];
   const int b = blockIdx.x, tid = threadIdx.x;
+  const int k_begin = blockIdx.y * PREP_CHUNK, k_end = min(K, k_begin + PREP_CHUNK);
   bf16* hi = XB + (size_t)b * K;
   bf16* lo = XB + (size_t)(Bp + b) * K;
   if (b >= batch) {
-    for (int k = tid; k < K; k += 256) { hi[k] = __float2bfloat16_rn(0.f); lo[k] = __float2bfloat16_rn(0.f); }
+    for (int k = k_begin + tid * 8; k < k_end; k += 2048) {
+      *reinterpret_cast<uint4*>(hi + k) = make_uint4(0, 0, 0, 0);
+      *reinterpret_cast<uint4*>(lo + k) = make_uint4(0, 0, 0, 0);
+    }
     return;
   }
   const float* xr = x + (size_t)b * ldx;
   float r = 1.f;
   if (mode == PREP_NORM) {
     float ss = 0.f;
-    for (int k = tid; k < K; k += 256) { float v = xr[k]; ss = fmaf(v, v, ss); }
+    for (int k = tid * 4; k < K; k += 1024) {
+      const float4 v = *reinterpret_cast<const float4*>(xr + k);
+      ss = fmaf(v.x, v.x, ss); ss = fmaf(v.y, v.y, ss); ss = fmaf(v.z, v.z, ss); ss = fmaf(v.w, v.w, ss);
+    }
     ss = warp_sum(ss);
     if ((tid & 31) == 0) red[tid >> 5] = ss;
     __syncthreads();
@@ -196,22 +207,43 @@ __global__ void __launch_bounds__(256) step_prep_kernel(int mode, const float* _
     for (int w = 0; w < 8; ++w) t += red[w];
     r = rsqrtf(t / (float)K + eps);
   }
-  for (int k = tid; k < K; k += 256) {
-    float v;
+  for (int k = k_begin + tid * 8; k < k_end; k += 2048) {
+    float v[8];
     if (mode == PREP_SWIGLU) {
-      float g = xr[map_row(mg, k)], u = xr[map_row(mu, k)];
-      v = g / (1.f + __expf(-g)) * u;
-    } else if (mode == PREP_NORM) {
-      v = gain[k] * xr[k] * r;
+      // gate and up rows of 8 consecutive outputs are 8 consecutive elements each (interleave blocks are multiples of 8)
+      const float* g = xr + map_row(mg, k);
+      const float* u = xr + map_row(mu, k);
+      const float4 g0 = *reinterpret_cast<const float4*>(g), g1 = *reinterpret_cast<const float4*>(g + 4);
+      const float4 u0 = *reinterpret_cast<const float4*>(u), u1 = *reinterpret_cast<const float4*>(u + 4);
+      const float gv[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w}, uv[8] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[i] = __fdividef(gv[i], 1.f + __expf(-gv[i])) * uv[i];
     } else {
-      v = xr[k];
+      const float4 a0 = *reinterpret_cast<const float4*>(xr + k), a1 = *reinterpret_cast<const float4*>(xr + k + 4);
+      v[0] = a0.x; v[1] = a0.y; v[2] = a0.z; v[3] = a0.w; v[4] = a1.x; v[5] = a1.y; v[6] = a1.z; v[7] = a1.w;
+      if (mode == PREP_NORM) {
+        const float4 c0 = *reinterpret_cast<const float4*>(gain + k), c1 = *reinterpret_cast<const float4*>(gain + k + 4);
+        const float gg[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = gg[i] * v[i] * r;
+      }
     }
-    bf16 h = __float2bfloat16_rn(v);
-    hi[k] = h;
-    lo[k] = __float2bfloat16_rn(v - __bfloat162float(h));
+    uint32_t h[4], l[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const __nv_bfloat162 hh = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+      const float2 hf = __bfloat1622float2(hh);
+      const __nv_bfloat162 ll = __floats2bfloat162_rn(v[2 * i] - hf.x, v[2 * i + 1] - hf.y);
+      h[i] = *reinterpret_cast<const uint32_t*>(&hh);
+      l[i] = *reinterpret_cast<const uint32_t*>(&ll);
+    }
+    *reinterpret_cast<uint4*>(hi + k) = make_uint4(h[0], h[1], h[2], h[3]);
+    *reinterpret_cast<uint4*>(lo + k) = make_uint4(l[0], l[1], l[2], l[3]);
   }
-  if (zero_ptr)
-    for (int i = tid; i < zero_n; i += 256) zero_ptr[(size_t)b * zero_ld + i] = 0.f;
+  if (zero_ptr) {
+    const int n_chunks = gridDim.y;
+    for (int i = blockIdx.y * 256 + tid; i < zero_n; i += n_chunks * 256) zero_ptr[(size_t)b * zero_ld + i] = 0.f;
+  }
 }
 
 int pow2_ceil(int v) { int p = 1; while (p < v) p <<= 1; return p; }
@@ -228,7 +260,7 @@ void launch_step_prep(const LaunchCtx& ctx, int mode, const float* x, int ldx, i
   const int Bp = step_tc_rows(batch);
   RowMap mg{0, G, 0, K}, mu{G == 0 ? K : 0, G, 1, K};
   ++*ctx.n_launch;
-  step_prep_kernel<<<Bp, 256, 0, ctx.st>>>(mode, x, ldx, K, batch, Bp, gain, eps, mg, mu, XB, zero_ptr, zero_ld, zero_n);
+  step_prep_kernel<<<dim3(Bp, (K + PREP_CHUNK - 1) / PREP_CHUNK), 256, 0, ctx.st>>>(mode, x, ldx, K, batch, Bp, gain, eps, mg, mu, XB, zero_ptr, zero_ld, zero_n);
 }
 
 cudaError_t launch_step_gemm_tc(const bf16* W, int ldw, int N, int K, const bf16* XB, int batch, float* Y, int ldy, int n_sm,
