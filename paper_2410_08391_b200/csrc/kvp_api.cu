@@ -376,6 +376,16 @@ kvp_status kvp_create(const kvp_model_cfg* aux, const kvp_model_cfg* base, const
   if (const char* e = getenv("KVP_NO_TC")) h->use_tc = !(e[0] == '1');
   if (const char* e = getenv("KVP_NO_GRAPH")) h->use_graph = !(e[0] == '1');
   if (const char* e = getenv("KVP_NO_MEGA")) h->use_mega = !(e[0] == '1');
+  if (const char* e = getenv("KVP_NO_SIDE")) h->use_side = !(e[0] == '1');
+  if (h->use_side) {
+    if (cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking) != cudaSuccess) h->side = nullptr;
+    if (h->side && (cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+                    cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming) != cudaSuccess)) {
+      cudaStreamDestroy(h->side);
+      h->side = nullptr;
+    }
+    cudaGetLastError();
+  }
   size_t off = 0;
   bool bf = opt->dtype == KVP_BF16;
   plan_model(h->aux, aux, h->es, bf, off, false);
@@ -546,6 +556,9 @@ static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int
     KVP_TIMED(KVP_CLASS_OTHER, launch_attn_schedule(cu_dev, batch, attn_sched, ctx.st, ctx.n_launch));
   }
   // ---- stage 1 + 2: auxiliary prefill, each layer's K/V pushed through the predictor ----
+  // (only worth it while a layer's kernels leave SMs idle: with many tokens every kernel fills the GPU by itself)
+  const bool fork = h->side != nullptr && !h->timing && T <= 4096;
+  bool pending_join = false;
   KVP_TIMED(KVP_CLASS_OTHER, launch_embed(ctx, tokens, nullptr, T, P + A.embed, A.vocab, A.d, x));
   for (int j = 0; j <= h->j_max; ++j) {
     const LayerPlan& L = A.L[j];
@@ -553,6 +566,10 @@ static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int
     KVP_TIMED(KVP_CLASS_OTHER, launch_rmsnorm(ctx, x, (const float*)(P + L.attn_norm), A.eps, T, A.d, hbuf, h->opt.dtype, h_lo));
     int col_begin = last ? L.dq : 0;
     const int n_out = L.nqkv - col_begin, q_heads = last ? 0 : L.nq;
+    if (pending_join) {   // the previous layer's predictor still reads the K/V buffers this projection overwrites
+      cudaStreamWaitEvent(s, h->ev_join, 0);
+      pending_join = false;
+    }
     TcGemm tq{};
     tq.A = (const bf16*)hbuf; tq.lda = A.d; tq.A2 = (const bf16*)h_lo; tq.lda2 = A.d; tq.split_begin = L.dq - col_begin;
     tq.W = (const bf16*)(P + L.wqkv + (size_t)col_begin * A.d * es); tq.ldw = A.d; tq.M = T; tq.N = n_out; tq.K = A.d;
@@ -573,6 +590,13 @@ static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int
     // predictor: K_hat_i = K_A,j FK_i^T, V_hat_i = V_A,j FV_i^T for every base layer i with j_i = j
     const PredGroup& pg = h->groups[j];
     if (pg.n_seg > 0) {
+      LaunchCtx pctx = ctx;
+      if (fork) {
+        cudaEventRecord(h->ev_fork, s);
+        cudaStreamWaitEvent(h->side, h->ev_fork, 0);
+        pctx.st = h->side;
+      }
+      const LaunchCtx& ctx = pctx;      // the predictor's launches go to the side stream
       for (int kv = 0; kv < 2; ++kv) {
         GemmArgs p{};
         p.A = qkv + (size_t)(L.dq + kv * L.dkv) * es; p.lda = L.nqkv; p.M = T; p.K = L.dkv;
@@ -593,6 +617,10 @@ static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int
         tp.W = (const bf16*)p.W; tp.ldw = p.ldw; tp.M = T; tp.N = p.N; tp.K = p.K; tp.epi = TC_PAGED; tp.paged = p.paged;
         if (!try_tc(h, ctx, tp, KVP_CLASS_PREDICTOR, &tc_err))
           KVP_TIMED(KVP_CLASS_PREDICTOR, launch_gemm_simt(ctx, p, EPI_PAGED));
+      }
+      if (fork) {
+        cudaEventRecord(h->ev_join, h->side);
+        pending_join = true;
       }
     }
     if (last) break;
@@ -627,6 +655,7 @@ static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int
     td.epi = TC_RESID; td.X = x; td.ldx = A.d;
     if (!try_tc(h, ctx, td, KVP_CLASS_AUX_GEMM, &tc_err)) KVP_TIMED(KVP_CLASS_AUX_GEMM, launch_gemm_simt(ctx, d, EPI_RESID));
   }
+  if (pending_join) cudaStreamWaitEvent(s, h->ev_join, 0);     // the base step reads what the predictor wrote
   if (tc_err != cudaSuccess) return fail(h, KVP_ERR_CUDA, "tensor-core GEMM launch: %s", cudaGetErrorString(tc_err));
   // ---- stage 3: one base step per sequence on its last prompt token ----
   if (!base_step_fused(h, ctx, cache, w, ws, batch, cs.max_len, false, tokens, last_idx, logits_out, first_token, &tc_err)) {

@@ -71,6 +71,11 @@ struct kvp_handle {
   bool use_graph = true;
   bool use_mega = true;                 // persistent kernel for the base step when it applies
   uint64_t graph_clock = 0;
+  // The predictor GEMMs of an auxiliary layer depend only on that layer's K/V projection, so they
+  // run on a stream of the handle's own beside the layer's attention and FFN (fork / join by events).
+  cudaStream_t side = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+  bool use_side = true;
   // instrumentation
   struct TimingRec { int cls; int64_t launches; cudaEvent_t a, b; };
   bool timing = false;
@@ -80,6 +85,9 @@ struct kvp_handle {
     for (auto& r : recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
     for (auto e : free_events) cudaEventDestroy(e);
     for (auto& g : graphs) cudaGraphExecDestroy(g.exec);
+    if (ev_fork) cudaEventDestroy(ev_fork);
+    if (ev_join) cudaEventDestroy(ev_join);
+    if (side) cudaStreamDestroy(side);
   }
 };
 
