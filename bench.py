@@ -221,7 +221,7 @@ def main():
     alg = {  # algorithmic work of each class per step: (amount, bound, unit scale)
         "aux_gemm": (work["aux_gemm_flops"], "tensor"), "aux_attn": (work["attn_flops"], "tensor"),
         "predictor": (work["pred_flops"], "tensor"), "step_gemv": (work["step_weight_bytes"], "hbm"),
-        "step_attn": (work["cache_bytes"], "hbm"),
+        "step_attn": (work["cache_bytes"], "hbm"), "step_fused": (work["step_bytes"], "hbm"),
     }
     dom = max(alg, key=lambda c: per_step[c][0])
     amount, bound = alg[dom]
@@ -239,6 +239,16 @@ def main():
                 "launches_per_step": per_step[dom][1], "avg_launch_ms": per_step[dom][0] / max(per_step[dom][1], 1),
                 "class_ms_per_step": {c: round(v[0], 4) for c, v in per_step.items()},
                 "timing": "separate pass with CUDA events around every launch"}
+    def frac_of(c):
+        amt, bnd = alg[c]
+        t = per_step[c][0] * 1e-3
+        if t <= 0:
+            return None
+        if bnd == "tensor":
+            pk = (peaks["bf16_tflops_sustained"] or peaks["bf16_tflops"]) / (16.0 if pair.dtype == "f32" else 1.0)
+            return {"bound": bnd, "achieved": amt / t / 1e12, "peak": pk, "unit": "TFLOP/s", "frac": amt / t / 1e12 / pk}
+        return {"bound": bnd, "achieved": amt / t / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": amt / t / 1e9 / peaks["hbm_gbs"]}
+    roofline["per_class"] = {c: frac_of(c) for c in alg if per_step[c][0] > 0}
     t12 = (per_step["aux_gemm"][0] + per_step["aux_attn"][0] + per_step["predictor"][0]) * 1e-3
     tensor_frac = work["tensor_flops"] / max(t12, 1e-12) / 1e12 / (peaks["bf16_tflops_sustained"] or peaks["bf16_tflops"])
 
