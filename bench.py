@@ -91,6 +91,21 @@ def blas_threads() -> int:
         return os.cpu_count() or 1
 
 
+def max_over_ranks(ms: float, dist, device) -> float:
+    """Slowest rank's time: the replicas run side by side, the job is done when the last one is."""
+    if dist is None:
+        return float(ms)
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(tokens_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Prompt tokens per second of all replicas together."""
+    return world * tokens_per_rank / (ms_per_step * 1e-3)
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -180,12 +195,9 @@ def main():
     ms = e0.elapsed_time(e1)
     clocks = sampler.stop(t0, t1) if sampler else None
     sess.poll()
-    if dist is not None:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, dist, dev)
     ms_step = ms / args.steps
-    value = world * work["tokens"] / (ms_step * 1e-3)
+    value = whole_job_value(work["tokens"], world, ms_step)
 
     # ---- end to end through the host entry point: pinned host tokens in, host logits out ----
     th = torch.from_numpy(pr.tokens).pin_memory()
@@ -203,11 +215,8 @@ def main():
         step_host()
     torch.cuda.synchronize()
     e2e_ms = (time.perf_counter() - w0) * 1e3 / args.steps
-    if dist is not None:
-        t = torch.tensor([e2e_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e_value = world * work["tokens"] / (e2e_ms * 1e-3)
+    e2e_ms = max_over_ranks(e2e_ms, dist, dev)
+    e2e_value = whole_job_value(work["tokens"], world, e2e_ms)
 
     # ---- per-kernel-class device times (separate pass: events around every launch) ----
     kvp.kvp_timing_enable(sess.h, True)
