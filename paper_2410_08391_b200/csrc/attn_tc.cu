@@ -86,16 +86,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   constexpr int BKV = C::BKV, QB = C::Q_BYTES, KB = C::KV_BYTES, PB = C::P_BYTES, NBOX = HD / 64;
   constexpr int KV_BOX = BKV * 128;     // bytes of one 64-column box of a K or V tile
   extern __shared__ uint8_t smem_raw[];
-  const int2 item = p.sched[blockIdx.y];
-  const int b = item.x, q0 = item.y;
-  const int base = p.cu[b], L = p.cu[b + 1] - base;
-  const int head = blockIdx.x, kvh = head / (p.nq / p.nkv);
-  // key tiles each query tile needs (tile 1 may lie beyond the end of the sequence)
-  int n_kv[2];
-  n_kv[0] = (min(L, q0 + BQ) + BKV - 1) / BKV;
-  n_kv[1] = q0 + BQ < L ? (min(L, q0 + 2 * BQ) + BKV - 1) / BKV : 0;
-  const int n_max = max(n_kv[0], n_kv[1]);
-
+  pdl_trigger();
+  if (threadIdx.x == 32) { prefetch_tensormap(&map_q); prefetch_tensormap(&map_kv); }
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t sQ = smem_u32(smem), sP = sQ + 2 * QB, sKV = sP + 2 * PB;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 2 * QB + 2 * PB + STAGES * 2 * KB);
@@ -124,6 +116,17 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();         // set-up above overlapped the previous kernel's tail; its results are needed from here on
+  const int2 item = p.sched[blockIdx.y];
+  const int b = item.x, q0 = item.y;
+  const int base = p.cu[b], L = p.cu[b + 1] - base;
+  const int head = blockIdx.x, kvh = head / (p.nq / p.nkv);
+  // key tiles each query tile needs (tile 1 may lie beyond the end of the sequence)
+  int n_kv[2];
+  n_kv[0] = (min(L, q0 + BQ) + BKV - 1) / BKV;
+  n_kv[1] = q0 + BQ < L ? (min(L, q0 + 2 * BQ) + BKV - 1) / BKV : 0;
+  const int n_max = max(n_kv[0], n_kv[1]);
+
 
   if (warp == 0) {
     if (lane == 0) {
@@ -358,8 +361,7 @@ cudaError_t go(const CUtensorMap& mq, const CUtensorMap& mkv, const Params& p, d
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  attn_tc_kernel<HD><<<grid, N_THREADS, Cfg<HD>::SMEM, st>>>(mq, mkv, p);
-  return cudaGetLastError();
+  return launch_overlapped(attn_tc_kernel<HD>, grid, dim3(N_THREADS), Cfg<HD>::SMEM, st, mq, mkv, p);
 }
 }  // namespace
 

@@ -20,6 +20,25 @@ template <> __device__ __forceinline__ bf16 from_f<bf16>(float v) { return __flo
 
 __device__ __forceinline__ void dev_flag(int* status, int code) { atomicCAS(status, DEV_OK, code); }
 
+// Programmatic dependent launch.  A kernel started with launch_overlapped() may begin while the
+// kernel before it in the stream is still running (once every CTA of that kernel has called
+// pdl_trigger() or exited); it must call pdl_wait() before its first access to global memory,
+// which returns when the earlier kernel has finished and its writes are visible.  Both calls do
+// nothing in a kernel launched the ordinary way.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <class... KArgs, class... Args>
+inline cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

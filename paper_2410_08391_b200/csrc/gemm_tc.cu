@@ -321,6 +321,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  pdl_trigger();      // the next kernel's CTAs may take SMs as this kernel's CTAs leave them
+  if (threadIdx.x == 32) {   // tensor maps on their way while the barriers and tensor memory are set up
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
+    if (p.has_a2) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a2) : "memory");
+  }
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 2); mbar_init(empty_bar(s), 1); }   // two loaders per stage
@@ -337,6 +343,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const int num_kb = (p.K + BK - 1) / BK;
+  pdl_wait();         // set-up above overlapped the previous kernel's tail; its results are needed from here on
 
   if (warp == 0 || warp == 2) {
     // ---------------- TMA producers: warp 0 loads the A tile of every stage, warp 2 the W tile ----------------
@@ -460,8 +467,7 @@ cudaError_t go(const CUtensorMap& a, const CUtensorMap& a2, const CUtensorMap& w
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  gemm_tc_kernel<EPI, BN><<<grid, N_THREADS, Tile<BN>::SMEM_BYTES, st>>>(a, a2, w, p);
-  return cudaGetLastError();
+  return launch_overlapped(gemm_tc_kernel<EPI, BN>, dim3(grid), dim3(N_THREADS), Tile<BN>::SMEM_BYTES, st, a, a2, w, p);
 }
 
 template <int BN>

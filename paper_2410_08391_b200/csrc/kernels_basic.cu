@@ -117,6 +117,8 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restr
                                int d, T* __restrict__ out, T* __restrict__ out_lo) {
   int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   int lane = threadIdx.x & 31;
+  pdl_trigger();
+  pdl_wait();
   if (row >= rows) return;
   const float* xr = x + (size_t)row * d;
   float ss = 0.f;
@@ -136,8 +138,8 @@ void launch_rmsnorm(const LaunchCtx& ctx, const float* x, const float* gain, flo
   if (rows == 0) return;
   LAUNCH_COUNT(ctx);
   int grid = (rows + 7) / 8;
-  if (out_dtype == 0) rmsnorm_kernel<float><<<grid, 256, 0, ctx.st>>>(x, gain, eps, rows, d, (float*)out, (float*)nullptr);
-  else rmsnorm_kernel<bf16><<<grid, 256, 0, ctx.st>>>(x, gain, eps, rows, d, (bf16*)out, (bf16*)out_lo);
+  if (out_dtype == 0) launch_overlapped(rmsnorm_kernel<float>, dim3(grid), dim3(256), 0, ctx.st, x, gain, eps, rows, d, (float*)out, (float*)nullptr);
+  else launch_overlapped(rmsnorm_kernel<bf16>, dim3(grid), dim3(256), 0, ctx.st, x, gain, eps, rows, d, (bf16*)out, (bf16*)out_lo);
 }
 
 // ---------------------------------------------------------------------------------------
