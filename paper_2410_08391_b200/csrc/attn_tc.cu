@@ -77,6 +77,7 @@ struct Params {
   bf16* out; int ldo;
   float scale_log2e;
   int* status;
+  int tiles;                            // query tiles per CTA: 2, or 1 when pairs would leave SMs idle
 };
 
 template <int HD>
@@ -124,7 +125,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   // key tiles each query tile needs (tile 1 may lie beyond the end of the sequence)
   int n_kv[2];
   n_kv[0] = (min(L, q0 + BQ) + BKV - 1) / BKV;
-  n_kv[1] = q0 + BQ < L ? (min(L, q0 + 2 * BQ) + BKV - 1) / BKV : 0;
+  n_kv[1] = (p.tiles == 2 && q0 + BQ < L) ? (min(L, q0 + 2 * BQ) + BKV - 1) / BKV : 0;
   const int n_max = max(n_kv[0], n_kv[1]);
 
 
@@ -325,11 +326,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 
 // Work list: pairs of query tiles of all sequences, those nearest the end of their sequence
 // (most key tiles) first.  One block, thread = sequence.
-__global__ void __launch_bounds__(256) attn_schedule_kernel(const int* __restrict__ cu, int batch, int2* __restrict__ sched) {
+__global__ void __launch_bounds__(256) attn_schedule_kernel(const int* __restrict__ cu, int batch, int tiles, int2* __restrict__ sched) {
   __shared__ int s_warp[8];
   __shared__ int s_base;
   const int b = threadIdx.x, warp = b >> 5, lane = b & 31;
-  const int np = b < batch ? (cu[b + 1] - cu[b] + 2 * BQ - 1) / (2 * BQ) : 0;
+  const int span = tiles * BQ;            // queries per work item
+  const int np = b < batch ? (cu[b + 1] - cu[b] + span - 1) / span : 0;
   int max_np = np;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) max_np = max(max_np, __shfl_xor_sync(0xffffffffu, max_np, o));
@@ -346,7 +348,7 @@ __global__ void __launch_bounds__(256) attn_schedule_kernel(const int* __restric
     __syncthreads();
     int pos = s_base + __popc(bal & ((1u << lane) - 1u));
     for (int w = 0; w < warp; ++w) pos += s_warp[w];
-    if (has) sched[pos] = make_int2(b, (np - 1 - r) * 2 * BQ);
+    if (has) sched[pos] = make_int2(b, (np - 1 - r) * span);
     __syncthreads();
     if (b == 0) { int t = 0; for (int w = 0; w < 8; ++w) t += s_warp[w]; s_base += t; }
     __syncthreads();
@@ -369,24 +371,24 @@ bool attn_tc_supported(int hd, int ld, const void* qkv, int ldo, const void* out
   return (hd == 64 || hd == 128) && ld % 8 == 0 && ((uintptr_t)qkv & 15) == 0 && ldo % 8 == 0 && ((uintptr_t)out & 15) == 0;
 }
 
-int attn_tc_items(const int* cu_host, int batch) {
+int attn_tc_items(const int* cu_host, int batch, int tiles) {
   int n = 0;
-  for (int b = 0; b < batch; ++b) n += (cu_host[b + 1] - cu_host[b] + 2 * BQ - 1) / (2 * BQ);
+  for (int b = 0; b < batch; ++b) n += (cu_host[b + 1] - cu_host[b] + tiles * BQ - 1) / (tiles * BQ);
   return n;
 }
 
-void launch_attn_schedule(const int* cu_dev, int batch, int2* sched, cudaStream_t st, int64_t* n_launch) {
+void launch_attn_schedule(const int* cu_dev, int batch, int tiles, int2* sched, cudaStream_t st, int64_t* n_launch) {
   ++*n_launch;
-  attn_schedule_kernel<<<1, 256, 0, st>>>(cu_dev, batch, sched);
+  attn_schedule_kernel<<<1, 256, 0, st>>>(cu_dev, batch, tiles, sched);
 }
 
 cudaError_t launch_attn_tc(const bf16* qkv, int ld, int total, int nq, int nkv, int hd, const int* cu_dev, const int2* sched,
-                           int n_items, bf16* out, int ldo, int* status, cudaStream_t st, int64_t* n_launch) {
+                           int n_items, int tiles, bf16* out, int ldo, int* status, cudaStream_t st, int64_t* n_launch) {
   CUtensorMap mq, mkv;
   const int bkv = hd == 64 ? 128 : 64;
   if (!tc_make_map_bf16(&mq, qkv, total, (long long)(nq + 2 * nkv) * hd, ld, BQ)) return cudaErrorInvalidValue;
   if (!tc_make_map_bf16(&mkv, qkv, total, (long long)(nq + 2 * nkv) * hd, ld, bkv)) return cudaErrorInvalidValue;
-  Params p{cu_dev, sched, nq, nkv, out, ldo, (1.f / sqrtf((float)hd)) * 1.4426950408889634f, status};
+  Params p{cu_dev, sched, nq, nkv, out, ldo, (1.f / sqrtf((float)hd)) * 1.4426950408889634f, status, tiles};
   dim3 grid(nq, n_items);
   ++*n_launch;
   return hd == 64 ? go<64>(mq, mkv, p, grid, st) : go<128>(mq, mkv, p, grid, st);

@@ -137,7 +137,7 @@ WsLayout ws_layout(const kvp_handle* h, int64_t Bm, int64_t Tm) {
   const int64_t k_max = std::max((int64_t)B.d, std::max((int64_t)B.max_dq, (int64_t)B.max_ffn));
   w.xbt = take(2 * Bp * k_max * 2);
   w.gub = take(Bm * 2 * (size_t)B.max_ffn * 4);
-  w.attn_sched = take((size_t)(Tm / 256 + Bm + 1) * 8);
+  w.attn_sched = take((size_t)(Tm / 128 + Bm + 1) * 8);
   w.total = off;
   return w;
 }
@@ -550,10 +550,15 @@ static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int
   KVP_TIMED(KVP_CLASS_OTHER, launch_build_index(ctx, cs.cu.data(), batch, T, cu_dev, tok_pos, tok_slot, last_idx, cache->block_table,
                      cache->max_pages_per_seq, cache->n_pages, cache->seq_lens));
   int2* attn_sched = (int2*)(ws + w.attn_sched);
-  const int attn_items = attn_tc_items(cs.cu.data(), batch);
+  // two query tiles per CTA share their K/V tiles; with so few tokens that even the widest layer's pairs
+  // would leave SMs idle, one tile per CTA finishes sooner
+  int max_nq = 1;
+  for (int j = 0; j <= h->j_max; ++j) max_nq = std::max(max_nq, A.L[j].nq);
+  const int attn_tiles = attn_tc_items(cs.cu.data(), batch, 2) * max_nq < h->n_sm ? 1 : 2;
+  const int attn_items = attn_tc_items(cs.cu.data(), batch, attn_tiles);
   if (h->use_tc && h->opt.dtype == KVP_BF16 && (A.L[0].hd == 64 || A.L[0].hd == 128)) {
     KVP_TIMED(KVP_CLASS_OTHER, launch_rope_table(ctx, rope_tab, cs.max_len, A.L[0].hd, A.theta));
-    KVP_TIMED(KVP_CLASS_OTHER, launch_attn_schedule(cu_dev, batch, attn_sched, ctx.st, ctx.n_launch));
+    KVP_TIMED(KVP_CLASS_OTHER, launch_attn_schedule(cu_dev, batch, attn_tiles, attn_sched, ctx.st, ctx.n_launch));
   }
   // ---- stage 1 + 2: auxiliary prefill, each layer's K/V pushed through the predictor ----
   // (only worth it while a layer's kernels leave SMs idle: with many tokens every kernel fills the GPU by itself)
@@ -626,7 +631,7 @@ static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int
     if (last) break;
     if (h->use_tc && split && attn_items <= 65535 && attn_tc_supported(L.hd, L.nqkv, qkv, L.dq, attn)) {
       TimedScope ts(h, ctx.st, KVP_CLASS_AUX_ATTN);
-      cudaError_t e = launch_attn_tc((const bf16*)qkv, L.nqkv, T, L.nq, L.nkv, L.hd, cu_dev, attn_sched, attn_items, (bf16*)attn,
+      cudaError_t e = launch_attn_tc((const bf16*)qkv, L.nqkv, T, L.nq, L.nkv, L.hd, cu_dev, attn_sched, attn_items, attn_tiles, (bf16*)attn,
                                      L.dq, ctx.status, ctx.st, ctx.n_launch);
       if (e != cudaSuccess && tc_err == cudaSuccess) tc_err = e;
     } else {
