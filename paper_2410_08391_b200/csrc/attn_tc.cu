@@ -173,36 +173,50 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         tc_fence_after();
         for (int g = 0; g < 2; ++g) if (n_kv[g] > 0) issue_s(g, 0);
       }
-      for (int j = 0; j < n_max && ok; ++j) {
-        const int stage = j % STAGES;
-        if (j + 1 < n_max) {
-          const int s1 = (j + 1) % STAGES;
-          ok = mbar_wait(kv_full(s1), ((j + 1) / STAGES) & 1, abort_flag, p.status);
-          if (!ok) break;
-          tc_fence_after();
-          for (int g = 0; g < 2 && ok; ++g)
-            if (j + 1 < n_kv[g]) {
-              ok = mbar_wait(s_free(g), j & 1, abort_flag, p.status);      // S(j) of this tile is in registers
-              if (!ok) break;
-              tc_fence_after();
-              issue_s(g, s1);
-            }
-          if (!ok) break;
-        }
-        const uint32_t sv = sKV + stage * 2 * KB + KB;
-        for (int g = 0; g < 2 && ok; ++g)
-          if (j < n_kv[g]) {
-            ok = mbar_wait(p_ready(g), j & 1, abort_flag, p.status);
-            if (!ok) break;
+      // Event loop: whichever of the two groups has something ready gets it issued, so a group never
+      // waits behind the other one's softmax.  js = next S tile, jp = next P V product of a group.
+      int js[2] = {1, 1}, jp[2] = {0, 0};
+      int released = 0;                 // key tiles whose stage has been handed back to the loader
+      uint32_t idle = 0;
+      while (ok && (jp[0] < n_kv[0] || jp[1] < n_kv[1])) {
+        bool progress = false;
+#pragma unroll
+        for (int g = 0; g < 2; ++g) {
+          if (jp[g] < n_kv[g] && mbar_test(p_ready(g), jp[g] & 1)) {
             tc_fence_after();
+            const uint32_t sv = sKV + (jp[g] % STAGES) * 2 * KB + KB;
 #pragma unroll
             for (int kk = 0; kk < BKV / 16; ++kk)
               tc_mma_bf16(tmem_base + 256 + g * 128, desc_kmajor(sP + g * PB + (kk >> 2) * 16384 + (kk & 3) * 32),
-                          desc_mnmajor(sv + kk * 2048, KV_BOX), idesc_pv, (j > 0 || kk > 0) ? 1u : 0u);
+                          desc_mnmajor(sv + kk * 2048, KV_BOX), idesc_pv, (jp[g] > 0 || kk > 0) ? 1u : 0u);
             tc_commit(pv_done(g));
+            ++jp[g];
+            progress = true;
           }
-        if (!ok) break;
-        tc_commit(kv_empty(stage));
+          // S of the next key tile: its K tile has landed and the group holds the previous S in registers
+          if (js[g] < n_kv[g] && mbar_test(s_free(g), (js[g] - 1) & 1) && mbar_test(kv_full(js[g] % STAGES), (js[g] / STAGES) & 1)) {
+            tc_fence_after();
+            issue_s(g, js[g] % STAGES);
+            ++js[g];
+            progress = true;
+          }
+        }
+        // a stage goes back to the loader once every group that uses its tile has issued S and P V on it
+        while (released < n_max && (n_kv[0] <= released || jp[0] > released) && (n_kv[1] <= released || jp[1] > released)) {
+          tc_commit(kv_empty(released % STAGES));
+          ++released;
+          progress = true;
+        }
+        if (progress) {
+          idle = 0;
+        } else if (++idle > SPIN_LIMIT) {
+          *abort_flag = 1;
+          dev_flag(p.status, DEV_TIMEOUT);
+          ok = false;
+        } else if ((idle & 63u) == 63u) {
+          if (*abort_flag) ok = false;
+          __nanosleep(32);
+        }
       }
       if (!ok) drain_after_abort();
     }
