@@ -200,9 +200,10 @@ bool try_tc(kvp_handle* h, const LaunchCtx& ctx, TcGemm& t, int cls, cudaError_t
   return true;
 }
 
-// Are the step's projections run on the tensor cores (batches the CUDA-core kernels are too slow for)?
+// Are the step's projections run on the tensor cores?  (Everything the persistent kernel does not take:
+// batches of more than 4 rows, and small batches over long caches.)
 bool step_uses_tc(const kvp_handle* h, int batch) {
-  if (!h->use_tc || h->opt.dtype != KVP_BF16 || batch <= 4 || step_tc_rows(batch) > 128) return false;
+  if (!h->use_tc || h->opt.dtype != KVP_BF16 || step_tc_rows(batch) > 128) return false;
   const ModelPlan& B = h->base;
   if (B.d % 8) return false;
   for (int i = 0; i < B.n_layers; ++i)
@@ -266,6 +267,9 @@ bool base_step_fused(kvp_handle* h, const LaunchCtx& ctx, const kvp_cache* cache
                      int32_t* token_out, cudaError_t* err) {
   const ModelPlan& B = h->base;
   int k_max = std::max(B.d, std::max(B.max_dq, B.max_ffn));
+  // its attention phase reads cache pages with plain loads: fine for a few thousand keys, several times
+  // slower than the ring-fed kernel beyond that
+  if (max_keys > 4096) return false;
   if (!h->use_mega || B.n_layers > MEGA_MAX_LAYERS || !step_mega_supported(batch, B.L[0].hd, k_max, B.max_group, h->es)) return false;
   // bulk copies need 16-byte rows: every projection's row length must be a multiple of 16 bytes
   for (int i = 0; i < B.n_layers; ++i)

@@ -32,6 +32,10 @@ CASES = [
     # more than 4 sequences: the step's projections run on the tensor cores (operand rows padded to 16, 24)
     ("t_hd128", [40, 9, 130, 17, 64, 65, 3, 90, 128], "fanin"),
     ("t_scaled", [20, 33, 5, 64, 65, 1, 40, 41, 42, 43, 44, 45, 46, 47, 48, 49, 50], "fanin"),
+    # a cache of more than 4096 entries with a small batch: the step leaves the persistent kernel for the
+    # tensor-core projections + ring-fed attention over 66 pages in several key-range splits
+    ("t_small", [4200, 70], "fanin"),
+    ("t_hd128", [4100], "n002"),
 ]
 
 
