@@ -106,6 +106,21 @@ def whole_job_value(tokens_per_rank: int, world: int, ms_per_step: float) -> flo
     return world * tokens_per_rank / (ms_per_step * 1e-3)
 
 
+def measured_traffic(workload: str, kernel_class: str):
+    """DRAM bytes per launch of a kernel class from the committed ncu capture, or None when there is no
+    capture for this workload / class or the kernel's source has changed since it was taken."""
+    import hashlib
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    if not os.path.exists(path):
+        return None
+    for rec in json.load(open(path)):
+        if rec["workload"] == workload and rec["kernel_class"] == kernel_class:
+            src = os.path.join(ROOT, rec["source"])
+            if os.path.exists(src) and hashlib.sha256(open(src, "rb").read()).hexdigest() == rec["source_sha256"]:
+                return rec["dram_bytes_per_launch"]
+    return None
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -244,7 +259,8 @@ def main():
     else:
         peak, achieved, unit = peaks["hbm_gbs"], amount / t_dom / 1e9, "GB/s"
     roofline = {"kernel_class": dom, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit,
-                "frac": achieved / peak, "traffic": None, "peak_source": peaks["source"],
+                "frac": achieved / peak, "traffic": measured_traffic(args.workload, dom),
+                "algorithmic_per_launch": amount / max(per_step[dom][1], 1), "peak_source": peaks["source"],
                 "launches_per_step": per_step[dom][1], "avg_launch_ms": per_step[dom][0] / max(per_step[dom][1], 1),
                 "class_ms_per_step": {c: round(v[0], 4) for c, v in per_step.items()},
                 "timing": "separate pass with CUDA events around every launch"}

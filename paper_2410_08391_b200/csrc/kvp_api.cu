@@ -138,6 +138,7 @@ WsLayout ws_layout(const kvp_handle* h, int64_t Bm, int64_t Tm) {
   w.xbt = take(2 * Bp * k_max * 2);
   w.gub = take(Bm * 2 * (size_t)B.max_ffn * 4);
   w.attn_sched = take((size_t)(Tm / 128 + Bm + 1) * 8);
+  w.attn_done = take((size_t)Bm * B.max_nkv * 4);
   w.total = off;
   return w;
 }
@@ -284,6 +285,8 @@ bool base_step_fused(kvp_handle* h, const LaunchCtx& ctx, const kvp_cache* cache
   p.block_table = cache->block_table; p.mpps = cache->max_pages_per_seq; p.n_pages = cache->n_pages; p.seq_lens = cache->seq_lens;
   p.xb = (float*)(ws + w.xb); p.qkvb = (float*)(ws + w.qkvb); p.ab = (float*)(ws + w.ab); p.actb = (float*)(ws + w.actb);
   p.part = (float*)(ws + w.part);
+  p.attn_done = (int*)(ws + w.attn_done);
+  cudaMemsetAsync(p.attn_done, 0, (size_t)batch * B.max_nkv * 4, ctx.st);
   p.logits = logits; p.token_out = token_out; p.status = ctx.status;
   p.trace = getenv("KVP_MEGA_TRACE") ? (long long*)((char*)ctx.status + 256) : nullptr;
   int min_nkv = B.L[0].nkv;

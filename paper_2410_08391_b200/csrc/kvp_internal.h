@@ -44,7 +44,7 @@ struct PackSlot {
 
 struct WsLayout {
   size_t status, cu, last_idx, tok_pos, tok_slot, rope_tab, x, h, h_lo, qkv, qkv32, kv_lo, attn, gu, act;
-  size_t xb, hb, qkvb, ab, actb, part, tok_stage, first_stage, xbt, gub, attn_sched, total;
+  size_t xb, hb, qkvb, ab, actb, part, tok_stage, first_stage, xbt, gub, attn_sched, attn_done, total;
 };
 
 struct kvp_handle {

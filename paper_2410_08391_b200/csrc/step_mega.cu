@@ -5,7 +5,7 @@
 // from HBM.  Here one CTA of 16 warps per SM stays resident for the whole step.  The operations
 // become phases separated by a grid-wide barrier (one global counter, bounded spin):
 //   per layer:  q(kv) projection (RMSNorm fused) | [append k,v] | attention over cache pages |
-//               [merge of key-range splits] | O projection + residual | gate/up + SwiGLU (RMSNorm
+//               (key-range splits merged by the CTA that finishes a group's last split) | O projection + residual | gate/up + SwiGLU (RMSNorm
 //               fused) | down projection + residual;   then LM head (final RMSNorm fused) + argmax.
 // Weights never pass through registers on their way from HBM: every warp owns a small ring of
 // shared-memory slots that it fills with bulk asynchronous copies (cp.async.bulk, completion on
@@ -445,6 +445,7 @@ __global__ void __launch_bounds__(NT, 1) step_mega_kernel(const __grid_constant_
   extern __shared__ __align__(128) unsigned char sm_raw[];
   __shared__ float red[NW * BB];
   __shared__ int s_flag;
+  __shared__ int s_last;
   __shared__ int s_abort_mem;
   __shared__ __align__(8) unsigned long long s_bars[NW * NSLOT];
   volatile int* s_abort = &s_abort_mem;
@@ -523,43 +524,56 @@ __global__ void __launch_bounds__(NT, 1) step_mega_kernel(const __grid_constant_
       }
       BARRIER();
     }
-    // ---- attention over the cache
+    // ---- attention over the cache.  With split key ranges the CTA that finishes the last split of a
+    // (sequence, kv head) merges that group's partial results on the spot (a counter per group tells
+    // it so), which saves a separate merge phase and its grid barrier.
     {
       const int n_items = batch * L.nkv * p.n_split;
+      const int group = L.nq / L.nkv, ldr = p.hd + 2;
       for (int it = blockIdx.x; it < n_items; it += gridDim.x) {
-        int sp = it % p.n_split, r = it / p.n_split;
+        const int sp = it % p.n_split, r = it / p.n_split;
         attn_item<T>(p, L, r / L.nkv, r % L.nkv, sp, p.n_split, p.qkvb, n_out, sm_raw, p.part, p.ab);
+        if (p.n_split > 1) {
+          __threadfence();                       // this CTA's partial results are visible before it counts itself done
+          __syncthreads();
+          if (tid == 0) {
+            const int before = atomicAdd(p.attn_done + r, 1);
+            s_last = before == p.n_split - 1;
+            if (s_last) atomicExch(p.attn_done + r, 0);      // ready for the next layer
+          }
+          __syncthreads();
+          if (s_last) {
+            __threadfence();
+            if (warp < group) {                  // one warp per q head of the group
+              const int head = (r / L.nkv) * L.nq + (r % L.nkv) * group + warp;
+              const float* pr = p.part + (size_t)head * p.n_split * ldr;
+              float mm = -INFINITY;
+              for (int s = lane; s < p.n_split; s += 32) mm = fmaxf(mm, __ldcg(pr + (size_t)s * ldr + p.hd));
+              mm = warp_max(mm);
+              // the loads of different splits do not depend on one another: unrolled, they are in flight together
+              float ll = 0.f, o0 = 0.f, o1 = 0.f, o2 = 0.f, o3 = 0.f;
+#pragma unroll 8
+              for (int s = 0; s < p.n_split; ++s) {
+                const float* rr = pr + (size_t)s * ldr;
+                const float ms = __ldcg(rr + p.hd);
+                const float f = (ms == -INFINITY) ? 0.f : __expf(ms - mm);
+                ll = fmaf(__ldcg(rr + p.hd + 1), f, ll);
+                if (lane < p.hd) o0 = fmaf(__ldcg(rr + lane), f, o0);
+                if (lane + 32 < p.hd) o1 = fmaf(__ldcg(rr + lane + 32), f, o1);
+                if (lane + 64 < p.hd) o2 = fmaf(__ldcg(rr + lane + 64), f, o2);
+                if (lane + 96 < p.hd) o3 = fmaf(__ldcg(rr + lane + 96), f, o3);
+              }
+              float* dst = p.ab + (size_t)head * p.hd;
+              if (lane < p.hd) dst[lane] = o0 / ll;
+              if (lane + 32 < p.hd) dst[lane + 32] = o1 / ll;
+              if (lane + 64 < p.hd) dst[lane + 64] = o2 / ll;
+              if (lane + 96 < p.hd) dst[lane + 96] = o3 / ll;
+            }
+          }
+        }
       }
     }
     BARRIER();
-    if (p.n_split > 1) {   // merge the key-range splits: one warp per (sequence, q head)
-      const int ldr = p.hd + 2;
-      for (int it = gw; it < batch * L.nq; it += GW) {
-        const float* pr = p.part + (size_t)it * p.n_split * ldr;
-        float mm = -INFINITY;
-        for (int s = lane; s < p.n_split; s += 32) mm = fmaxf(mm, __ldcg(pr + (size_t)s * ldr + p.hd));
-        mm = warp_max(mm);
-        // the loads of different splits do not depend on one another: unrolled, they are in flight together
-        float ll = 0.f, o0 = 0.f, o1 = 0.f, o2 = 0.f, o3 = 0.f;
-#pragma unroll 8
-        for (int s = 0; s < p.n_split; ++s) {
-          const float* r = pr + (size_t)s * ldr;
-          const float ms = __ldcg(r + p.hd);
-          const float f = (ms == -INFINITY) ? 0.f : __expf(ms - mm);
-          ll = fmaf(__ldcg(r + p.hd + 1), f, ll);
-          if (lane < p.hd) o0 = fmaf(__ldcg(r + lane), f, o0);
-          if (lane + 32 < p.hd) o1 = fmaf(__ldcg(r + lane + 32), f, o1);
-          if (lane + 64 < p.hd) o2 = fmaf(__ldcg(r + lane + 64), f, o2);
-          if (lane + 96 < p.hd) o3 = fmaf(__ldcg(r + lane + 96), f, o3);
-        }
-        float* dst = p.ab + (size_t)it * p.hd;
-        if (lane < p.hd) dst[lane] = o0 / ll;
-        if (lane + 32 < p.hd) dst[lane + 32] = o1 / ll;
-        if (lane + 64 < p.hd) dst[lane + 64] = o2 / ll;
-        if (lane + 96 < p.hd) dst[lane + 96] = o3 / ll;
-      }
-      BARRIER();
-    }
     // ---- O projection + residual
     stage_x<BB>(p.ab, L.dq, L.dq, batch, nullptr, 0.f, xs, red);
     gemv_phase<T, BB>(p, stream_desc(p, 4 * i + 1), ws, ring_ptr, xs, p.xb, p.d, gw, GW, lane, nullptr, s_abort);

@@ -20,6 +20,7 @@ struct MegaParams {
   const int* block_table; int mpps, n_pages;
   int* seq_lens;
   float *xb, *qkvb, *ab, *actb, *part;           // workspace: residual, projections, attention out, FFN act, partials
+  int* attn_done;                                // [batch * max n_kv] splits finished per (sequence, kv head); zero on entry, left zero
   float* logits; int* token_out;
   int stage_bytes, slot_bytes;                   // shared-memory plan (set by the launcher)
   long long* trace;                              // optional: clock64 of CTA 0 around every barrier (debugging aid)
