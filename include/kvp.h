@@ -17,7 +17,8 @@
  *     kvp_create() ran; "host" pointers are ordinary host memory.
  *   - The caller owns ALL device memory (weights, packed weights, workspace, cache
  *     pools, block table, outputs).  The handle borrows the packed-weight pointer
- *     until kvp_destroy(); it owns only host metadata and TMA descriptors.
+ *     until kvp_destroy(); it owns host metadata, the CUDA graphs it records, and one
+ *     internal stream with two events (created by kvp_create on the current device).
  *   - Calls that take a stream only enqueue work on it and return without
  *     synchronising (except the *_host variant, which synchronises the stream);
  *     arguments are validated on the host before anything is launched.
@@ -27,6 +28,9 @@
  *     word is cleared by kvp_prefill_predict() at its start and by kvp_poll_status();
  *     poll once on a fresh workspace before using it for kvp_decode_step() alone.
  *   - Matrices are [out_features, in_features], row-major, dense.
+ *   - Reproducibility: some projections add partial sums with fp32 atomic adds, so two runs
+ *     on the same inputs agree up to fp32 reassociation (about 1e-6 relative in the fp32
+ *     quantities, occasionally one bf16 unit in a stored cache element), not bit for bit.
  */
 #ifndef KVP_H_
 #define KVP_H_
@@ -171,7 +175,10 @@ kvp_status kvp_load_weights(kvp_handle* h, const kvp_tensor* tensors, int32_t n,
  * The first call with a given set of arguments (pointers, lengths, stream) records the kernel
  * schedule into a CUDA graph owned by the handle; later calls with the same arguments replay it
  * (the token values themselves may change between calls).  If `stream` is already being
- * captured by the caller, the kernels are enqueued into the caller's capture instead. */
+ * captured by the caller, the kernels are enqueued into the caller's capture instead.
+ * For short prompts part of the work (the predictor) is enqueued on the handle's internal
+ * stream, forked from and joined back into `stream` with events; from the caller's point of
+ * view everything is ordered on `stream` as usual. */
 kvp_status kvp_prefill_predict(kvp_handle* h, const int32_t* tokens, const int32_t* lengths,
                                int32_t batch, const kvp_cache* cache, void* workspace,
                                size_t workspace_bytes, float* logits_out, int32_t* first_token,
