@@ -36,6 +36,9 @@ CASES = [
     # tensor-core projections + ring-fed attention over 66 pages in several key-range splits
     ("t_small", [4200, 70], "fanin"),
     ("t_hd128", [4100], "n002"),
+    # more sequences than the tensor-core step path takes (128): the CUDA-core projections serve the step;
+    # many one- and two-token prompts
+    ("t_small", [1, 2, 3, 5, 8, 13, 21, 34, 55, 89] * 13, "fanin"),
 ]
 
 
