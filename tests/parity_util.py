@@ -22,7 +22,7 @@ def make_session(pair, W, prompts, extra_len=0):
                        max_len=int(prompts.lengths.max()), extra_len=extra_len)
 
 
-def compare_prefill(sess, pair, W, prompts, seqs=None):
+def compare_prefill(sess, pair, W, prompts, seqs=None, gap=GAP):
     """Runs kvp_prefill_predict on the whole batch; compares the listed sequences with the oracle.
     Returns (worst K error, worst V error, worst logits error, n argmax compared)."""
     import torch
@@ -47,7 +47,7 @@ def compare_prefill(sess, pair, W, prompts, seqs=None):
         assert e3 <= tol, f"seq {b}: logits err {e3:.3e} > {tol}"
         el = max(el, e3)
         assert int(first[b]) == int(np.argmax(logits[b])), "first token is not the argmax of the returned logits"
-        if orc.top2_gap(ref_logits) > GAP:
+        if orc.top2_gap(ref_logits) > gap:
             assert int(first[b]) == ref_tok, f"seq {b}: first token {first[b]} != oracle {ref_tok}"
             n_arg += 1
     return ek, ev, el, n_arg
