@@ -182,7 +182,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         bool progress = false;
 #pragma unroll
         for (int g = 0; g < 2; ++g) {
-          if (jp[g] < n_kv[g] && mbar_test(p_ready(g), jp[g] & 1)) {
+          if (jp[g] < n_kv[g] && mbar_poll(p_ready(g), jp[g] & 1)) {
             tc_fence_after();
             const uint32_t sv = sKV + (jp[g] % STAGES) * 2 * KB + KB;
 #pragma unroll
@@ -194,7 +194,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             progress = true;
           }
           // S of the next key tile: its K tile has landed and the group holds the previous S in registers
-          if (js[g] < n_kv[g] && mbar_test(s_free(g), (js[g] - 1) & 1) && mbar_test(kv_full(js[g] % STAGES), (js[g] / STAGES) & 1)) {
+          if (js[g] < n_kv[g] && mbar_poll(s_free(g), (js[g] - 1) & 1) && mbar_poll(kv_full(js[g] % STAGES), (js[g] / STAGES) & 1)) {
             tc_fence_after();
             issue_s(g, js[g] % STAGES);
             ++js[g];
@@ -215,7 +215,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           ok = false;
         } else if ((idle & 63u) == 63u) {
           if (*abort_flag) ok = false;
-          __nanosleep(32);
         }
       }
       if (!ok) drain_after_abort();
