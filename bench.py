@@ -150,9 +150,10 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="c2", choices=["c1", "c2", "c3", "c4", "c5"])
+    ap.add_argument("--workload", default="c2", choices=["c1", "c2", "c3", "c4", "c5", "qa", "lp75", "lp50", "lp25"])
     ap.add_argument("--impl", default="kvp", choices=["kvp", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--decode-steps", type=int, default=16, help="generation steps timed after the TTFT measurement (0 = none)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "kvp" else args.warmup
     if args.impl == "reference":
@@ -179,7 +180,8 @@ def main():
     pr = wl.prompts(args.workload, seed=0)
     lens = [int(x) for x in pr.lengths]
     work = wl.algorithmic_work(pair, lens)
-    sess = kvp.Session(pair, W, max_batch=pr.batch, max_total_tokens=pr.total, max_len=max(lens), device=dev)
+    sess = kvp.Session(pair, W, max_batch=pr.batch, max_total_tokens=pr.total, max_len=max(lens), device=dev,
+                       extra_len=max(args.decode_steps, 0) + 3)
     toks = torch.from_numpy(pr.tokens).to(dev)
 
     def barrier():
@@ -232,6 +234,30 @@ def main():
     e2e_ms = (time.perf_counter() - w0) * 1e3 / args.steps
     e2e_ms = max_over_ranks(e2e_ms, dist, dev)
     e2e_value = whole_job_value(work["tokens"], world, e2e_ms)
+
+    # ---- generation loop after the first token (Fig. 2(b), loop body): secondary figure ----
+    decode = None
+    if args.decode_steps > 0:
+        step()                                  # a fresh predicted cache and first tokens
+        cur = list(lens)
+        tok = sess.first[:pr.batch].clone()
+        for _ in range(3):                      # warm-up steps (they extend the cache too)
+            _, nxt = sess.decode_step(tok, cur)
+            tok = nxt.clone()
+            cur = [c + 1 for c in cur]
+        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        d0.record(stream)
+        for _ in range(args.decode_steps):
+            _, nxt = sess.decode_step(tok, cur)
+            tok.copy_(nxt)
+            cur = [c + 1 for c in cur]
+        d1.record(stream)
+        torch.cuda.synchronize()
+        sess.poll()
+        dms = max_over_ranks(d0.elapsed_time(d1) / args.decode_steps, dist, dev)
+        decode = {"steps": args.decode_steps, "ms_per_step": dms, "tok_per_s": world * pr.batch / (dms * 1e-3),
+                  "ttft_over_step": ms_step / dms}
 
     # ---- per-kernel-class device times (separate pass: events around every launch) ----
     kvp.kvp_timing_enable(sess.h, True)
@@ -289,6 +315,7 @@ def main():
                 "d2h_bytes_per_step": int(pr.batch * pair.base.vocab * 4 + pr.batch * 4)},
         "roofline": roofline,
         "tensor_frac_stage12": tensor_frac,
+        "decode": decode,
         "clocks": clocks,
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

@@ -2,6 +2,8 @@
 paper or the mathematics fixes, never against the oracle itself or the CUDA path."""
 import math
 
+import os
+
 import numpy as np
 import pytest
 
@@ -337,3 +339,17 @@ def test_config_1_runs_in_seconds_and_is_finite():
     kv_hat, logits, tok = res[0]
     assert len(kv_hat) == 4 and kv_hat[0][0].shape == (64, 64) and logits.shape == (512,)
     assert np.isfinite(logits).all() and 0 <= tok < 512
+
+
+def test_layer_pruned_workload_pairs_use_the_maps_of_table_1():
+    """The KVP-LP pairs of the workload module carry the printed j_i rows (Table 1) and as many auxiliary
+    layers as Table 4 (Appendix A) retains."""
+    rows = {}
+    for line in open(os.path.join(os.path.dirname(__file__), "golden", "layer_maps.txt")):
+        if line.startswith("LP | OE1.1B"):
+            f = [x.strip() for x in line.split("|")]
+            rows[f[1]] = (int(f[3]), tuple(int(x) for x in f[5].split()))
+    for name, key in (("lp75", "OE1.1B-KVP-LP-0.75"), ("lp50", "OE1.1B-KVP-LP-0.50"), ("lp25", "OE1.1B-KVP-LP-0.25")):
+        p = wl.pair(name)
+        assert p.aux.n_layers == rows[key][0] and p.layer_map == rows[key][1]
+        assert p.aux.d_model == p.base.d_model and p.aux.layers[0] == p.base.layers[0]

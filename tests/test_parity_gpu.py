@@ -29,6 +29,9 @@ CASES = [
     ("t_scaled", [100, 33, 257], "fanin"),
     ("t_scaled", [100, 33, 257], "n002"),
     ("t_bias", [40, 90], "fanin"),
+    # layer-pruned auxiliary model (KVP-LP): same width as the base, square predictor matrices
+    ("t_lp", [100, 59, 59, 7], "fanin"),
+    ("t_lp", [130], "n002"),
     # more than 4 sequences: the step's projections run on the tensor cores (operand rows padded to 16, 24)
     ("t_hd128", [40, 9, 130, 17, 64, 65, 3, 90, 128], "fanin"),
     ("t_scaled", [20, 33, 5, 64, 65, 1, 40, 41, 42, 43, 44, 45, 46, 47, 48, 49, 50], "fanin"),

@@ -100,6 +100,16 @@ _MAP_28_FROM_16 = (0, 0, 1, 1, 2, 2, 3, 3, 4, 4, 5, 5, 6, 6, 7, 7, 8, 8, 9, 9,
                    10, 10, 11, 11, 12, 13, 14, 15)
 
 
+# Table 1 of the paper, rows OE1.1B-KVP-LP-0.75 / 0.50 / 0.25, typed in as data: the auxiliary model
+# is the base model with only 21 / 14 / 7 of its 28 layers retained (Appendix A, Table 4), so both
+# models have the same width and the predictor matrices are square.
+_MAP_LP = {
+    "lp75": (0, 1, 2, 2, 3, 4, 5, 5, 6, 7, 8, 8, 9, 10, 11, 11, 12, 13, 14, 14, 15, 16, 17, 17, 18, 19, 20, 20),
+    "lp50": (0, 0, 1, 1, 2, 2, 3, 3, 4, 4, 5, 5, 6, 6, 7, 7, 8, 8, 9, 9, 10, 10, 11, 11, 12, 12, 13, 13),
+    "lp25": (0, 0, 0, 0, 1, 1, 1, 1, 2, 2, 2, 2, 3, 3, 3, 3, 4, 4, 4, 4, 5, 5, 5, 5, 6, 6, 6, 6),
+}
+
+
 def pair(name: str) -> PairCfg:
     """The five configurations of the benchmark plan plus small test pairs."""
     if name == "c1":      # tiny fp32 pair
@@ -121,7 +131,19 @@ def pair(name: str) -> PairCfg:
         aux = layerwise_scaled_model(16, 1280, 8, 20, 64, 32000)
         base = layerwise_scaled_model(28, 2048, 12, 32, 64, 32000)
         return PairCfg("c4", aux, base, _MAP_28_FROM_16)
+    if name == "qa":      # the c2 pair on the paper-shaped prompt batch (Sec. 6: 64 prompts of the average 1-shot length)
+        p = pair("c2")
+        return PairCfg("qa", p.aux, p.base, p.layer_map)
+    if name in _MAP_LP:   # KVP-LP: auxiliary = the 1.1B-shaped base with layers pruned (Sec. 4.2, Appendix A)
+        m = _MAP_LP[name]
+        base = uniform_model(28, 2048, 32, 8, 64, 5632, 32000)
+        aux = uniform_model(max(m) + 1, 2048, 32, 8, 64, 5632, 32000)
+        return PairCfg(name, aux, base, m)
     # ---- reduced pairs used by tests (several tiles, ragged tails, odd widths) ----
+    if name == "t_lp":        # layer-pruned pair scaled down: aux = every second layer of an 8-layer base
+        base = uniform_model(8, 256, 8, 2, 64, 448, 1000)
+        aux = uniform_model(4, 256, 8, 2, 64, 448, 1000)
+        return PairCfg("t_lp", aux, base, (0, 0, 1, 1, 2, 2, 3, 3))
     if name == "t_small":     # bf16, head_dim 64, GQA 4:1, non-multiple-of-128 widths
         aux = uniform_model(3, 192, 4, 1, 64, 320, 1000)
         base = uniform_model(5, 256, 8, 2, 64, 448, 1000)
@@ -309,6 +331,11 @@ def prompts(name: str, seed: int = 0) -> Prompts:
     if name == "c5":
         lens = np.full(4, 16384, np.int32)
         return Prompts(uniform_tokens(int(lens.sum()), v, seed), lens)
+    if name == "qa" or name in _MAP_LP:
+        # the shape of the paper's CPU timing (Sec. 6): batch 64, every prompt of the average TriviaQA
+        # 1-shot length, 59 tokens; synthetic Zipf token ids stand in for the dataset's prompts
+        lens = np.full(64, 59, np.int32)
+        return Prompts(zipf_tokens(int(lens.sum()), v, seed), lens)
     raise KeyError(name)
 
 
