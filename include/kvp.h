@@ -77,6 +77,9 @@ typedef struct {
   int32_t vocab;
   float rope_theta;
   float rms_eps;
+  int32_t qk_norm;             /* 1: queries and keys are RMS-normalised per head (over head_dim, eps = rms_eps,
+                                  gains "L{l}.q_norm" / "L{l}.k_norm" [head_dim]) before RoPE: OpenELM's key norm
+                                  (Sec. 7 "Analysis").  The cache then holds normalised, rotated keys. 0: off. */
   const kvp_layer_cfg* layers; /* host, [n_layers]; copied by kvp_create */
 } kvp_model_cfg;
 
@@ -93,6 +96,7 @@ typedef struct {
  *   "aux.L{j}.attn_norm" [d_A]   "aux.L{j}.ffn_norm" [d_A]
  *   "aux.L{j}.wq" [nq*hd, d_A]   "aux.L{j}.wk" / "wv" [nkv*hd, d_A]   "aux.L{j}.wo" [d_A, nq*hd]
  *   "aux.L{j}.w_gate" / "w_up" [ffn, d_A]   "aux.L{j}.w_down" [d_A, ffn]
+ *   with qk_norm: "aux.L{j}.q_norm" [hd] and "aux.L{j}.k_norm" [hd]
  *   the same under "base.", plus "base.final_norm" [d_B] and "base.lm_head" [vocab, d_B]
  *   "pred.L{i}.fk" / "fv" [d_kvB_i, d_kvA_{j_i}]  and, with predictor_bias, "pred.L{i}.bk" / "bv" [d_kvB_i]
  * Auxiliary layers above max_i j_i, "aux.final_norm" and "aux.lm_head" are never read

@@ -138,6 +138,19 @@ def _w(W: Dict[str, np.ndarray], name: str) -> np.ndarray:
     return W[name].astype(F64)
 
 
+def qk_norm(cfg, W, b: str, q, k):
+    """OpenELM normalises queries and keys (Sec. 7 "key norm"): an RMSNorm over head_dim of every
+    head, one gain vector per layer for q and one for k, applied before RoPE.  Off unless the
+    model asks for it; q may be None (a caller that only needs keys)."""
+    if not getattr(cfg, "qk_norm", False):
+        return q, k
+    if q is not None:
+        q = rmsnorm(q, W[b + "q_norm"], cfg.rms_eps)
+    if k is not None:
+        k = rmsnorm(k, W[b + "k_norm"], cfg.rms_eps)
+    return q, k
+
+
 # ----------------------------------------------------------------------------
 # a decoder over a whole prompt (used for A, and for B in the invariants)
 # ----------------------------------------------------------------------------
@@ -161,6 +174,7 @@ def decoder_prefill(cfg, W, prefix: str, tokens: np.ndarray, *, pos0: int = 0,
         q = (h @ _w(W, b + "wq").T).reshape(L, lc.n_q_heads, lc.head_dim)
         k = (h @ _w(W, b + "wk").T).reshape(L, lc.n_kv_heads, lc.head_dim)
         v = (h @ _w(W, b + "wv").T).reshape(L, lc.n_kv_heads, lc.head_dim)
+        q, k = qk_norm(cfg, W, b, q, k)
         q = rope(q, pos, cfg.rope_theta)
         k = rope(k, pos, cfg.rope_theta)
         kv.append((k.reshape(L, -1), v.reshape(L, -1)))
@@ -223,7 +237,9 @@ def base_first_step(pair, W, token: int, kv_hat):
     for i, lc in enumerate(cfg.layers):
         b = f"base.L{i}."
         h = rmsnorm(x, W[b + "attn_norm"], cfg.rms_eps)
-        q = rope((h @ _w(W, b + "wq").T).reshape(1, lc.n_q_heads, lc.head_dim), pos, cfg.rope_theta)
+        q = (h @ _w(W, b + "wq").T).reshape(1, lc.n_q_heads, lc.head_dim)
+        q, _ = qk_norm(cfg, W, b, q, None)
+        q = rope(q, pos, cfg.rope_theta)
         kh, vh = kv_hat[i]
         a = attention(q, kh.reshape(L, lc.n_kv_heads, lc.head_dim),
                       vh.reshape(L, lc.n_kv_heads, lc.head_dim), pos)
@@ -244,8 +260,11 @@ def decode_step(pair, W, token: int, cache):
     for i, lc in enumerate(cfg.layers):
         b = f"base.L{i}."
         h = rmsnorm(x, W[b + "attn_norm"], cfg.rms_eps)
-        q = rope((h @ _w(W, b + "wq").T).reshape(1, lc.n_q_heads, lc.head_dim), pos, cfg.rope_theta)
-        k = rope((h @ _w(W, b + "wk").T).reshape(1, lc.n_kv_heads, lc.head_dim), pos, cfg.rope_theta)
+        q = (h @ _w(W, b + "wq").T).reshape(1, lc.n_q_heads, lc.head_dim)
+        k = (h @ _w(W, b + "wk").T).reshape(1, lc.n_kv_heads, lc.head_dim)
+        q, k = qk_norm(cfg, W, b, q, k)
+        q = rope(q, pos, cfg.rope_theta)
+        k = rope(k, pos, cfg.rope_theta)
         v = h @ _w(W, b + "wv").T
         K = np.concatenate([cache[i][0], k.reshape(1, -1)], axis=0)
         V = np.concatenate([cache[i][1], v.reshape(1, -1)], axis=0)

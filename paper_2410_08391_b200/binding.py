@@ -31,7 +31,7 @@ class LayerCfgC(C.Structure):
 
 class ModelCfgC(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("d_model", C.c_int32), ("vocab", C.c_int32), ("rope_theta", C.c_float),
-                ("rms_eps", C.c_float), ("layers", C.POINTER(LayerCfgC))]
+                ("rms_eps", C.c_float), ("qk_norm", C.c_int32), ("layers", C.POINTER(LayerCfgC))]
 
 
 class OptionsC(C.Structure):
@@ -107,7 +107,7 @@ def _i32arr(v: Sequence[int]):
 
 def _model_c(m):
     layers = (LayerCfgC * m.n_layers)(*[LayerCfgC(l.n_q_heads, l.n_kv_heads, l.head_dim, l.ffn_dim) for l in m.layers])
-    return ModelCfgC(m.n_layers, m.d_model, m.vocab, m.rope_theta, m.rms_eps, layers), layers
+    return ModelCfgC(m.n_layers, m.d_model, m.vocab, m.rope_theta, m.rms_eps, 1 if getattr(m, "qk_norm", False) else 0, layers), layers
 
 
 # ---- functions with the C names -------------------------------------------------------------

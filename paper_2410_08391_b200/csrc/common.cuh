@@ -61,6 +61,19 @@ __device__ __forceinline__ void rope_sincos(int pos, double inv_freq, float* s, 
 }
 void fill_inv_freq(InvFreq* f, int hd, float theta);
 
+// Query / key norm: r[h] = 1 / sqrt(mean_c x[h * hd + c]^2 + eps) for h < n_heads (x in global memory,
+// read through L2).  One warp per head; every thread of the block must call it; ends with a block barrier.
+__device__ __forceinline__ void head_rnorm(const float* x, int n_heads, int hd, float eps, float* r_shared) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+  for (int h = warp; h < n_heads; h += nw) {
+    float ss = 0.f;
+    for (int c = lane; c < hd; c += 32) { const float v = __ldcg(x + (size_t)h * hd + c); ss = fmaf(v, v, ss); }
+    ss = warp_sum(ss);
+    if (lane == 0) r_shared[h] = rsqrtf(ss / (float)hd + eps);
+  }
+  __syncthreads();
+}
+
 // Where the predictor GEMM scatters its columns: the concatenated outputs of all base
 // layers fed by one auxiliary layer; segment s covers columns [col0[s], col0[s+1]).
 struct PagedOut {
@@ -124,9 +137,12 @@ void launch_rmsnorm(const LaunchCtx&, const float* x, const float* gain, float e
                     void* out, int out_dtype, void* out_lo = nullptr);
 // fp32 projection output [rows, n_heads*hd] -> RoPE on the first n_heads_rot heads -> run dtype
 // `out` (row stride ld_out) and, for heads >= lo_head_begin, the bf16 lo part in `out_lo`.
+// With q_gain / k_gain (fp32 [head_dim], or null): heads < n_q_heads are RMS-normalised with q_gain and the
+// other rotated heads with k_gain (eps) before RoPE.
 void launch_rope_split(const LaunchCtx&, const float* in, int ld_in, int rows, int n_heads, int n_heads_rot,
                        int head_dim, const int* tok_pos, float theta, void* out, int ld_out,
-                       void* out_lo, int ld_lo, int lo_head_begin);
+                       void* out_lo, int ld_lo, int lo_head_begin, int n_q_heads = 0, const float* q_gain = nullptr,
+                       const float* k_gain = nullptr, float eps = 0.f);
 void launch_swiglu(const LaunchCtx&, const void* gu, int rows, int ffn, int G, void* act);
 void launch_gemm_simt(const LaunchCtx&, const GemmArgs&, int epi);
 void launch_attn_prefill_simt(const LaunchCtx&, const void* qkv, int ld, int nq, int nkv, int hd,
@@ -140,10 +156,10 @@ void launch_step_gemv(const LaunchCtx&, const void* W, int ldw, int N, int K, co
 void launch_step_attn(const LaunchCtx&, const float* q, int ldq, int nq, int nkv, int hd, float theta,
                       const void* kpool, const void* vpool, const int* block_table,
                       int max_pages_per_seq, int n_pages, const int* seq_lens, int extra, int batch,
-                      int max_keys, float* part, float* out);
+                      int max_keys, float* part, float* out, const float* q_gain = nullptr, float eps = 0.f);
 void launch_step_append(const LaunchCtx&, const float* qkv, int nq, int nkv, int hd, float theta,
                         void* kpool, void* vpool, const int* block_table, int max_pages_per_seq,
-                        int n_pages, const int* seq_lens, int batch);
+                        int n_pages, const int* seq_lens, int batch, const float* k_gain = nullptr, float eps = 0.f);
 void launch_argmax(const LaunchCtx&, const float* logits, int batch, int vocab, int* out);
 void launch_add_int(const LaunchCtx&, int* v, int n, int delta);
 int step_attn_splits(int batch, int nkv, int max_keys);
@@ -151,4 +167,5 @@ int step_attn_splits(int batch, int nkv, int max_keys);
 bool step_attn_ring_supported(int dtype, int nq, int nkv, int hd, const void* kpool, const void* vpool);
 cudaError_t launch_step_attn_ring(const LaunchCtx&, const float* q, int ldq, int nq, int nkv, int hd, float theta,
                                   const void* kpool, const void* vpool, const int* block_table, int max_pages_per_seq,
-                                  int n_pages, const int* seq_lens, int extra, int batch, int n_split, float* part, float* out);
+                                  int n_pages, const int* seq_lens, int extra, int batch, int n_split, float* part, float* out,
+                                  const float* q_gain = nullptr, float eps = 0.f);

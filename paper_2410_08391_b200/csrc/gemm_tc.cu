@@ -154,6 +154,7 @@ struct Params {
   int rot_cols; int hd;
   const float2* rope_tab; const int* tok_pos;
   int ffn;               // SwiGLU: output width
+  const float* q_gain; const float* k_gain; int q_cols; float eps;   // TC_QKV: query / key norm (null = off)
   PagedOut paged;
 };
 
@@ -267,6 +268,21 @@ __device__ __forceinline__ void epilogue_tile(const Params& p, uint32_t tmem_acc
 #pragma unroll 1
     for (int h0 = 0; h0 < BN; h0 += p.hd) {
       if (n0 + h0 >= p.N) break;
+      // query / key norm: this thread's row of the head is scaled by 1 / rms and the head's gain before RoPE
+      const float* gain = (n0 + h0 < p.rot_cols) ? (n0 + h0 < p.q_cols ? p.q_gain : p.k_gain) : nullptr;
+      float rn = 1.f;
+      if (gain) {          // (uniform over the warp) first pass over the head's columns: mean square
+        float ss = 0.f;
+#pragma unroll 1
+        for (int j = 0; j < p.hd; j += 32) {
+          float a[32];
+          tmem_ld32(tmem_acc + h0 + j, a);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) ss = fmaf(a[i], a[i], ss);
+        }
+        rn = rsqrtf(ss / (float)p.hd + p.eps);
+      }
 #pragma unroll 1
       for (int j = 0; j < half; j += 32) {
         float a[32], b[32];
@@ -275,6 +291,10 @@ __device__ __forceinline__ void epilogue_tile(const Params& p, uint32_t tmem_acc
         tmem_ld_wait();
         int n = n0 + h0 + j;
         if (!row_ok) continue;
+        if (gain) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) { a[i] *= rn * gain[j + i]; b[i] *= rn * gain[half + j + i]; }
+        }
         if (n < p.rot_cols) {
 #pragma unroll
           for (int i = 0; i < 32; i += 2) {
@@ -531,6 +551,7 @@ cudaError_t launch_gemm_tc(const TcGemm& g, int* status, cudaStream_t st, int64_
   p.M = g.M; p.N = g.N; p.K = g.K; p.split_begin = g.split_begin; p.has_a2 = g.A2 != nullptr; p.status = status;
   p.stream_k = stream_k ? 1 : 0;
   p.C = g.C; p.ldc = g.ldc; p.X = g.X; p.ldx = g.ldx; p.C_lo = g.C_lo; p.ld_lo = g.ld_lo; p.lo_col_begin = g.lo_col_begin;
+  p.q_gain = g.q_gain; p.k_gain = g.k_gain; p.q_cols = g.q_cols; p.eps = g.eps;
   p.rot_cols = g.rot_cols; p.hd = g.hd; p.rope_tab = g.rope_tab; p.tok_pos = g.tok_pos; p.ffn = g.ffn; p.paged = g.paged;
   const int tiles = ((g.M + BM - 1) / BM) * ((g.N + bn - 1) / bn);
   const long long kblocks = (long long)tiles * ((g.K + BK - 1) / BK);

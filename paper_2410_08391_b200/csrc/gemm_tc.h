@@ -24,6 +24,9 @@ struct TcGemm {
   const float2* rope_tab;          // [position][hd/2] (cos, sin)
   const int* tok_pos;              // [M] position of each row in its sequence
   int ffn;
+  // TC_QKV with query / key norm: columns < q_cols are query heads (gain q_gain), the other rotated columns key
+  // heads (gain k_gain); null gains = no norm
+  const float* q_gain; const float* k_gain; int q_cols; float eps;
   PagedOut paged;
   int n_sm;
   int bn;                          // tile width: 128, 256, or 0 = chosen by the launcher

@@ -150,7 +150,8 @@ template <class T>
 __global__ void rope_split_kernel(const float* __restrict__ in, int ld_in, int rows, int n_heads, int n_heads_rot,
                                   int hd, const int* __restrict__ tok_pos, const __grid_constant__ InvFreq inv,
                                   T* __restrict__ out, int ld_out, T* __restrict__ out_lo, int ld_lo,
-                                  int lo_head_begin) {
+                                  int lo_head_begin, int n_q_heads, const float* __restrict__ q_gain,
+                                  const float* __restrict__ k_gain, float eps) {
   int half = hd >> 1;
   size_t n = (size_t)rows * n_heads * half;
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
@@ -161,6 +162,14 @@ __global__ void rope_split_kernel(const float* __restrict__ in, int ld_in, int r
     const float* p = in + (size_t)r * ld_in + (size_t)h * hd + c;
     float y1 = p[0], y2 = p[half];
     if (h < n_heads_rot) {
+      const float* gain = h < n_q_heads ? q_gain : k_gain;
+      if (gain) {   // query / key norm over the head (this generic path recomputes the head's mean square per element)
+        const float* hp = in + (size_t)r * ld_in + (size_t)h * hd;
+        float ss = 0.f;
+        for (int e = 0; e < hd; ++e) ss = fmaf(hp[e], hp[e], ss);
+        const float rn = rsqrtf(ss / (float)hd + eps);
+        y1 *= rn * gain[c]; y2 *= rn * gain[c + half];
+      }
       float sn, cs;
       rope_sincos(tok_pos[r], inv.f[c], &sn, &cs);
       float x1 = y1, x2 = y2;
@@ -180,7 +189,7 @@ __global__ void rope_split_kernel(const float* __restrict__ in, int ld_in, int r
 
 void launch_rope_split(const LaunchCtx& ctx, const float* in, int ld_in, int rows, int n_heads, int n_heads_rot, int hd,
                        const int* tok_pos, float theta, void* out, int ld_out, void* out_lo, int ld_lo,
-                       int lo_head_begin) {
+                       int lo_head_begin, int n_q_heads, const float* q_gain, const float* k_gain, float eps) {
   size_t n = (size_t)rows * n_heads * (hd / 2);
   if (n == 0) return;
   InvFreq inv;
@@ -188,9 +197,9 @@ void launch_rope_split(const LaunchCtx& ctx, const float* in, int ld_in, int row
   int grid = grid_for(n, 256);
   LAUNCH_COUNT(ctx);
   if (ctx.dtype == 0)
-    rope_split_kernel<float><<<grid, 256, 0, ctx.st>>>(in, ld_in, rows, n_heads, n_heads_rot, hd, tok_pos, inv, (float*)out, ld_out, (float*)nullptr, 0, 0);
+    rope_split_kernel<float><<<grid, 256, 0, ctx.st>>>(in, ld_in, rows, n_heads, n_heads_rot, hd, tok_pos, inv, (float*)out, ld_out, (float*)nullptr, 0, 0, n_q_heads, q_gain, k_gain, eps);
   else
-    rope_split_kernel<bf16><<<grid, 256, 0, ctx.st>>>(in, ld_in, rows, n_heads, n_heads_rot, hd, tok_pos, inv, (bf16*)out, ld_out, (bf16*)out_lo, ld_lo, lo_head_begin);
+    rope_split_kernel<bf16><<<grid, 256, 0, ctx.st>>>(in, ld_in, rows, n_heads, n_heads_rot, hd, tok_pos, inv, (bf16*)out, ld_out, (bf16*)out_lo, ld_lo, lo_head_begin, n_q_heads, q_gain, k_gain, eps);
 }
 
 // ---------------------------------------------------------------------------------------

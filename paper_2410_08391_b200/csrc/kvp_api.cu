@@ -33,6 +33,7 @@ const char* validate_model(const kvp_model_cfg* m) {
   if (!m || !m->layers) return "model config or its layer array is NULL";
   if (m->n_layers <= 0 || m->n_layers > 1024) return "n_layers out of range";
   if (m->d_model <= 0 || m->vocab <= 0) return "d_model and vocab must be positive";
+  if (m->qk_norm != 0 && m->qk_norm != 1) return "qk_norm must be 0 or 1";
   if (!(m->rope_theta > 0.f) || !(m->rms_eps >= 0.f)) return "rope_theta must be > 0 and rms_eps >= 0";
   for (int l = 0; l < m->n_layers; ++l) {
     const kvp_layer_cfg& c = m->layers[l];
@@ -48,12 +49,14 @@ const char* unsupported_model(const kvp_model_cfg* m) {
     const kvp_layer_cfg& c = m->layers[l];
     if (c.head_dim % 2 || c.head_dim > 128) return "head_dim must be even and <= 128";
     if (c.n_q_heads / c.n_kv_heads > 8) return "more than 8 query heads per kv head";
+    if (m->qk_norm && c.n_kv_heads > 64) return "key norm with more than 64 kv heads";
   }
   return nullptr;
 }
 
 void plan_model(ModelPlan& p, const kvp_model_cfg* m, int es, bool bf16_mode, size_t& off, bool with_head) {
   p.n_layers = m->n_layers; p.d = m->d_model; p.vocab = m->vocab; p.theta = m->rope_theta; p.eps = m->rms_eps;
+  p.qk_norm = m->qk_norm != 0;
   p.max_nqkv = p.max_dq = p.max_dkv = p.max_ffn = p.max_group = p.max_nkv = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
   p.embed = take((size_t)m->vocab * m->d_model * es);
@@ -70,6 +73,8 @@ void plan_model(ModelPlan& p, const kvp_model_cfg* m, int es, bool bf16_mode, si
     L.wd = take((size_t)p.d * L.ffn * es);
     L.attn_norm = take((size_t)p.d * 4);
     L.ffn_norm = take((size_t)p.d * 4);
+    L.q_norm = L.k_norm = 0;
+    if (p.qk_norm) { L.q_norm = take((size_t)L.hd * 4); L.k_norm = take((size_t)L.hd * 4); }
     p.max_nqkv = std::max(p.max_nqkv, L.nqkv); p.max_dq = std::max(p.max_dq, L.dq);
     p.max_ffn = std::max(p.max_ffn, L.ffn); p.max_group = std::max(p.max_group, L.nq / L.nkv);
     p.max_nkv = std::max(p.max_nkv, L.nkv); p.max_dkv = std::max(p.max_dkv, L.dkv);
@@ -89,6 +94,10 @@ void add_model_slots(kvp_handle* h, const char* prefix, const ModelPlan& p, int 
     const LayerPlan& L = p.L[l];
     h->slots[name(l, "attn_norm")] = PackSlot{L.attn_norm, 1, p.d, 0, RowMap{0, 0, 0, 0}};
     h->slots[name(l, "ffn_norm")] = PackSlot{L.ffn_norm, 1, p.d, 0, RowMap{0, 0, 0, 0}};
+    if (p.qk_norm) {
+      h->slots[name(l, "q_norm")] = PackSlot{L.q_norm, 1, L.hd, 0, RowMap{0, 0, 0, 0}};
+      h->slots[name(l, "k_norm")] = PackSlot{L.k_norm, 1, L.hd, 0, RowMap{0, 0, 0, 0}};
+    }
     h->slots[name(l, "wq")] = PackSlot{L.wqkv, L.dq, p.d, dt, RowMap{0, 0, 0, 0}};
     h->slots[name(l, "wk")] = PackSlot{L.wqkv, L.dkv, p.d, dt, RowMap{L.dq, 0, 0, 0}};
     h->slots[name(l, "wv")] = PackSlot{L.wqkv, L.dkv, p.d, dt, RowMap{L.dq + L.dkv, 0, 0, 0}};
@@ -243,12 +252,14 @@ void base_layer_step(kvp_handle* h, const LaunchCtx& ctx, int i, const kvp_cache
   else
     KVP_TIMED(KVP_CLASS_STEP_GEMV, launch_step_gemv(ctx, P + L.wqkv, B.d, n_out, B.d, xb, B.d, batch, qkvb, n_out, GEMV_STORE, 0, 0,
                                                     (const float*)(P + L.attn_norm), B.eps, hb));
+  const float* qn = B.qk_norm ? (const float*)(P + L.q_norm) : nullptr;
+  const float* kn = B.qk_norm ? (const float*)(P + L.k_norm) : nullptr;
   if (generation)
     KVP_TIMED(KVP_CLASS_OTHER, launch_step_append(ctx, qkvb, L.nq, L.nkv, L.hd, B.theta, cache->k_pools[i], cache->v_pools[i], cache->block_table,
-                       cache->max_pages_per_seq, cache->n_pages, cache->seq_lens, batch));
+                       cache->max_pages_per_seq, cache->n_pages, cache->seq_lens, batch, kn, B.eps));
   KVP_TIMED(KVP_CLASS_STEP_ATTN, launch_step_attn(ctx, qkvb, n_out, L.nq, L.nkv, L.hd, B.theta, cache->k_pools[i], cache->v_pools[i], cache->block_table,
                    cache->max_pages_per_seq, cache->n_pages, cache->seq_lens, generation ? 1 : 0, batch, max_keys,
-                   (float*)(ws + w.part), ab));
+                   (float*)(ws + w.part), ab, qn, B.eps));
   if (tc) {
     float* gub = (float*)(ws + w.gub);
     step_proj_tc(h, ctx, w, ws, PREP_PLAIN, ab, L.dq, L.dq, batch, nullptr, 0, P + L.wo, B.d, xb, B.d, false, err);
@@ -295,6 +306,8 @@ bool base_step_fused(kvp_handle* h, const LaunchCtx& ctx, const kvp_cache* cache
     MegaLayer& m = p.layers[i];
     m.wqkv = P + L.wqkv; m.wo = P + L.wo; m.wgu = P + L.wgu; m.wd = P + L.wd;
     m.attn_norm = (const float*)(P + L.attn_norm); m.ffn_norm = (const float*)(P + L.ffn_norm);
+    m.q_norm = B.qk_norm ? (const float*)(P + L.q_norm) : nullptr;
+    m.k_norm = B.qk_norm ? (const float*)(P + L.k_norm) : nullptr;
     m.kpool = cache->k_pools[i]; m.vpool = cache->v_pools[i];
     m.nq = L.nq; m.nkv = L.nkv; m.dq = L.dq; m.nqkv = L.nqkv; m.ffn = L.ffn; m.G = L.G;
     min_nkv = std::min(min_nkv, L.nkv);
@@ -440,9 +453,9 @@ kvp_status kvp_create(const kvp_model_cfg* aux, const kvp_model_cfg* base, const
   for (auto& kv : h->slots) {
     const std::string& n = kv.first;
     bool is_kv = ends_with(n, ".wk") || ends_with(n, ".wv");
-    bool base_kv = n.rfind("base.L", 0) == 0 && is_kv;
+    bool base_kv = n.rfind("base.L", 0) == 0 && (is_kv || ends_with(n, ".k_norm"));
     // in the last mapped auxiliary layer only the attention norm and the K/V projections are live
-    bool aux_last_dead = n.rfind(last, 0) == 0 && !(ends_with(n, ".attn_norm") || is_kv);
+    bool aux_last_dead = n.rfind(last, 0) == 0 && !(ends_with(n, ".attn_norm") || ends_with(n, ".k_norm") || is_kv);
     if (aux_last_dead) continue;            // accepted if given, never required
     (base_kv ? h->req_decode_extra : h->req_prefill).push_back(n);
   }
@@ -588,6 +601,9 @@ static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int
     tq.epi = TC_QKV; tq.C = (bf16*)(qkv + (size_t)col_begin * es); tq.ldc = L.nqkv;
     tq.C_lo = (bf16*)kv_lo; tq.ld_lo = 2 * L.dkv; tq.lo_col_begin = q_heads * L.hd;
     tq.rot_cols = (q_heads + L.nkv) * L.hd; tq.hd = L.hd; tq.rope_tab = rope_tab; tq.tok_pos = tok_pos;
+    const float* qn = A.qk_norm ? (const float*)(P + L.q_norm) : nullptr;
+    const float* kn = A.qk_norm ? (const float*)(P + L.k_norm) : nullptr;
+    tq.q_gain = qn; tq.k_gain = kn; tq.q_cols = q_heads * L.hd; tq.eps = A.eps;
     if (!try_tc(h, ctx, tq, KVP_CLASS_AUX_GEMM, &tc_err)) {
       GemmArgs g{};
       g.A = hbuf; g.lda = A.d; g.M = T; g.K = A.d;
@@ -597,7 +613,7 @@ static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int
       g.C = qkv32; g.ldc = g.N;
       KVP_TIMED(KVP_CLASS_AUX_GEMM, launch_gemm_simt(ctx, g, EPI_STORE32));
       KVP_TIMED(KVP_CLASS_OTHER, launch_rope_split(ctx, qkv32, g.N, T, g.N / L.hd, q_heads + L.nkv, L.hd, tok_pos, A.theta,
-                                                   qkv + (size_t)col_begin * es, L.nqkv, kv_lo, 2 * L.dkv, q_heads));
+                                                   qkv + (size_t)col_begin * es, L.nqkv, kv_lo, 2 * L.dkv, q_heads, q_heads, qn, kn, A.eps));
     }
     // predictor: K_hat_i = K_A,j FK_i^T, V_hat_i = V_A,j FV_i^T for every base layer i with j_i = j
     const PredGroup& pg = h->groups[j];

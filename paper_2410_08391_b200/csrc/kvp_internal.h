@@ -15,11 +15,13 @@ struct LayerPlan {
   int dq, dkv, nqkv;   // nq*hd, nkv*hd, (nq + 2 nkv)*hd
   int G;               // gate/up row interleave of the packed w_gate/w_up (0 = [gate; up])
   size_t wqkv, wo, wgu, wd, attn_norm, ffn_norm;   // byte offsets into the packed buffer
+  size_t q_norm, k_norm;                           // query / key norm gains (fp32 [hd]); only with qk_norm
 };
 
 struct ModelPlan {
   int n_layers, d, vocab;
   float theta, eps;
+  bool qk_norm;
   std::vector<LayerPlan> L;
   size_t embed, final_norm, lm_head;
   int max_nqkv, max_dq, max_dkv, max_ffn, max_group, max_nkv;

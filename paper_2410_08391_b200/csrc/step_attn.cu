@@ -49,7 +49,8 @@ __global__ void __launch_bounds__(512) step_attn_ring_kernel(const float* __rest
                                                              const bf16* __restrict__ kpool, const bf16* __restrict__ vpool,
                                                              const int* __restrict__ block_table, int mpps, int n_pages,
                                                              const int* __restrict__ seq_lens, int extra, int n_split,
-                                                             float* __restrict__ part, float* __restrict__ out, int* status) {
+                                                             float* __restrict__ part, float* __restrict__ out, int* status,
+                                                             const float* __restrict__ q_gain, float eps) {
   constexpr int PAGE_BYTES = PAGE_TOKENS * HD * 2;       // one K or V page of one kv head
   constexpr int CH = HD / 8;                             // 16-byte pieces per key row
   constexpr int DP = HD / 64;                            // dims per thread in the value sum (1 or 2)
@@ -62,6 +63,7 @@ __global__ void __launch_bounds__(512) step_attn_ring_kernel(const float* __rest
   float* alpha = l_run + MAXG;
   __shared__ __align__(8) unsigned long long bars[ST];
   __shared__ int s_ok;
+  __shared__ float rq[MAXG];
   const int group = nq / nkv;
   const int sp = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -94,7 +96,8 @@ __global__ void __launch_bounds__(512) step_attn_ring_kernel(const float* __rest
     s_ok = 1;
     for (int it = 0; it < min(ST - 1, n_it); ++it) issue(it);
   }
-  // queries of the group: RoPE at the last position, scaled by 1/sqrt(hd)
+  // queries of the group: (query norm,) RoPE at the last position, scaled by 1/sqrt(hd)
+  if (q_gain) head_rnorm(q + (size_t)b * ldq + (size_t)kvh * group * HD, group, HD, eps, rq);
   {
     const float scale = rsqrtf((float)HD);
     constexpr int half = HD / 2;
@@ -103,7 +106,8 @@ __global__ void __launch_bounds__(512) step_attn_ring_kernel(const float* __rest
       const float* qh = q + (size_t)b * ldq + (size_t)(kvh * group + h) * HD;
       float sn, cs;
       rope_sincos(pos, inv.f[c], &sn, &cs);
-      const float x1 = qh[c], x2 = qh[c + half];
+      float x1 = qh[c], x2 = qh[c + half];
+      if (q_gain) { x1 *= rq[h] * q_gain[c]; x2 *= rq[h] * q_gain[c + half]; }
       qs[h * HD + c] = (x1 * cs - x2 * sn) * scale;
       qs[h * HD + c + half] = (x2 * cs + x1 * sn) * scale;
     }
@@ -228,7 +232,7 @@ __global__ void __launch_bounds__(512) step_attn_ring_kernel(const float* __rest
 template <int HD>
 cudaError_t go(dim3 grid, int threads, cudaStream_t st, const float* q, int ldq, int nq, int nkv, const InvFreq& inv, const bf16* kpool,
                const bf16* vpool, const int* block_table, int mpps, int n_pages, const int* seq_lens, int extra, int n_split,
-               float* part, float* out, int* status) {
+               float* part, float* out, int* status, const float* q_gain, float eps) {
   const size_t smem = (size_t)ST * 2 * PAGE_TOKENS * HD * 2 + (size_t)(MAXG * HD + MAXG * PAGE_TOKENS + 3 * MAXG) * sizeof(float);
   static bool attr_set = false;
   if (!attr_set) {
@@ -237,7 +241,7 @@ cudaError_t go(dim3 grid, int threads, cudaStream_t st, const float* q, int ldq,
     attr_set = true;
   }
   step_attn_ring_kernel<HD><<<grid, threads, smem, st>>>(q, ldq, nq, nkv, inv, kpool, vpool, block_table, mpps, n_pages, seq_lens, extra,
-                                                         n_split, part, out, status);
+                                                         n_split, part, out, status, q_gain, eps);
   return cudaGetLastError();
 }
 
@@ -250,7 +254,7 @@ bool step_attn_ring_supported(int dtype, int nq, int nkv, int hd, const void* kp
 
 cudaError_t launch_step_attn_ring(const LaunchCtx& ctx, const float* q, int ldq, int nq, int nkv, int hd, float theta, const void* kpool,
                                   const void* vpool, const int* block_table, int mpps, int n_pages, const int* seq_lens, int extra,
-                                  int batch, int n_split, float* part, float* out) {
+                                  int batch, int n_split, float* part, float* out, const float* q_gain, float eps) {
   InvFreq inv;
   fill_inv_freq(&inv, hd, theta);
   dim3 grid(n_split, nkv, batch);
@@ -258,7 +262,7 @@ cudaError_t launch_step_attn_ring(const LaunchCtx& ctx, const float* q, int ldq,
   ++*ctx.n_launch;
   if (hd == 64)
     return go<64>(grid, threads, ctx.st, q, ldq, nq, nkv, inv, (const bf16*)kpool, (const bf16*)vpool, block_table, mpps, n_pages, seq_lens,
-                  extra, n_split, part, out, ctx.status);
+                  extra, n_split, part, out, ctx.status, q_gain, eps);
   return go<128>(grid, threads, ctx.st, q, ldq, nq, nkv, inv, (const bf16*)kpool, (const bf16*)vpool, block_table, mpps, n_pages, seq_lens,
-                 extra, n_split, part, out, ctx.status);
+                 extra, n_split, part, out, ctx.status, q_gain, eps);
 }

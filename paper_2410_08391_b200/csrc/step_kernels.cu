@@ -275,8 +275,10 @@ __global__ void __launch_bounds__(128) step_attn_kernel(const float* __restrict_
                                                         const T* __restrict__ kpool, const T* __restrict__ vpool,
                                                         const int* __restrict__ block_table, int mpps, int n_pages,
                                                         const int* __restrict__ seq_lens, int extra, int n_split,
-                                                        float* __restrict__ part, float* __restrict__ out, int* status) {
+                                                        float* __restrict__ part, float* __restrict__ out, int* status,
+                                                        const float* __restrict__ q_gain, float eps) {
   extern __shared__ float sm[];
+  __shared__ float rq[MAXG];
   int group = nq / nkv;
   float* qs = sm;                              // [MAXG][hd]
   float* red = qs + MAXG * hd;                 // [4 warps][MAXG][hd + 2]
@@ -286,12 +288,14 @@ __global__ void __launch_bounds__(128) step_attn_kernel(const float* __restrict_
   int pos = n_keys - 1;
   float scale = rsqrtf((float)hd);
   int half = hd >> 1;
+  if (q_gain) head_rnorm(q + (size_t)b * ldq + (size_t)kvh * group * hd, group, hd, eps, rq);
   for (int i = threadIdx.x; i < group * half; i += blockDim.x) {
     int h = i / half, c = i - h * half;
     const float* qh = q + (size_t)b * ldq + (size_t)(kvh * group + h) * hd;
     float sn, cs;
     rope_sincos(pos, inv.f[c], &sn, &cs);
     float x1 = qh[c], x2 = qh[c + half];
+    if (q_gain) { x1 *= rq[h] * q_gain[c]; x2 *= rq[h] * q_gain[c + half]; }
     qs[h * hd + c] = (x1 * cs - x2 * sn) * scale;
     qs[h * hd + c + half] = (x2 * cs + x1 * sn) * scale;
   }
@@ -437,8 +441,10 @@ __global__ void __launch_bounds__(128) step_attn_paged_kernel(const float* __res
                                                               const T* __restrict__ kpool, const T* __restrict__ vpool,
                                                               const int* __restrict__ block_table, int mpps, int n_pages,
                                                               const int* __restrict__ seq_lens, int extra, int n_split,
-                                                              float* __restrict__ part, float* __restrict__ out, int* status) {
+                                                              float* __restrict__ part, float* __restrict__ out, int* status,
+                                                              const float* __restrict__ q_gain, float eps) {
   extern __shared__ __align__(16) unsigned char sm_raw[];
+  __shared__ float rq[MAXG];
   const int group = nq / nkv;
   const int row_bytes = hd * (int)sizeof(T) + 16;           // padded: conflict-free row-per-thread reads
   unsigned char* Ks = sm_raw;
@@ -454,12 +460,14 @@ __global__ void __launch_bounds__(128) step_attn_paged_kernel(const float* __res
   const int pos = n_keys - 1;
   const float scale = rsqrtf((float)hd);
   const int half = hd >> 1;
+  if (q_gain) head_rnorm(q + (size_t)b * ldq + (size_t)kvh * group * hd, group, hd, eps, rq);
   for (int i = tid; i < group * half; i += 128) {
     int h = i / half, c = i - h * half;
     const float* qh = q + (size_t)b * ldq + (size_t)(kvh * group + h) * hd;
     float sn, cs;
     rope_sincos(pos, inv.f[c], &sn, &cs);
     float x1 = qh[c], x2 = qh[c + half];
+    if (q_gain) { x1 *= rq[h] * q_gain[c]; x2 *= rq[h] * q_gain[c + half]; }
     qs[h * hd + c] = (x1 * cs - x2 * sn) * scale;
     qs[h * hd + c + half] = (x2 * cs + x1 * sn) * scale;
   }
@@ -583,14 +591,15 @@ int step_attn_splits(int batch, int nkv, int max_keys) {
 
 void launch_step_attn(const LaunchCtx& ctx, const float* q, int ldq, int nq, int nkv, int hd, float theta,
                       const void* kpool, const void* vpool, const int* block_table, int mpps, int n_pages,
-                      const int* seq_lens, int extra, int batch, int max_keys, float* part, float* out) {
+                      const int* seq_lens, int extra, int batch, int max_keys, float* part, float* out, const float* q_gain,
+                      float eps) {
   // every sequence attends to seq_lens[b] + extra keys; max_keys bounds that count (host copy).
   InvFreq inv;
   fill_inv_freq(&inv, hd, theta);
   int n_split = step_attn_splits(batch, nkv, max_keys);
   dim3 grid(n_split, nkv, batch);
   if (step_attn_ring_supported(ctx.dtype, nq, nkv, hd, kpool, vpool)) {
-    launch_step_attn_ring(ctx, q, ldq, nq, nkv, hd, theta, kpool, vpool, block_table, mpps, n_pages, seq_lens, extra, batch, n_split, part, out);
+    launch_step_attn_ring(ctx, q, ldq, nq, nkv, hd, theta, kpool, vpool, block_table, mpps, n_pages, seq_lens, extra, batch, n_split, part, out, q_gain, eps);
     if (n_split > 1) {
       ++*ctx.n_launch;
       step_attn_merge_kernel<<<dim3(nq, batch), 64, 0, ctx.st>>>(part, nq, hd, n_split, out);
@@ -604,19 +613,19 @@ void launch_step_attn(const LaunchCtx& ctx, const float* q, int ldq, int nq, int
     if (ctx.dtype == 0) {
       cudaFuncSetAttribute(step_attn_paged_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       step_attn_paged_kernel<float><<<grid, 128, smem, ctx.st>>>(q, ldq, nq, nkv, hd, inv, (const float*)kpool, (const float*)vpool,
-                                                                 block_table, mpps, n_pages, seq_lens, extra, n_split, part, out, ctx.status);
+                                                                 block_table, mpps, n_pages, seq_lens, extra, n_split, part, out, ctx.status, q_gain, eps);
     } else {
       step_attn_paged_kernel<bf16><<<grid, 128, smem, ctx.st>>>(q, ldq, nq, nkv, hd, inv, (const bf16*)kpool, (const bf16*)vpool,
-                                                                block_table, mpps, n_pages, seq_lens, extra, n_split, part, out, ctx.status);
+                                                                block_table, mpps, n_pages, seq_lens, extra, n_split, part, out, ctx.status, q_gain, eps);
     }
   } else {
     size_t smem = (size_t)(MAXG * hd + 4 * MAXG * (hd + 2)) * sizeof(float);
     if (ctx.dtype == 0)
       step_attn_kernel<float><<<grid, 128, smem, ctx.st>>>(q, ldq, nq, nkv, hd, inv, (const float*)kpool, (const float*)vpool,
-                                                           block_table, mpps, n_pages, seq_lens, extra, n_split, part, out, ctx.status);
+                                                           block_table, mpps, n_pages, seq_lens, extra, n_split, part, out, ctx.status, q_gain, eps);
     else
       step_attn_kernel<bf16><<<grid, 128, smem, ctx.st>>>(q, ldq, nq, nkv, hd, inv, (const bf16*)kpool, (const bf16*)vpool,
-                                                          block_table, mpps, n_pages, seq_lens, extra, n_split, part, out, ctx.status);
+                                                          block_table, mpps, n_pages, seq_lens, extra, n_split, part, out, ctx.status, q_gain, eps);
   }
   if (n_split > 1) {
     ++*ctx.n_launch;
@@ -631,8 +640,11 @@ namespace {
 template <class T>
 __global__ void step_append_kernel(const float* __restrict__ qkv, int nq, int nkv, int hd, const __grid_constant__ InvFreq inv,
                                    T* __restrict__ kpool, T* __restrict__ vpool, const int* __restrict__ block_table,
-                                   int mpps, int n_pages, const int* __restrict__ seq_lens, int* status) {
+                                   int mpps, int n_pages, const int* __restrict__ seq_lens, int* status,
+                                   const float* __restrict__ k_gain, float eps) {
+  __shared__ float rk[64];
   int b = blockIdx.x;
+  if (k_gain) head_rnorm(qkv + (size_t)b * (nq + 2 * nkv) * hd + (size_t)nq * hd, nkv, hd, eps, rk);   // nkv <= 64 (checked by the launcher)
   int pos = seq_lens[b];
   int pg = pos / PAGE_TOKENS;
   int page = pg < mpps ? block_table[(size_t)b * mpps + pg] : -1;
@@ -645,6 +657,7 @@ __global__ void step_append_kernel(const float* __restrict__ qkv, int nq, int nk
     float sn, cs;
     rope_sincos(pos, inv.f[c], &sn, &cs);
     float x1 = kin[h * hd + c], x2 = kin[h * hd + c + half];
+    if (k_gain) { x1 *= rk[h] * k_gain[c]; x2 *= rk[h] * k_gain[c + half]; }
     size_t off = (((size_t)page * nkv + h) * PAGE_TOKENS + row) * hd;
     kpool[off + c] = from_f<T>(x1 * cs - x2 * sn);
     kpool[off + c + half] = from_f<T>(x2 * cs + x1 * sn);
@@ -655,12 +668,13 @@ __global__ void step_append_kernel(const float* __restrict__ qkv, int nq, int nk
 }  // namespace
 
 void launch_step_append(const LaunchCtx& ctx, const float* qkv, int nq, int nkv, int hd, float theta, void* kpool,
-                        void* vpool, const int* block_table, int mpps, int n_pages, const int* seq_lens, int batch) {
+                        void* vpool, const int* block_table, int mpps, int n_pages, const int* seq_lens, int batch,
+                        const float* k_gain, float eps) {
   InvFreq inv;
   fill_inv_freq(&inv, hd, theta);
   ++*ctx.n_launch;
   if (ctx.dtype == 0)
-    step_append_kernel<float><<<batch, 128, 0, ctx.st>>>(qkv, nq, nkv, hd, inv, (float*)kpool, (float*)vpool, block_table, mpps, n_pages, seq_lens, ctx.status);
+    step_append_kernel<float><<<batch, 128, 0, ctx.st>>>(qkv, nq, nkv, hd, inv, (float*)kpool, (float*)vpool, block_table, mpps, n_pages, seq_lens, ctx.status, k_gain, eps);
   else
-    step_append_kernel<bf16><<<batch, 128, 0, ctx.st>>>(qkv, nq, nkv, hd, inv, (bf16*)kpool, (bf16*)vpool, block_table, mpps, n_pages, seq_lens, ctx.status);
+    step_append_kernel<bf16><<<batch, 128, 0, ctx.st>>>(qkv, nq, nkv, hd, inv, (bf16*)kpool, (bf16*)vpool, block_table, mpps, n_pages, seq_lens, ctx.status, k_gain, eps);
 }

@@ -336,12 +336,14 @@ __device__ __noinline__ void attn_item(const MegaParams& p, const MegaLayer& L, 
   const float scale = rsqrtf((float)hd);
   const int half = hd >> 1;
   __syncthreads();                                   // shared memory free (previous item / phase)
+  if (L.q_norm) head_rnorm(q + (size_t)b * ldq + (size_t)kvh * group * hd, group, hd, p.eps, ps);   // ps is free until the first page's scores
   for (int i = tid; i < group * half; i += NT) {
     int h = i / half, c = i - h * half;
     const float* qh = q + (size_t)b * ldq + (size_t)(kvh * group + h) * hd;
     float sn, cs;
     rope_sincos(pos, p.inv.f[c], &sn, &cs);
     float x1 = __ldcg(qh + c), x2 = __ldcg(qh + c + half);
+    if (L.q_norm) { const float rn = ps[h]; x1 *= rn * L.q_norm[c]; x2 *= rn * L.q_norm[c + half]; }
     qs[h * hd + c] = (x1 * cs - x2 * sn) * scale;
     qs[h * hd + c + half] = (x2 * cs + x1 * sn) * scale;
   }
@@ -510,11 +512,15 @@ __global__ void __launch_bounds__(NT, 1) step_mega_kernel(const __grid_constant_
         int row = pos % PAGE_TOKENS, half = p.hd >> 1;
         const float* kin = p.qkvb + (size_t)b * n_out + L.dq;
         const float* vin = kin + (size_t)L.nkv * p.hd;
+        float* rk = reinterpret_cast<float*>(sm_raw);     // the staging area is idle in this phase
+        __syncthreads();
+        if (L.k_norm) head_rnorm(kin, L.nkv, p.hd, p.eps, rk);
         for (int e = tid; e < L.nkv * half; e += NT) {
           int h = e / half, c = e - h * half;
           float sn, cs;
           rope_sincos(pos, p.inv.f[c], &sn, &cs);
           float x1 = __ldcg(kin + h * p.hd + c), x2 = __ldcg(kin + h * p.hd + c + half);
+          if (L.k_norm) { x1 *= rk[h] * L.k_norm[c]; x2 *= rk[h] * L.k_norm[c + half]; }
           size_t off = (((size_t)page * L.nkv + h) * PAGE_TOKENS + row) * p.hd;
           ((T*)L.kpool)[off + c] = from_f<T>(x1 * cs - x2 * sn);
           ((T*)L.kpool)[off + c + half] = from_f<T>(x2 * cs + x1 * sn);

@@ -7,6 +7,7 @@ constexpr int MEGA_MAX_LAYERS = 64;
 struct MegaLayer {
   const void *wqkv, *wo, *wgu, *wd;      // packed weights of the layer (run dtype)
   const float *attn_norm, *ffn_norm;
+  const float *q_norm, *k_norm;          // query / key norm gains [hd], or null
   void *kpool, *vpool;                   // cache pools of the layer
   int nq, nkv, dq, nqkv, ffn, G;
 };

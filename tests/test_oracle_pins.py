@@ -227,9 +227,10 @@ def test_whole_path_matches_scalar_brute_force(bias):
 # --------------------------------------------------------------------------
 # invariants of the method
 # --------------------------------------------------------------------------
-def _identity_setup(seed=0, regime="fanin", L=12):
-    model = wl.ModelCfg(d_model=32, vocab=50, layers=(wl.LayerCfg(4, 2, 8, 40), wl.LayerCfg(2, 1, 8, 24),
-                                                      wl.LayerCfg(4, 4, 8, 56)))
+def _identity_setup(seed=0, regime="fanin", L=12, qk_norm=False):
+    model = wl.ModelCfg(d_model=32, vocab=50, qk_norm=qk_norm,
+                        layers=(wl.LayerCfg(4, 2, 8, 40), wl.LayerCfg(2, 1, 8, 24),
+                                wl.LayerCfg(4, 4, 8, 56)))
     pair = wl.identity_pair(model)
     W = wl.make_weights(pair, seed=seed, regime=regime)
     for k in list(W):
@@ -242,11 +243,12 @@ def _identity_setup(seed=0, regime="fanin", L=12):
     return pair, W, toks
 
 
-def test_identity_predictor_reproduces_base_cache_and_logits():
+@pytest.mark.parametrize("qk_norm", [False, True])
+def test_identity_predictor_reproduces_base_cache_and_logits(qk_norm):
     """aux == base, j_i = i, F = I: the predicted cache is the base model's own prompt cache,
     and the first step (query at position L-1 over L entries, nothing appended) gives the
     base model's ordinary prefill logits at the last position."""
-    pair, W, toks = _identity_setup()
+    pair, W, toks = _identity_setup(qk_norm=qk_norm)
     kv_base, _, logits_full = orc.decoder_prefill(pair.base, W, "base", toks, want_logits=True)
     kv_hat = orc.predict_kv(pair, W, orc.aux_prefill(pair, W, toks))
     for (k, v), (kh, vh) in zip(kv_base, kv_hat):
@@ -256,8 +258,9 @@ def test_identity_predictor_reproduces_base_cache_and_logits():
     np.testing.assert_allclose(logits, logits_full[-1], rtol=1e-10, atol=1e-12)
 
 
-def test_prefill_equals_token_by_token_decoding():
-    pair, W, toks = _identity_setup(seed=1)
+@pytest.mark.parametrize("qk_norm", [False, True])
+def test_prefill_equals_token_by_token_decoding(qk_norm):
+    pair, W, toks = _identity_setup(seed=1, qk_norm=qk_norm)
     kv_full, _, logits_full = orc.decoder_prefill(pair.base, W, "base", toks, want_logits=True)
     cache = [(np.zeros((0, lc.d_kv)), np.zeros((0, lc.d_kv))) for lc in pair.base.layers]
     for t, tok in enumerate(toks):
@@ -283,11 +286,48 @@ def test_decode_step_after_prediction_appends_base_own_entry():
     np.testing.assert_allclose(logits, logits_full[-1], rtol=1e-9, atol=1e-11)
 
 
-def test_shifting_all_positions_changes_nothing():
-    pair, W, toks = _identity_setup(seed=3)
+@pytest.mark.parametrize("qk_norm", [False, True])
+def test_shifting_all_positions_changes_nothing(qk_norm):
+    """With query / key norm this also fixes the order: gains that differ between the two members
+    of a rotated pair keep the scores a function of relative position only if they are applied
+    before the rotation."""
+    pair, W, toks = _identity_setup(seed=3, qk_norm=qk_norm)
     _, x0, l0 = orc.decoder_prefill(pair.base, W, "base", toks, want_logits=True)
     _, x1, l1 = orc.decoder_prefill(pair.base, W, "base", toks, want_logits=True, pos0=37)
     np.testing.assert_allclose(l1, l0, rtol=1e-8, atol=1e-10)
+
+
+def test_qk_norm_makes_every_cached_key_head_unit_rms():
+    """Sec. 7 ("key norm"): with gains of one, every head of every cached key is an RMS-normalised
+    vector, and RoPE (a rotation) keeps its length: |k_head|^2 = head_dim / (1 + eps / ms)."""
+    pair, W, toks = _identity_setup(seed=4, qk_norm=True)
+    for n in list(W):
+        if n.endswith("q_norm") or n.endswith("k_norm"):
+            W[n] = np.ones_like(W[n])
+    kv, _, _ = orc.decoder_prefill(pair.base, W, "base", toks)
+    for (k, _), lc in zip(kv, pair.base.layers):
+        heads = k.reshape(len(toks), lc.n_kv_heads, lc.head_dim)
+        ms = (heads ** 2).mean(-1)
+        assert np.all(ms < 1.0) and np.all(ms > 1.0 - 1e-3), (ms.min(), ms.max())
+
+
+def test_qk_norm_removes_the_scale_of_the_query_and_key_projections():
+    """Scaling W_q and W_k of a layer by positive constants cannot change anything once queries
+    and keys are RMS-normalised per head (up to the eps inside the root); without the norm the
+    same scaling must change the logits."""
+    for qk_norm in (True, False):
+        pair, W, toks = _identity_setup(seed=5, qk_norm=qk_norm)
+        _, _, l0 = orc.decoder_prefill(pair.base, W, "base", toks, want_logits=True)
+        W2 = dict(W)
+        for l in range(pair.base.n_layers):
+            W2[f"base.L{l}.wq"] = W[f"base.L{l}.wq"] * np.float32(4.0)
+            W2[f"base.L{l}.wk"] = W[f"base.L{l}.wk"] * np.float32(0.5)
+        _, _, l1 = orc.decoder_prefill(pair.base, W2, "base", toks, want_logits=True)
+        diff = np.abs(l1 - l0).max() / np.abs(l0).max()
+        if qk_norm:
+            assert diff < 1e-4, diff
+        else:
+            assert diff > 1e-3, diff
 
 
 def test_predictor_is_one_matrix_product_per_layer():

@@ -42,6 +42,16 @@ CASES = [
     # more sequences than the tensor-core step path takes (128): the CUDA-core projections serve the step;
     # many one- and two-token prompts
     ("t_small", [1, 2, 3, 5, 8, 13, 21, 34, 55, 89] * 13, "fanin"),
+    # query / key norm (Sec. 7, "key norm"): bf16 with both head sizes (fused into the QKV epilogue and the
+    # persistent step), fp32 (CUDA-core kernels), more than 4 sequences (tensor-core step projections +
+    # ring attention), a long cache (paged step attention in splits) and the 130-sequence CUDA-core step
+    ("t_small_qkn", [150, 37, 1, 64, 65], "fanin"),
+    ("t_small_qkn", [129, 40], "n002"),
+    ("t_small_qkn_f32", [129, 40, 1], "fanin"),
+    ("t_hd128_qkn", [130, 70, 2], "fanin"),
+    ("t_hd128_qkn", [40, 9, 130, 17, 64, 65, 3, 90, 128], "fanin"),
+    ("t_small_qkn", [4200, 70], "fanin"),
+    ("t_small_qkn", [1, 2, 3, 5, 8, 13, 21, 34, 55, 89] * 13, "fanin"),
 ]
 
 
@@ -63,7 +73,10 @@ def test_prefill_predict_matches_oracle(name, lens, regime):
 
 
 @pytest.mark.parametrize("name,regime,lens", [("t_small", "fanin", [70, 63, 5]), ("t_small_f32", "fanin", [70, 63, 5]),
-                                              ("c1", "n002", [64]), ("t_small", "n002", [70, 63, 5, 64, 1, 30])],
+                                              ("c1", "n002", [64]), ("t_small", "n002", [70, 63, 5, 64, 1, 30]),
+                                              ("t_small_qkn", "fanin", [70, 63, 5]),
+                                              ("t_small_qkn_f32", "fanin", [70, 5]),
+                                              ("t_hd128_qkn", "fanin", [70, 63, 5, 64, 1, 30])],
                          ids=lambda v: str(v).replace(" ", ""))
 def test_decode_steps_match_oracle(name, regime, lens):
     import torch

@@ -52,6 +52,7 @@ class ModelCfg:
     layers: Tuple[LayerCfg, ...]
     rope_theta: float = 10000.0
     rms_eps: float = 1e-6
+    qk_norm: bool = False               # per-head RMSNorm of queries and keys before RoPE (OpenELM's "key norm", Sec. 7)
 
     @property
     def n_layers(self) -> int:
@@ -69,8 +70,8 @@ class PairCfg:
     predictor_bias: bool = False
 
 
-def uniform_model(n_layers, d_model, n_q, n_kv, head_dim, ffn, vocab) -> ModelCfg:
-    return ModelCfg(d_model=d_model, vocab=vocab,
+def uniform_model(n_layers, d_model, n_q, n_kv, head_dim, ffn, vocab, qk_norm=False) -> ModelCfg:
+    return ModelCfg(d_model=d_model, vocab=vocab, qk_norm=qk_norm,
                     layers=tuple(LayerCfg(n_q, n_kv, head_dim, ffn) for _ in range(n_layers)))
 
 
@@ -140,6 +141,14 @@ def pair(name: str) -> PairCfg:
         aux = uniform_model(max(m) + 1, 2048, 32, 8, 64, 5632, 32000)
         return PairCfg(name, aux, base, m)
     # ---- reduced pairs used by tests (several tiles, ragged tails, odd widths) ----
+    if name in ("t_small_qkn", "t_small_qkn_f32"):   # t_small with query / key norm in both models
+        aux = uniform_model(3, 192, 4, 1, 64, 320, 1000, qk_norm=True)
+        base = uniform_model(5, 256, 8, 2, 64, 448, 1000, qk_norm=True)
+        return PairCfg(name, aux, base, (0, 0, 1, 1, 2), dtype="f32" if name.endswith("f32") else "bf16")
+    if name == "t_hd128_qkn":
+        aux = uniform_model(3, 384, 3, 1, 128, 1024, 2048, qk_norm=True)
+        base = uniform_model(4, 768, 6, 2, 128, 2048, 2048, qk_norm=True)
+        return PairCfg("t_hd128_qkn", aux, base, (0, 1, 1, 2))
     if name == "t_lp":        # layer-pruned pair scaled down: aux = every second layer of an 8-layer base
         base = uniform_model(8, 256, 8, 2, 64, 448, 1000)
         aux = uniform_model(4, 256, 8, 2, 64, 448, 1000)
@@ -203,6 +212,9 @@ def weight_shapes(p: PairCfg, with_aux_head: bool = False) -> Dict[str, Tuple[in
             s[b + "wk"] = (lc.d_kv, m.d_model)
             s[b + "wv"] = (lc.d_kv, m.d_model)
             s[b + "wo"] = (m.d_model, lc.d_q)
+            if m.qk_norm:
+                s[b + "q_norm"] = (lc.head_dim,)
+                s[b + "k_norm"] = (lc.head_dim,)
             s[b + "ffn_norm"] = (m.d_model,)
             s[b + "w_gate"] = (lc.ffn_dim, m.d_model)
             s[b + "w_up"] = (lc.ffn_dim, m.d_model)
