@@ -202,7 +202,7 @@ bool ends_with(const std::string& s, const char* suf) {
 // Tries the tcgen05 GEMM; returns false when the shape is not one it takes (caller falls back).
 bool try_tc(kvp_handle* h, const LaunchCtx& ctx, TcGemm& t, int cls, cudaError_t* err) {
   if (!h->use_tc || h->opt.dtype != KVP_BF16) return false;
-  t.n_sm = h->n_sm;
+  t.n_sm = h->gemm_sms;
   if (!tc_gemm_supported(t)) return false;
   TimedScope ts(h, ctx.st, cls);
   cudaError_t e = launch_gemm_tc(t, ctx.status, ctx.st, ctx.n_launch);
@@ -273,10 +273,10 @@ void base_layer_step(kvp_handle* h, const LaunchCtx& ctx, int i, const kvp_cache
   KVP_TIMED(KVP_CLASS_STEP_GEMV, launch_step_gemv(ctx, P + L.wd, L.ffn, B.d, L.ffn, actb, L.ffn, batch, xb, B.d, GEMV_RESID, 0, 0));
 }
 
-// The whole base step (all layers, LM head, argmax) as one persistent kernel; false = not applicable.
-bool base_step_fused(kvp_handle* h, const LaunchCtx& ctx, const kvp_cache* cache, const WsLayout& w, char* ws, int batch,
-                     int max_keys, bool generation, const int* tokens, const int* gather_idx, float* logits,
-                     int32_t* token_out, cudaError_t* err) {
+// Parameters of the persistent step kernel for this call; false = the kernel does not apply.
+bool mega_prepare(kvp_handle* h, const LaunchCtx& ctx, const kvp_cache* cache, const WsLayout& w, char* ws, int batch,
+                  int max_keys, bool generation, const int* tokens, const int* gather_idx, float* logits,
+                  int32_t* token_out, MegaParams* out, int* k_max_out) {
   const ModelPlan& B = h->base;
   int k_max = std::max(B.d, std::max(B.max_dq, B.max_ffn));
   // its attention phase reads cache pages with plain loads: fine for a few thousand keys, several times
@@ -287,7 +287,8 @@ bool base_step_fused(kvp_handle* h, const LaunchCtx& ctx, const kvp_cache* cache
   for (int i = 0; i < B.n_layers; ++i)
     if ((B.d * h->es) % 16 || (B.L[i].dq * h->es) % 16 || (B.L[i].ffn * h->es) % 16) return false;
   const char* P = h->packed;
-  MegaParams p{};
+  MegaParams& p = *out;
+  p = MegaParams{};
   p.n_layers = B.n_layers; p.d = B.d; p.vocab = B.vocab; p.hd = B.L[0].hd; p.batch = batch; p.generation = generation ? 1 : 0;
   p.eps = B.eps;
   fill_inv_freq(&p.inv, p.hd, B.theta);
@@ -297,7 +298,6 @@ bool base_step_fused(kvp_handle* h, const LaunchCtx& ctx, const kvp_cache* cache
   p.xb = (float*)(ws + w.xb); p.qkvb = (float*)(ws + w.qkvb); p.ab = (float*)(ws + w.ab); p.actb = (float*)(ws + w.actb);
   p.part = (float*)(ws + w.part);
   p.attn_done = (int*)(ws + w.attn_done);
-  cudaMemsetAsync(p.attn_done, 0, (size_t)batch * B.max_nkv * 4, ctx.st);
   p.logits = logits; p.token_out = token_out; p.status = ctx.status;
   p.trace = getenv("KVP_MEGA_TRACE") ? (long long*)((char*)ctx.status + 256) : nullptr;
   int min_nkv = B.L[0].nkv;
@@ -313,6 +313,20 @@ bool base_step_fused(kvp_handle* h, const LaunchCtx& ctx, const kvp_cache* cache
     min_nkv = std::min(min_nkv, L.nkv);
   }
   p.n_split = step_attn_splits(batch, min_nkv, max_keys);   // sized for the layer with the fewest kv heads
+  p.layer_begin = 0; p.layer_end = B.n_layers; p.do_embed = 1; p.do_head = 1; p.counter_idx = 0;
+  *k_max_out = k_max;
+  return true;
+}
+
+// The whole base step (all layers, LM head, argmax) as one persistent kernel; false = not applicable.
+// The caller has cleared the first MEGA_STATUS_BYTES of the status block (or at least its counters).
+bool base_step_fused(kvp_handle* h, const LaunchCtx& ctx, const kvp_cache* cache, const WsLayout& w, char* ws, int batch,
+                     int max_keys, bool generation, const int* tokens, const int* gather_idx, float* logits,
+                     int32_t* token_out, cudaError_t* err) {
+  MegaParams p;
+  int k_max = 0;
+  if (!mega_prepare(h, ctx, cache, w, ws, batch, max_keys, generation, tokens, gather_idx, logits, token_out, &p, &k_max)) return false;
+  cudaMemsetAsync(p.attn_done, 0, (size_t)batch * h->base.max_nkv * 4, ctx.st);
   TimedScope ts(h, ctx.st, KVP_CLASS_STEP_FUSED);
   cudaError_t e = launch_step_mega(p, h->opt.dtype, k_max, h->n_sm, ctx.st, ctx.n_launch);
   if (e != cudaSuccess && *err == cudaSuccess) *err = e;
@@ -404,6 +418,14 @@ kvp_status kvp_create(const kvp_model_cfg* aux, const kvp_model_cfg* base, const
       cudaStreamDestroy(h->side);
       h->side = nullptr;
     }
+    cudaGetLastError();
+  }
+  h->gemm_sms = h->n_sm;
+  if (const char* e = getenv("KVP_STEP_SMS")) h->step_sms = atoi(e);
+  if (h->step_sms < 8 || h->step_sms > h->n_sm - 32 || !h->side) h->step_sms = 0;
+  if (h->step_sms) {
+    if (cudaStreamCreateWithFlags(&h->step_st, cudaStreamNonBlocking) != cudaSuccess) h->step_st = nullptr;
+    if (!h->step_st || cudaEventCreateWithFlags(&h->ev_step, cudaEventDisableTiming) != cudaSuccess) h->step_sms = 0;
     cudaGetLastError();
   }
   size_t off = 0;
@@ -548,7 +570,7 @@ static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int
   const ModelPlan& A = h->aux;
   const char* P = h->packed;
   const int T = cs.total, es = h->es;
-  cudaMemsetAsync(status, 0, 16, s);
+  cudaMemsetAsync(status, 0, MEGA_STATUS_BYTES, s);
 
   int* cu_dev = (int*)(ws + w.cu);
   int* tok_pos = (int*)(ws + w.tok_pos);
@@ -584,6 +606,22 @@ static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int
   // (only worth it while a layer's kernels leave SMs idle: with many tokens every kernel fills the GPU by itself)
   const bool fork = h->side != nullptr && !h->timing && T <= 4096;
   bool pending_join = false;
+  // The base step in pieces beside the prefill: piece j = the base layers whose cache (and that of every
+  // layer below them) is complete once auxiliary layer j has gone through the predictor.
+  MegaParams mp;
+  int mega_kmax = 0, piece = 0, base_done = 0;
+  bool piped = fork && h->step_sms > 0 && h->j_max + 1 <= MEGA_COUNTERS &&
+               mega_prepare(h, ctx, cache, w, ws, batch, cs.max_len, false, tokens, last_idx, logits_out, first_token, &mp, &mega_kmax);
+  std::vector<int> ready_after(h->j_max + 2, 0);      // ready_after[j] = base layers runnable after auxiliary layer j
+  if (piped) {
+    int dep = 0, i = 0;
+    for (int j = 0; j <= h->j_max; ++j) {
+      while (i < h->base.n_layers && std::max(dep, h->map[i]) <= j) { dep = std::max(dep, h->map[i]); ++i; }
+      ready_after[j] = i;
+    }
+    cudaMemsetAsync(mp.attn_done, 0, (size_t)batch * h->base.max_nkv * 4, s);
+    h->gemm_sms = h->n_sm - h->step_sms;
+  }
   KVP_TIMED(KVP_CLASS_OTHER, launch_embed(ctx, tokens, nullptr, T, P + A.embed, A.vocab, A.d, x));
   for (int j = 0; j <= h->j_max; ++j) {
     const LayerPlan& L = A.L[j];
@@ -650,6 +688,16 @@ static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int
         cudaEventRecord(h->ev_join, h->side);
         pending_join = true;
       }
+      if (piped && (ready_after[j] > base_done || last)) {
+        cudaStreamWaitEvent(h->step_st, h->ev_join, 0);
+        MegaParams q = mp;
+        q.layer_begin = base_done; q.layer_end = last ? h->base.n_layers : ready_after[j];
+        q.do_embed = base_done == 0; q.do_head = last; q.counter_idx = piece++;
+        // the last piece starts when the prefill has nothing left to run: it takes every SM
+        cudaError_t e = launch_step_mega(q, h->opt.dtype, mega_kmax, last ? h->n_sm : h->step_sms, h->step_st, ctx.n_launch);
+        if (e != cudaSuccess && tc_err == cudaSuccess) tc_err = e;
+        base_done = q.layer_end;
+      }
     }
     if (last) break;
     if (h->use_tc && split && attn_items <= 65535 && attn_tc_supported(L.hd, L.nqkv, qkv, L.dq, attn)) {
@@ -684,9 +732,14 @@ static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int
     if (!try_tc(h, ctx, td, KVP_CLASS_AUX_GEMM, &tc_err)) KVP_TIMED(KVP_CLASS_AUX_GEMM, launch_gemm_simt(ctx, d, EPI_RESID));
   }
   if (pending_join) cudaStreamWaitEvent(s, h->ev_join, 0);     // the base step reads what the predictor wrote
-  if (tc_err != cudaSuccess) return fail(h, KVP_ERR_CUDA, "tensor-core GEMM launch: %s", cudaGetErrorString(tc_err));
+  h->gemm_sms = h->n_sm;
+  if (piped) {                 // the step is already enqueued in pieces: join its stream
+    cudaEventRecord(h->ev_step, h->step_st);
+    cudaStreamWaitEvent(s, h->ev_step, 0);
+  }
+  if (tc_err != cudaSuccess) return fail(h, KVP_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(tc_err));
   // ---- stage 3: one base step per sequence on its last prompt token ----
-  if (!base_step_fused(h, ctx, cache, w, ws, batch, cs.max_len, false, tokens, last_idx, logits_out, first_token, &tc_err)) {
+  if (!piped && !base_step_fused(h, ctx, cache, w, ws, batch, cs.max_len, false, tokens, last_idx, logits_out, first_token, &tc_err)) {
     KVP_TIMED(KVP_CLASS_OTHER, launch_embed(ctx, tokens, last_idx, batch, P + h->base.embed, h->base.vocab, h->base.d, (float*)(ws + w.xb)));
     for (int i = 0; i < h->base.n_layers; ++i) base_layer_step(h, ctx, i, cache, w, ws, batch, cs.max_len, false, &tc_err);
     base_head(h, ctx, w, ws, batch, logits_out, first_token, &tc_err);
@@ -806,7 +859,7 @@ kvp_status kvp_decode_step(kvp_handle* h, const int32_t* tokens, const int32_t* 
   char* ws = (char*)workspace;
   LaunchCtx ctx{(cudaStream_t)stream, &h->n_launch, (int*)(ws + w.status), h->opt.dtype};
   cudaError_t mega_err = cudaSuccess;
-  cudaMemsetAsync((int*)(ws + w.status) + 1, 0, 4, ctx.st);     // barrier counter of the persistent kernel
+  cudaMemsetAsync((char*)(ws + w.status) + 128, 0, MEGA_COUNTERS * 4, ctx.st);     // barrier counters of the persistent kernel
   if (base_step_fused(h, ctx, cache, w, ws, batch, cs.max_len + 1, true, tokens, nullptr, logits_out, next_token, &mega_err)) {
     if (mega_err != cudaSuccess) return fail(h, KVP_ERR_CUDA, "base step launch: %s", cudaGetErrorString(mega_err));
     return check_cuda(h, "kvp_decode_step");
@@ -849,7 +902,7 @@ kvp_status kvp_poll_status(kvp_handle* h, void* workspace, void* stream) {
   cudaStream_t s = (cudaStream_t)stream;
   int code = 0;
   if (cudaStreamSynchronize(s) != cudaSuccess || cudaMemcpy(&code, workspace, 4, cudaMemcpyDeviceToHost) != cudaSuccess ||
-      cudaMemset(workspace, 0, 16) != cudaSuccess) {
+      cudaMemset(workspace, 0, MEGA_STATUS_BYTES) != cudaSuccess) {
     cudaError_t e = cudaGetLastError();
     return fail(h, KVP_ERR_CUDA, "kvp_poll_status: %s", cudaGetErrorString(e));
   }

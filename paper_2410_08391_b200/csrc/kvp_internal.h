@@ -78,6 +78,14 @@ struct kvp_handle {
   cudaStream_t side = nullptr;
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   bool use_side = true;
+  // The base step at small batch is one persistent kernel bound by HBM latency, the auxiliary prefill a chain
+  // of tensor-core kernels: base layer i only needs the predicted cache of layers <= i, so the step runs in
+  // pieces (one per auxiliary layer that completes some base layers' cache) on a stream of its own, on
+  // `step_sms` SMs, while the prefill's kernels size their grids for the others.  0 = the step runs after the prefill.
+  cudaStream_t step_st = nullptr;
+  cudaEvent_t ev_step = nullptr;
+  int step_sms = 72;
+  int gemm_sms = 148;                   // SMs the tensor-core GEMMs of the current call size their grids for
   // instrumentation
   struct TimingRec { int cls; int64_t launches; cudaEvent_t a, b; };
   bool timing = false;
@@ -90,6 +98,8 @@ struct kvp_handle {
     if (ev_fork) cudaEventDestroy(ev_fork);
     if (ev_join) cudaEventDestroy(ev_join);
     if (side) cudaStreamDestroy(side);
+    if (ev_step) cudaEventDestroy(ev_step);
+    if (step_st) cudaStreamDestroy(step_st);
   }
 };
 

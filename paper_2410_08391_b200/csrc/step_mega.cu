@@ -111,7 +111,7 @@ __device__ __forceinline__ void stream_load_phase(const MegaParams& p, WarpStrea
 // Keep the ring full: issue copies of the next chunks of the schedule into free slots.
 template <class T>
 __device__ __forceinline__ void stream_fill(const MegaParams& p, WarpStream& ws, int gw, int GW, int lane) {
-  const int n_stream = 4 * p.n_layers + 1;
+  const int n_stream = 4 * p.layer_end + (p.do_head ? 1 : 0);     // schedule entries of this launch end here
   while (ws.issued - ws.consumed < (unsigned)NSLOT) {
     while (ws.ps < n_stream && ws.n >= ws.N) {
       if (++ws.ps < n_stream) stream_load_phase<T>(p, ws, gw);
@@ -456,7 +456,7 @@ __global__ void __launch_bounds__(NT, 1) step_mega_kernel(const __grid_constant_
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int gw = blockIdx.x * NW + warp, GW = gridDim.x * NW;
   const int batch = p.batch;
-  unsigned* counter = reinterpret_cast<unsigned*>(p.status) + 1;
+  unsigned* counter = reinterpret_cast<unsigned*>(p.status) + 32 + p.counter_idx;
   unsigned long long* best = reinterpret_cast<unsigned long long*>(reinterpret_cast<char*>(p.status) + 64);
   if (tid == 0) {
     *s_abort = 0;
@@ -465,7 +465,7 @@ __global__ void __launch_bounds__(NT, 1) step_mega_kernel(const __grid_constant_
   }
   __syncthreads();
   WarpStream ws;
-  ws.ps = 0; ws.issued = 0; ws.consumed = 0;
+  ws.ps = 4 * p.layer_begin; ws.issued = 0; ws.consumed = 0;
   ws.slot_bytes = p.slot_bytes;
   const unsigned char* ring_ptr = sm_raw + p.stage_bytes + (size_t)warp * NSLOT * p.slot_bytes;
   ws.ring = smem_u32(ring_ptr);
@@ -477,15 +477,16 @@ __global__ void __launch_bounds__(NT, 1) step_mega_kernel(const __grid_constant_
 #define BARRIER()                                                                                                   \
   do {                                                                                                              \
     ++phase;                                                                                                        \
-    if (p.trace && blockIdx.x == 0 && tid == 0 && phase < 1000) p.trace[2 * phase] = clock64();                     \
+    if (p.trace && blockIdx.x == 0 && tid == 0 && phase < 900) p.trace[2 * phase] = clock64();                     \
     if (!grid_barrier(counter, phase * gridDim.x, p.status, s_abort, &s_flag)) {                                    \
       for (int i_ = 0; i_ < 2000; ++i_) __nanosleep(1000); /* let copies in flight land before the CTA goes */      \
       return;                                                                                                       \
     }                                                                                                               \
-    if (p.trace && blockIdx.x == 0 && tid == 0 && phase < 1000) p.trace[2 * phase + 1] = clock64();                 \
+    if (p.trace && blockIdx.x == 0 && tid == 0 && phase < 900) p.trace[2 * phase + 1] = clock64();                 \
   } while (0)
 
   // embedding gather (+ clear the argmax slots)
+  if (p.do_embed)
   for (int i = blockIdx.x * NT + tid; i < batch * p.d; i += gridDim.x * NT) {
     int b = i / p.d, c = i - b * p.d;
     int tok = p.tokens[p.gather_idx ? p.gather_idx[b] : b];
@@ -496,7 +497,7 @@ __global__ void __launch_bounds__(NT, 1) step_mega_kernel(const __grid_constant_
   if (blockIdx.x == 0 && tid < BB) best[tid] = 0ull;
   BARRIER();
 
-  for (int i = 0; i < p.n_layers; ++i) {
+  for (int i = p.layer_begin; i < p.layer_end; ++i) {
     const MegaLayer& L = p.layers[i];
     const int n_out = p.generation ? L.nqkv : L.dq;
     // ---- q (k, v) projection
@@ -593,6 +594,7 @@ __global__ void __launch_bounds__(NT, 1) step_mega_kernel(const __grid_constant_
     gemv_phase<T, BB>(p, stream_desc(p, 4 * i + 3), ws, ring_ptr, xs, p.xb, p.d, gw, GW, lane, nullptr, s_abort);
     BARRIER();
   }
+  if (!p.do_head) return;             // a later launch carries on from the residual stream in xb
   // ---- LM head (final RMSNorm fused) with running argmax
   stage_x<BB>(p.xb, p.d, p.d, batch, p.final_norm, p.eps, xs, red);
   gemv_phase<T, BB>(p, stream_desc(p, 4 * p.n_layers), ws, ring_ptr, xs, p.logits, p.vocab, gw, GW, lane,

@@ -3,6 +3,8 @@
 #include "common.cuh"
 
 constexpr int MEGA_MAX_LAYERS = 64;
+constexpr int MEGA_COUNTERS = 32;      // grid-barrier counter words in the status block (one per launch of a step)
+constexpr int MEGA_STATUS_BYTES = 256; // what a caller clears before a step: status word, argmax slots, counters
 
 struct MegaLayer {
   const void *wqkv, *wo, *wgu, *wd;      // packed weights of the layer (run dtype)
@@ -23,9 +25,13 @@ struct MegaParams {
   float *xb, *qkvb, *ab, *actb, *part;           // workspace: residual, projections, attention out, FFN act, partials
   int* attn_done;                                // [batch * max n_kv] splits finished per (sequence, kv head); zero on entry, left zero
   float* logits; int* token_out;
+  // One launch may cover only base layers [layer_begin, layer_end): the residual stream stays in xb between
+  // launches.  do_embed: start from the token embeddings; do_head: end with the LM head and the token.
+  int layer_begin, layer_end, do_embed, do_head;
+  int counter_idx;                               // which grid-barrier counter word this launch uses (zero on entry)
   int stage_bytes, slot_bytes;                   // shared-memory plan (set by the launcher)
   long long* trace;                              // optional: clock64 of CTA 0 around every barrier (debugging aid)
-  int* status;                                   // [0] status word, [1] barrier counter, +64 bytes: argmax slots
+  int* status;                                   // [0] status word, +64 bytes: argmax slots, +128 bytes: MEGA_COUNTERS barrier counters
   MegaLayer layers[MEGA_MAX_LAYERS];
 };
 
