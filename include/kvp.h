@@ -17,8 +17,8 @@
  *     kvp_create() ran; "host" pointers are ordinary host memory.
  *   - The caller owns ALL device memory (weights, packed weights, workspace, cache
  *     pools, block table, outputs).  The handle borrows the packed-weight pointer
- *     until kvp_destroy(); it owns host metadata, the CUDA graphs it records, and one
- *     internal stream with two events (created by kvp_create on the current device).
+ *     until kvp_destroy(); it owns host metadata, the CUDA graphs it records, and two
+ *     internal streams with their events (created by kvp_create on the current device).
  *   - Calls that take a stream only enqueue work on it and return without
  *     synchronising (except the *_host variant, which synchronises the stream);
  *     arguments are validated on the host before anything is launched.
@@ -180,9 +180,11 @@ kvp_status kvp_load_weights(kvp_handle* h, const kvp_tensor* tensors, int32_t n,
  * schedule into a CUDA graph owned by the handle; later calls with the same arguments replay it
  * (the token values themselves may change between calls).  If `stream` is already being
  * captured by the caller, the kernels are enqueued into the caller's capture instead.
- * For short prompts part of the work (the predictor) is enqueued on the handle's internal
- * stream, forked from and joined back into `stream` with events; from the caller's point of
- * view everything is ordered on `stream` as usual. */
+ * For short prompts part of the work is enqueued on the handle's internal streams, forked from
+ * and joined back into `stream` with events: the predictor of an auxiliary layer beside that
+ * layer's attention and FFN, and (batch <= 4) the base model's step in pieces, each as soon as the
+ * predicted cache of its layers is complete (Fig. 2(b): B needs only the predicted cache).  From
+ * the caller's point of view everything is ordered on `stream` as usual. */
 kvp_status kvp_prefill_predict(kvp_handle* h, const int32_t* tokens, const int32_t* lengths,
                                int32_t batch, const kvp_cache* cache, void* workspace,
                                size_t workspace_bytes, float* logits_out, int32_t* first_token,

@@ -42,6 +42,9 @@ CASES = [
     # more sequences than the tensor-core step path takes (128): the CUDA-core projections serve the step;
     # many one- and two-token prompts
     ("t_small", [1, 2, 3, 5, 8, 13, 21, 34, 55, 89] * 13, "fanin"),
+    # a layer map that skips an auxiliary layer: no predictor and no piece of the base step after that layer
+    ("t_small_gap", [150, 37, 1, 64], "fanin"),
+    ("t_small_gap", [40, 9, 130, 17, 64, 65], "n002"),
     # query / key norm (Sec. 7, "key norm"): bf16 with both head sizes (fused into the QKV epilogue and the
     # persistent step), fp32 (CUDA-core kernels), more than 4 sequences (tensor-core step projections +
     # ring attention), a long cache (paged step attention in splits) and the 130-sequence CUDA-core step

@@ -157,6 +157,10 @@ def pair(name: str) -> PairCfg:
         aux = uniform_model(3, 192, 4, 1, 64, 320, 1000)
         base = uniform_model(5, 256, 8, 2, 64, 448, 1000)
         return PairCfg("t_small", aux, base, (0, 0, 1, 1, 2))
+    if name == "t_small_gap":
+        # same models as t_small; the map skips an auxiliary layer (it still runs: the layers above it need its output)
+        p = pair("t_small")
+        return PairCfg(name, p.aux, p.base, (0, 0, 2, 2, 2))
     if name == "t_small_f32":
         p = pair("t_small")
         return PairCfg("t_small_f32", p.aux, p.base, p.layer_map, dtype="f32")
