@@ -229,7 +229,7 @@ void step_proj_tc(kvp_handle* h, const LaunchCtx& ctx, const WsLayout& w, char* 
   bf16* XB = (bf16*)(ws + w.xbt);
   KVP_TIMED(KVP_CLASS_STEP_GEMV, launch_step_prep(ctx, mode, src, ld_src, K, batch, gain, h->base.eps, G, XB, clear ? Y : nullptr, ldy, N));
   TimedScope ts(h, ctx.st, KVP_CLASS_STEP_GEMV);
-  cudaError_t e = launch_step_gemm_tc((const bf16*)W, K, N, K, XB, batch, Y, ldy, h->n_sm, ctx.status, ctx.st, ctx.n_launch);
+  cudaError_t e = launch_step_gemm_tc((const bf16*)W, K, N, K, XB, batch, Y, ldy, h->step_grid_sms, ctx.status, ctx.st, ctx.n_launch);
   if (e != cudaSuccess && *err == cudaSuccess) *err = e;
 }
 
@@ -420,7 +420,9 @@ kvp_status kvp_create(const kvp_model_cfg* aux, const kvp_model_cfg* base, const
     }
     cudaGetLastError();
   }
-  h->gemm_sms = h->n_sm;
+  h->gemm_sms = h->step_grid_sms = h->n_sm;
+  if (const char* e = getenv("KVP_STEP_TC_SMS")) h->step_tc_sms = atoi(e);
+  if (h->step_tc_sms < 8 || h->step_tc_sms > h->n_sm) h->step_tc_sms = 0;
   if (const char* e = getenv("KVP_STEP_SMS")) h->step_sms = atoi(e);
   if (h->step_sms < 8 || h->step_sms > h->n_sm - 32 || !h->side) h->step_sms = 0;
   if (h->step_sms) {
@@ -622,6 +624,18 @@ static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int
     cudaMemsetAsync(mp.attn_done, 0, (size_t)batch * h->base.max_nkv * 4, s);
     h->gemm_sms = h->n_sm - h->step_sms;
   }
+  // More than 4 sequences: the step is a chain of short per-layer kernels bound by launch latency; the same
+  // pieces go to the step stream as plain launches.  Their projections size their grids for step_tc_sms SMs;
+  // the prefill's GEMMs keep the whole GPU (measured: restricting them costs more than the step gains).
+  const bool piped_tc = !piped && fork && h->step_sms > 0 && h->step_tc_sms > 0 && step_uses_tc(h, batch);
+  if (piped_tc) {
+    int dep = 0, i = 0;
+    for (int j = 0; j <= h->j_max; ++j) {
+      while (i < h->base.n_layers && std::max(dep, h->map[i]) <= j) { dep = std::max(dep, h->map[i]); ++i; }
+      ready_after[j] = i;
+    }
+    h->step_grid_sms = h->step_tc_sms;
+  }
   KVP_TIMED(KVP_CLASS_OTHER, launch_embed(ctx, tokens, nullptr, T, P + A.embed, A.vocab, A.d, x));
   for (int j = 0; j <= h->j_max; ++j) {
     const LayerPlan& L = A.L[j];
@@ -698,6 +712,18 @@ static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int
         if (e != cudaSuccess && tc_err == cudaSuccess) tc_err = e;
         base_done = q.layer_end;
       }
+      if (piped_tc && (ready_after[j] > base_done || last)) {
+        cudaStreamWaitEvent(h->step_st, h->ev_join, 0);
+        LaunchCtx sctx = ctx;
+        sctx.st = h->step_st;
+        const int end = last ? h->base.n_layers : ready_after[j];
+        if (last) h->step_grid_sms = h->n_sm;          // the prefill has nothing left to run
+        if (base_done == 0)
+          launch_embed(sctx, tokens, last_idx, batch, P + h->base.embed, h->base.vocab, h->base.d, (float*)(ws + w.xb));
+        for (int i = base_done; i < end; ++i) base_layer_step(h, sctx, i, cache, w, ws, batch, cs.max_len, false, &tc_err);
+        if (last) base_head(h, sctx, w, ws, batch, logits_out, first_token, &tc_err);
+        base_done = end;
+      }
     }
     if (last) break;
     if (h->use_tc && split && attn_items <= 65535 && attn_tc_supported(L.hd, L.nqkv, qkv, L.dq, attn)) {
@@ -732,14 +758,14 @@ static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int
     if (!try_tc(h, ctx, td, KVP_CLASS_AUX_GEMM, &tc_err)) KVP_TIMED(KVP_CLASS_AUX_GEMM, launch_gemm_simt(ctx, d, EPI_RESID));
   }
   if (pending_join) cudaStreamWaitEvent(s, h->ev_join, 0);     // the base step reads what the predictor wrote
-  h->gemm_sms = h->n_sm;
-  if (piped) {                 // the step is already enqueued in pieces: join its stream
+  h->gemm_sms = h->step_grid_sms = h->n_sm;
+  if (piped || piped_tc) {     // the step is already enqueued in pieces: join its stream
     cudaEventRecord(h->ev_step, h->step_st);
     cudaStreamWaitEvent(s, h->ev_step, 0);
   }
   if (tc_err != cudaSuccess) return fail(h, KVP_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(tc_err));
   // ---- stage 3: one base step per sequence on its last prompt token ----
-  if (!piped && !base_step_fused(h, ctx, cache, w, ws, batch, cs.max_len, false, tokens, last_idx, logits_out, first_token, &tc_err)) {
+  if (!piped && !piped_tc && !base_step_fused(h, ctx, cache, w, ws, batch, cs.max_len, false, tokens, last_idx, logits_out, first_token, &tc_err)) {
     KVP_TIMED(KVP_CLASS_OTHER, launch_embed(ctx, tokens, last_idx, batch, P + h->base.embed, h->base.vocab, h->base.d, (float*)(ws + w.xb)));
     for (int i = 0; i < h->base.n_layers; ++i) base_layer_step(h, ctx, i, cache, w, ws, batch, cs.max_len, false, &tc_err);
     base_head(h, ctx, w, ws, batch, logits_out, first_token, &tc_err);

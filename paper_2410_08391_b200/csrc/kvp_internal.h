@@ -86,6 +86,8 @@ struct kvp_handle {
   cudaEvent_t ev_step = nullptr;
   int step_sms = 72;
   int gemm_sms = 148;                   // SMs the tensor-core GEMMs of the current call size their grids for
+  int step_tc_sms = 96;                 // grid of the step's projections when its per-layer kernels (batch > 4) run beside the prefill
+  int step_grid_sms = 148;              // SMs the step's tensor-core projections size their grids for
   // instrumentation
   struct TimingRec { int cls; int64_t launches; cudaEvent_t a, b; };
   bool timing = false;
