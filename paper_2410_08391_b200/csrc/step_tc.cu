@@ -71,6 +71,7 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
   auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * S + 2 + a); };
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t tmem_cols = max(32, 2 * p.acc_stride);
+  pdl_trigger();      // the next kernel's CTAs may take SMs as this kernel's CTAs leave them
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -91,13 +92,31 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
       int stage = 0; uint32_t phase = 0;
       bool ok = true;
       const uint32_t tx = W_BYTES + 2 * p.Bp * BK * 2;
+      // The weights do not depend on the kernel before this one: the W tiles of the first S k-blocks are
+      // requested before the wait for that kernel, so they stream in while it finishes (all stages are free,
+      // in order, on a fresh pipeline).  The activation tiles of those k-blocks follow after the wait.
+      int pre = 0;
+      {
+        Sched ahead(p);
+        Work wa;
+        while (pre < S && ahead.next(wa)) {
+          for (int kb = wa.kb0; kb < wa.kb1 && pre < S; ++kb, ++pre) {
+            mbar_expect_tx(full_bar(pre), tx);
+            tma_load_2d(smem_base + pre * stage_bytes, &map_w, kb * BK, wa.n0, full_bar(pre));
+          }
+        }
+      }
+      pdl_wait();
+      int issued = 0;
       while (ok && sched.next(w)) {
-        for (int kb = w.kb0; kb < w.kb1 && ok; ++kb) {
-          ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status);
-          if (!ok) break;
+        for (int kb = w.kb0; kb < w.kb1 && ok; ++kb, ++issued) {
           const uint32_t sw = smem_base + stage * stage_bytes;
-          mbar_expect_tx(full_bar(stage), tx);
-          tma_load_2d(sw, &map_w, kb * BK, w.n0, full_bar(stage));
+          if (issued >= pre) {
+            ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status);
+            if (!ok) break;
+            mbar_expect_tx(full_bar(stage), tx);
+            tma_load_2d(sw, &map_w, kb * BK, w.n0, full_bar(stage));
+          }
           tma_load_2d(sw + W_BYTES, &map_x, kb * BK, 0, full_bar(stage));
           if (++stage == S) { stage = 0; phase ^= 1u; }
         }
@@ -138,6 +157,7 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
     Sched sched(p);
     Work w;
     int acc = 0; uint32_t acc_phase = 0;
+    pdl_wait();       // the output was cleared by the kernel before this one
     while (sched.next(w)) {
       bool ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status);
       ok = __all_sync(0xffffffffu, ok);
@@ -180,6 +200,8 @@ __global__ void __launch_bounds__(256) step_prep_kernel(int mode, const float* _
                                                         const float* __restrict__ gain, float eps, RowMap mg, RowMap mu,
                                                         bf16* __restrict__ XB, float* zero_ptr, int zero_ld, int zero_n) {
   __shared__ float red[8];
+  pdl_trigger();
+  pdl_wait();         // everything below reads or overwrites what earlier kernels of the step use
   const int b = blockIdx.x, tid = threadIdx.x;
   const int k_begin = blockIdx.y * PREP_CHUNK, k_end = min(K, k_begin + PREP_CHUNK);
   bf16* hi = XB + (size_t)b * K;
@@ -260,7 +282,8 @@ void launch_step_prep(const LaunchCtx& ctx, int mode, const float* x, int ldx, i
   const int Bp = step_tc_rows(batch);
   RowMap mg{0, G, 0, K}, mu{G == 0 ? K : 0, G, 1, K};
   ++*ctx.n_launch;
-  step_prep_kernel<<<dim3(Bp, (K + PREP_CHUNK - 1) / PREP_CHUNK), 256, 0, ctx.st>>>(mode, x, ldx, K, batch, Bp, gain, eps, mg, mu, XB, zero_ptr, zero_ld, zero_n);
+  launch_overlapped(step_prep_kernel, dim3(Bp, (K + PREP_CHUNK - 1) / PREP_CHUNK), dim3(256), 0, ctx.st, mode, x, ldx, K, batch, Bp, gain, eps,
+                    mg, mu, XB, zero_ptr, zero_ld, zero_n);
 }
 
 cudaError_t launch_step_gemm_tc(const bf16* W, int ldw, int N, int K, const bf16* XB, int batch, float* Y, int ldy, int n_sm,
@@ -285,6 +308,5 @@ cudaError_t launch_step_gemm_tc(const bf16* W, int ldw, int N, int K, const bf16
   const long long total = (long long)((N + BM - 1) / BM) * ((K + BK - 1) / BK);
   const int grid = (int)(total < n_sm ? total : n_sm);
   ++*n_launch;
-  step_gemm_kernel<<<grid, N_THREADS, smem, st>>>(mw, mx, p);
-  return cudaGetLastError();
+  return launch_overlapped(step_gemm_kernel, dim3(grid), dim3(N_THREADS), (size_t)smem, st, mw, mx, p);
 }
