@@ -293,7 +293,12 @@ class Session:
         self.device = torch.device(device)
         torch.cuda.set_device(self.device)
         self.h = kvp_create(pair.aux, pair.base, pair.layer_map, pair.dtype, pair.predictor_bias)
-        self.stream = torch.cuda.current_stream(self.device).cuda_stream
+        # The library replays a recorded CUDA graph per call, which the legacy default stream cannot record:
+        # when that is the current stream the session works on a stream of its own and orders it against the
+        # current stream around every call, so a caller still sees everything in the current stream's order.
+        cur = torch.cuda.current_stream(self.device)
+        self.torch_stream = torch.cuda.Stream(self.device) if cur.cuda_stream == 0 else cur
+        self.stream = self.torch_stream.cuda_stream
         self.packed = torch.empty(kvp_packed_weight_bytes(self.h) + 256, dtype=torch.uint8, device=self.device)
         self.load(weights)
         self.max_batch, self.max_total = max_batch, max_total_tokens
@@ -322,14 +327,33 @@ class Session:
             kvp_load_weights(self.h, batch, self.packed, self.stream)
             torch.cuda.synchronize()
 
+    def enter(self):
+        """Orders the session's stream after the current torch stream; returns the latter for leave()."""
+        cur = self.torch.cuda.current_stream(self.device)
+        if cur.cuda_stream != self.stream:
+            self.torch_stream.wait_stream(cur)
+        return cur
+
+    def leave(self, cur):
+        if cur.cuda_stream != self.stream:
+            cur.wait_stream(self.torch_stream)
+
     def prefill_predict(self, tokens_dev, lengths: Sequence[int]):
         b = len(lengths)
-        kvp_prefill_predict(self.h, tokens_dev, lengths, self.cache, self.workspace, self.logits, self.first, self.stream)
+        cur = self.enter()
+        try:
+            kvp_prefill_predict(self.h, tokens_dev, lengths, self.cache, self.workspace, self.logits, self.first, self.stream)
+        finally:
+            self.leave(cur)
         return self.logits[:b], self.first[:b]
 
     def decode_step(self, tokens_dev, lengths: Sequence[int]):
         b = len(lengths)
-        kvp_decode_step(self.h, tokens_dev, lengths, self.cache, self.workspace, self.logits, self.first, self.stream)
+        cur = self.enter()
+        try:
+            kvp_decode_step(self.h, tokens_dev, lengths, self.cache, self.workspace, self.logits, self.first, self.stream)
+        finally:
+            self.leave(cur)
         return self.logits[:b], self.first[:b]
 
     def poll(self):

@@ -783,7 +783,8 @@ kvp_status kvp_prefill_predict(kvp_handle* h, const int32_t* tokens, const int32
                                int32_t* first_token, void* stream) {
   cudaStream_t s = (cudaStream_t)stream;
   cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
-  bool graph_ok = h && h->use_graph && !h->timing && lengths && cache && cache->k_pools && cache->v_pools && batch > 0 &&
+  // (the legacy default stream cannot record)
+  bool graph_ok = h && h->use_graph && s != nullptr && s != cudaStreamLegacy && !h->timing && lengths && cache && cache->k_pools && cache->v_pools && batch > 0 &&
                   batch <= KVP_MAX_BATCH && cudaStreamIsCapturing(s, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusNone;
   if (!graph_ok) {
     cudaGetLastError();

@@ -35,7 +35,9 @@ def test_static_scratch_step_matches_workspace_step_twice_in_a_row():
         for step in range(2):
             nxt = torch.from_numpy(g.integers(0, pair.base.vocab, size=len(lens)).astype(np.int32)).to(a.device)
             la, ta = a.decode_step(nxt, cur)
+            c = b.enter()
             kvp.kvp_decode_step_static(b.h, nxt, cur, b.cache, b.logits, b.first, status, b.stream)
+            b.leave(c)
             torch.cuda.synchronize()
             assert int(status.item()) == 0
             la, lb = la.cpu().numpy(), b.logits[:len(lens)].cpu().numpy()
