@@ -181,7 +181,7 @@ def main():
     lens = [int(x) for x in pr.lengths]
     work = wl.algorithmic_work(pair, lens)
     sess = kvp.Session(pair, W, max_batch=pr.batch, max_total_tokens=pr.total, max_len=max(lens), device=dev,
-                       extra_len=max(args.decode_steps, 0) + 3)
+                       extra_len=2 * max(args.decode_steps, 0) + 4)
     toks = torch.from_numpy(pr.tokens).to(dev)
 
     def barrier():
@@ -258,6 +258,25 @@ def main():
         dms = max_over_ranks(d0.elapsed_time(d1) / args.decode_steps, dist, dev)
         decode = {"steps": args.decode_steps, "ms_per_step": dms, "tok_per_s": world * pr.batch / (dms * 1e-3),
                   "ttft_over_step": ms_step / dms}
+        # the same loop as ONE recorded step replayed: positions live in seq_lens on the device, the fed-back token
+        # in `tok`, so a recorded kvp_decode_step stays valid while the block table has room
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=sess.torch_stream):
+            _, nxt = sess.decode_step(tok, cur)
+            tok.copy_(nxt)
+        torch.cuda.synchronize()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record(sess.torch_stream)
+        with torch.cuda.stream(sess.torch_stream):
+            for _ in range(args.decode_steps):
+                graph.replay()
+        g1.record(sess.torch_stream)
+        torch.cuda.synchronize()
+        sess.poll()
+        want = [c + args.decode_steps for c in cur]
+        assert sess.cache.seq_lens[:pr.batch].cpu().tolist() == want, "replayed steps did not advance the cache"
+        gms = max_over_ranks(g0.elapsed_time(g1) / args.decode_steps, dist, dev)
+        decode.update({"graph_ms_per_step": gms, "graph_tok_per_s": world * pr.batch / (gms * 1e-3)})
 
     # ---- per-kernel-class device times (separate pass: events around every launch) ----
     kvp.kvp_timing_enable(sess.h, True)

@@ -203,7 +203,12 @@ kvp_status kvp_prefill_predict_host(kvp_handle* h, const int32_t* tokens_host,
  * q, k, v of `tokens[b]` with its own projections at position seq_lens[b], appends k
  * (after RoPE) and v to the cache, attends over seq_lens[b] + 1 entries and emits logits;
  * seq_lens[b] += 1.  lengths_host[b] must equal the current seq_lens[b] (host copy used
- * for validation and scheduling).  KVP_ERR_CACHE_FULL if a sequence has no room left. */
+ * for validation and scheduling).  KVP_ERR_CACHE_FULL if a sequence has no room left.
+ * The call may be recorded into a CUDA graph by the caller (stream capture) and replayed for the
+ * following steps: the kernels read positions from seq_lens and the token from `tokens` on the
+ * device; lengths_host only sizes the key-range splits and checks capacity at recording time, so
+ * the caller has to make sure that the block table has pages for every replayed step (the choice
+ * of kernels and splits stays the one made for the recorded length). */
 kvp_status kvp_decode_step(kvp_handle* h, const int32_t* tokens /* dev [batch] */,
                            const int32_t* lengths_host, int32_t batch, const kvp_cache* cache,
                            void* workspace, size_t workspace_bytes, float* logits_out,

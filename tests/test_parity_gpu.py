@@ -118,6 +118,54 @@ def test_decode_steps_match_oracle(name, regime, lens):
         s.close()
 
 
+@pytest.mark.parametrize("lens", [[70, 63, 5], [64, 1, 30, 9, 127, 128]], ids=lambda v: str(v).replace(" ", ""))
+def test_recorded_decode_step_replays_for_later_positions(lens):
+    """One kvp_decode_step recorded into a CUDA graph and replayed: positions come from seq_lens on the device and
+    the token from a device buffer, so every replay is the next step of the generation loop (Fig. 2(b))."""
+    import torch
+    pair = wl.pair("t_small")
+    W = wl.make_weights(pair, seed=5, regime="fanin")
+    pr = wl.custom_prompts(pair.base.vocab, lens, seed=5)
+    steps = 3
+    s = make_session(pair, W, pr, extra_len=steps + 1)
+    tol = TOL[pair.dtype]
+    try:
+        s.prefill_predict(torch.from_numpy(pr.tokens).to(s.device), lens)
+        s.poll()
+        ref = orc.prefill_predict(pair, W, pr)
+        caches = {b: ref[b][0] for b in range(pr.batch)}
+        g = np.random.default_rng(9)
+        forced = g.integers(0, pair.base.vocab, size=(steps + 1, pr.batch)).astype(np.int32)
+        tok = torch.from_numpy(forced[0]).to(s.device)
+        s.decode_step(tok, lens)                      # a warm-up step outside the recording (it is step 0)
+        s.poll()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=s.torch_stream):
+            s.decode_step(tok, [c + 1 for c in lens])
+        torch.cuda.synchronize()
+        for b in range(pr.batch):
+            _, caches[b] = orc.decode_step(pair, W, int(forced[0][b]), caches[b])
+        cur = [c + 1 for c in lens]
+        for step in range(1, steps + 1):
+            tok.copy_(torch.from_numpy(forced[step]).to(s.device))
+            torch.cuda.synchronize()
+            with torch.cuda.stream(s.torch_stream):
+                graph.replay()
+            torch.cuda.synchronize()
+            s.poll()
+            logits = s.logits[:pr.batch].cpu().numpy()
+            cur = [c + 1 for c in cur]
+            assert s.cache.seq_lens[:pr.batch].cpu().tolist() == cur
+            for b in range(pr.batch):
+                ref_logits, caches[b] = orc.decode_step(pair, W, int(forced[step][b]), caches[b])
+                assert rel_fro(logits[b], ref_logits) <= tol
+                for i in range(pair.base.n_layers):
+                    k, v = s.cache.gather(i, b, cur[b])
+                    assert rel_fro(k, caches[b][i][0]) <= tol and rel_fro(v, caches[b][i][1]) <= tol
+    finally:
+        s.close()
+
+
 def test_sequence_alone_equals_sequence_in_batch():
     import torch
     pair = wl.pair("t_small")
