@@ -155,12 +155,15 @@ def qk_norm(cfg, W, b: str, q, k):
 # a decoder over a whole prompt (used for A, and for B in the invariants)
 # ----------------------------------------------------------------------------
 def decoder_prefill(cfg, W, prefix: str, tokens: np.ndarray, *, pos0: int = 0,
-                    want_logits: bool = False, n_layers: Optional[int] = None):
+                    want_logits: bool = False, n_layers: Optional[int] = None, kv_given=None):
     """Run decoder `prefix` ("aux" or "base") over one prompt.
 
     Returns (kv, x, logits): kv[l] = (k, v) with k [L, nkv_l*hd] after RoPE and
     v [L, nkv_l*hd]; x the final residual stream [L, d]; logits [L, vocab] or None.
     `pos0` shifts every position (only the RoPE shift-invariance pin uses it).
+    `kv_given[l] = (K, V)`: attention reads these keys and values (entry s visible to query t >= s)
+    instead of the layer's own projections: the training-time forward of Sec. 4.1 ("masked
+    cross-attention with the predicted KV cache"); kv still returns the layer's own k, v.
     """
     L = len(tokens)
     pos = np.arange(L) + pos0
@@ -178,6 +181,9 @@ def decoder_prefill(cfg, W, prefix: str, tokens: np.ndarray, *, pos0: int = 0,
         q = rope(q, pos, cfg.rope_theta)
         k = rope(k, pos, cfg.rope_theta)
         kv.append((k.reshape(L, -1), v.reshape(L, -1)))
+        if kv_given is not None:
+            k = np.asarray(kv_given[l][0], dtype=F64).reshape(L, lc.n_kv_heads, lc.head_dim)
+            v = np.asarray(kv_given[l][1], dtype=F64).reshape(L, lc.n_kv_heads, lc.head_dim)
         a = attention(q, k, v, np.arange(L))
         x = x + a.reshape(L, -1) @ _w(W, b + "wo").T
         h2 = rmsnorm(x, W[b + "ffn_norm"], cfg.rms_eps)
@@ -274,6 +280,25 @@ def decode_step(pair, W, token: int, cache):
         x = _base_block_tail(cfg, W, i, x, a)
     logits = (rmsnorm(x, W["base.final_norm"], cfg.rms_eps) @ _w(W, "base.lm_head").T)[0]
     return logits, new_cache
+
+
+# ----------------------------------------------------------------------------
+# training-time forward and consistency terms  (Sec. 4.1 "Training", Sec. 4.3)
+# ----------------------------------------------------------------------------
+def train_forward(pair, W, tokens: np.ndarray):
+    """One prompt through the training-time graph, forward only (Fig. 2(a)):
+    KV_A <- A(I);  KV_hat <- P(KV_A);  b <- B(I) with KV_hat as the keys and values of every layer's
+    attention (query t sees predicted entries 0..t);  KV_B <- the base model's cache from its ordinary
+    forward over I.  Returns (logits_b [L, vocab], abs_k, abs_v, n_k) with abs_k[i] = sum over tokens and
+    columns of |K_hat_i - K_B,i|, abs_v[i] likewise, n_k[i] = L * d_kvB_i: the consistency loss of Sec. 4.3
+    is the mean abs_k[i] / n_k[i] (and the same for V), summed or averaged over layers."""
+    kv_hat = predict_kv(pair, W, aux_prefill(pair, W, tokens))
+    kv_b, _, _ = decoder_prefill(pair.base, W, "base", tokens)
+    _, _, logits = decoder_prefill(pair.base, W, "base", tokens, want_logits=True, kv_given=kv_hat)
+    abs_k = [float(np.abs(kh - kb).sum()) for (kh, _), (kb, _) in zip(kv_hat, kv_b)]
+    abs_v = [float(np.abs(vh - vb).sum()) for (_, vh), (_, vb) in zip(kv_hat, kv_b)]
+    n = [int(kb.size) for kb, _ in kv_b]
+    return logits, abs_k, abs_v, n
 
 
 def argmax_lowest(logits: np.ndarray) -> int:

@@ -297,6 +297,53 @@ def test_shifting_all_positions_changes_nothing(qk_norm):
     np.testing.assert_allclose(l1, l0, rtol=1e-8, atol=1e-10)
 
 
+# --------------------------------------------------------------------------
+# training-time forward (Sec. 4.1 "Training", Sec. 4.3 consistency loss)
+# --------------------------------------------------------------------------
+def test_train_forward_with_identity_predictor_is_the_base_models_own_forward():
+    """aux == base, F = I: the predicted cache is the base model's own, so the forward with the predicted
+    cache gives the base model's ordinary logits at EVERY position and the consistency terms vanish."""
+    pair, W, toks = _identity_setup(seed=6)
+    logits, abs_k, abs_v, n = orc.train_forward(pair, W, toks)
+    _, _, ref = orc.decoder_prefill(pair.base, W, "base", toks, want_logits=True)
+    np.testing.assert_allclose(logits, ref, rtol=1e-9, atol=1e-11)
+    assert max(abs_k) < 1e-9 and max(abs_v) < 1e-9
+    assert n == [len(toks) * lc.d_kv for lc in pair.base.layers]
+
+
+def test_train_forward_last_position_is_the_inference_first_step():
+    """The training-time forward at the last position sees predicted entries 0..L-1 and the query of the last
+    token: exactly the first step of inference (Fig. 2(b)), so its last row of logits equals that step's."""
+    pair = wl.pair("c1")
+    W = wl.make_weights(pair, seed=3, regime="fanin")
+    toks = wl.uniform_tokens(11, pair.base.vocab, 3)
+    logits, _, _, _ = orc.train_forward(pair, W, toks)
+    kv_hat = orc.predict_kv(pair, W, orc.aux_prefill(pair, W, toks))
+    step = orc.base_first_step(pair, W, int(toks[-1]), kv_hat)
+    np.testing.assert_allclose(logits[-1], step, rtol=1e-9, atol=1e-11)
+    # and every earlier row is the first step of the truncated prompt (the predicted cache is causal in the prompt)
+    for t in (0, 4):
+        kv_t = orc.predict_kv(pair, W, orc.aux_prefill(pair, W, toks[:t + 1]))
+        np.testing.assert_allclose(logits[t], orc.base_first_step(pair, W, int(toks[t]), kv_t), rtol=1e-8, atol=1e-10)
+
+
+def test_consistency_terms_are_plain_l1_sums():
+    """Zero predictor: K_hat = V_hat = 0, so the terms are the L1 norms of the base model's own cache, computed
+    here by scalar loops over one layer."""
+    pair = wl.pair("c1")
+    W = wl.make_weights(pair, seed=4, regime="fanin")
+    for n in list(W):
+        if n.startswith("pred."):
+            W[n] = np.zeros_like(W[n])
+    toks = wl.uniform_tokens(6, pair.base.vocab, 4)
+    _, abs_k, abs_v, _ = orc.train_forward(pair, W, toks)
+    kv_b, _, _ = orc.decoder_prefill(pair.base, W, "base", toks)
+    for i in (0, pair.base.n_layers - 1):
+        sk = sum(abs(float(x)) for row in kv_b[i][0] for x in row)
+        sv = sum(abs(float(x)) for row in kv_b[i][1] for x in row)
+        assert abs(abs_k[i] - sk) <= 1e-9 * sk and abs(abs_v[i] - sv) <= 1e-9 * sv
+
+
 def test_qk_norm_makes_every_cached_key_head_unit_rms():
     """Sec. 7 ("key norm"): with gains of one, every head of every cached key is an RMS-normalised
     vector, and RoPE (a rotation) keeps its length: |k_head|^2 = head_dim / (1 + eps / ms)."""
