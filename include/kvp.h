@@ -238,6 +238,25 @@ kvp_status kvp_decode_step_static(kvp_handle* h, const int32_t* tokens /* dev [b
                                   float* logits_out, int32_t* next_token, int32_t* status_out,
                                   void* stream);
 
+/* Training-time forward, no backward (Sec. 4.1 "Training", Fig. 2(a); consistency loss of Sec. 4.3).
+ * To be called after kvp_prefill_predict for the same tokens / lengths / cache: the cache then holds
+ * the predicted K_hat_i, V_hat_i of the whole prompt.  Two passes of the base model over ALL prompt tokens:
+ *   (1) its ordinary forward, whose own keys (after RoPE) and values are the target cache KV_B:
+ *       l1_k[i] = mean over tokens and columns of |K_hat_i - K_B,i|, l1_v[i] likewise (dev fp32 [n_base_layers]);
+ *       the paper's L_C is their sum (lambda_C = 1) or mean (lambda_C = 1 / n_B) over i, K and V together;
+ *   (2) the forward in which every layer's attention reads the predicted cache instead of the layer's own
+ *       keys and values (query t sees predicted entries 0..t: "masked cross-attention"):
+ *       logits_out = dev fp32 [sum(lengths), vocab], row t = logits after token t (the input of the paper's
+ *       base loss L_B); may be NULL, then pass (2) is skipped.
+ * The predicted cache is read in the run dtype (bf16 entries in bf16 mode).  The cache and seq_lens are not
+ * changed.  workspace: dev, 256-byte aligned, >= kvp_train_workspace_bytes(batch, sum(lengths)) (its own
+ * layout: base-model widths for every token).  Launches kernel by kernel on `stream`, no synchronisation.
+ * Needs every base tensor including wk / wv.  Errors as kvp_prefill_predict. */
+kvp_status kvp_train_workspace_bytes(const kvp_handle* h, int32_t max_batch, int64_t max_total_tokens, size_t* bytes);
+kvp_status kvp_train_forward(kvp_handle* h, const int32_t* tokens /* dev [sum(lengths)] */, const int32_t* lengths /* host */,
+                             int32_t batch, const kvp_cache* cache, void* workspace, size_t workspace_bytes,
+                             float* logits_out, float* l1_k, float* l1_v, void* stream);
+
 /* Synchronises `stream`, reads the device status word of `workspace`, clears it and returns
  * KVP_OK, KVP_ERR_TIMEOUT, KVP_ERR_BAD_INDEX or KVP_ERR_CUDA. */
 kvp_status kvp_poll_status(kvp_handle* h, void* workspace, void* stream);

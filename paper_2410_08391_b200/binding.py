@@ -52,7 +52,7 @@ EXPORTS = ["kvp_create", "kvp_destroy", "kvp_last_error", "kvp_layer_map_canonic
            "kvp_layer_map_uniform", "kvp_packed_weight_bytes", "kvp_workspace_bytes", "kvp_cache_layout",
            "kvp_load_weights", "kvp_prefill_predict", "kvp_prefill_predict_host", "kvp_decode_step",
            "kvp_poll_status", "kvp_launch_count", "kvp_timing_enable", "kvp_timing_read",
-           "kvp_decode_step_static"]
+           "kvp_decode_step_static", "kvp_train_workspace_bytes", "kvp_train_forward"]
 
 CLASS_NAMES = ["aux_gemm", "aux_attn", "predictor", "step_gemv", "step_attn", "other", "step_fused"]
 
@@ -83,6 +83,8 @@ def lib() -> C.CDLL:
         L.kvp_prefill_predict_host.argtypes = [vp, vp, C.POINTER(i32), i32, C.POINTER(CacheC), vp, C.c_size_t, vp, vp, vp, vp]
         L.kvp_decode_step.argtypes = [vp, vp, C.POINTER(i32), i32, C.POINTER(CacheC), vp, C.c_size_t, vp, vp, vp]
         L.kvp_decode_step_static.argtypes = [vp, vp, C.POINTER(i32), i32, C.POINTER(CacheC), vp, vp, vp, vp]
+        L.kvp_train_workspace_bytes.argtypes = [vp, i32, i64, C.POINTER(C.c_size_t)]
+        L.kvp_train_forward.argtypes = [vp, vp, C.POINTER(i32), i32, C.POINTER(CacheC), vp, C.c_size_t, vp, vp, vp, vp]
         L.kvp_poll_status.argtypes = [vp, vp, vp]
         L.kvp_launch_count.argtypes = [vp]
         L.kvp_launch_count.restype = i64
@@ -235,6 +237,19 @@ def kvp_decode_step_static(h, tokens, lengths_host: Sequence[int], cache: "Cache
                                         status_out.data_ptr() if status_out is not None else None, stream), h)
 
 
+def kvp_train_workspace_bytes(h, max_batch: int, max_total_tokens: int) -> int:
+    n = C.c_size_t()
+    _check(lib().kvp_train_workspace_bytes(h, max_batch, max_total_tokens, C.byref(n)), h)
+    return n.value
+
+
+def kvp_train_forward(h, tokens, lengths: Sequence[int], cache: "Cache", workspace, logits_out, l1_k, l1_v, stream: int) -> None:
+    cc = _cache_c(cache)
+    _check(lib().kvp_train_forward(h, tokens.data_ptr(), _i32arr(lengths), len(lengths), C.byref(cc), workspace.data_ptr(),
+                                   workspace.numel(), logits_out.data_ptr() if logits_out is not None else None,
+                                   l1_k.data_ptr(), l1_v.data_ptr(), stream), h)
+
+
 def kvp_poll_status(h, workspace, stream: int) -> None:
     _check(lib().kvp_poll_status(h, workspace.data_ptr(), stream), h)
 
@@ -355,6 +370,23 @@ class Session:
         finally:
             self.leave(cur)
         return self.logits[:b], self.first[:b]
+
+    def train_forward(self, tokens_dev, lengths: Sequence[int], want_logits: bool = True):
+        """After prefill_predict on the same prompt: (logits [T, vocab] or None, l1_k [n_B], l1_v [n_B]) on the device."""
+        torch = self.torch
+        total = int(sum(lengths))
+        need = kvp_train_workspace_bytes(self.h, len(lengths), total)
+        if getattr(self, "train_ws", None) is None or self.train_ws.numel() < need:
+            self.train_ws = torch.empty(need, dtype=torch.uint8, device=self.device)
+        logits = torch.empty((total, self.pair.base.vocab), dtype=torch.float32, device=self.device) if want_logits else None
+        l1_k = torch.empty(self.pair.base.n_layers, dtype=torch.float32, device=self.device)
+        l1_v = torch.empty_like(l1_k)
+        cur = self.enter()
+        try:
+            kvp_train_forward(self.h, tokens_dev, lengths, self.cache, self.train_ws, logits, l1_k, l1_v, self.stream)
+        finally:
+            self.leave(cur)
+        return logits, l1_k, l1_v
 
     def poll(self):
         kvp_poll_status(self.h, self.workspace, self.stream)

@@ -148,6 +148,14 @@ void launch_gemm_simt(const LaunchCtx&, const GemmArgs&, int epi);
 void launch_attn_prefill_simt(const LaunchCtx&, const void* qkv, int ld, int nq, int nkv, int hd,
                               const int* cu_dev, int batch, int total, void* out, int ldo);
 
+// training-time forward: consistency terms and the predicted cache as a layer's keys and values.
+// qkv: one layer's projection buffer [T, ld], own keys at column k_col, values at k_col + nkv * hd; kv_lo (bf16 mode,
+// may be null): lo parts [T, ld_lo] of keys then values.  sum_k / sum_v (device) += mean |predicted - own|.
+void launch_kv_l1(const LaunchCtx&, const void* qkv, int ld, int k_col, const void* kv_lo, int ld_lo, int T_tokens, int nkv,
+                  int hd, const int* tok_slot, const void* kpool, const void* vpool, float* sum_k, float* sum_v);
+void launch_kv_take(const LaunchCtx&, void* qkv, int ld, int k_col, int T_tokens, int nkv, int hd, const int* tok_slot,
+                    const void* kpool, const void* vpool);
+
 // base single-token step
 enum StepGemvMode : int { GEMV_STORE = 0, GEMV_RESID = 1, GEMV_SWIGLU = 2 };
 void launch_step_gemv(const LaunchCtx&, const void* W, int ldw, int N, int K, const float* x, int ldx,

@@ -943,3 +943,174 @@ kvp_status kvp_poll_status(kvp_handle* h, void* workspace, void* stream) {
 }
 
 }  // extern "C"
+
+// ---- training-time forward (Sec. 4.1 "Training", Sec. 4.3) ------------------------------------------------
+namespace {
+struct TrainWs {
+  size_t status, cu, last_idx, tok_pos, tok_slot, rope_tab, x, h, h_lo, qkv, qkv32, kv_lo, attn, gu, act, attn_sched, total;
+};
+TrainWs train_ws_layout(const kvp_handle* h, int64_t Bm, int64_t Tm) {
+  TrainWs w;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  const ModelPlan& B = h->base;
+  const size_t es = h->es;
+  w.status = take(16384);
+  w.cu = take((Bm + 1) * 4);
+  w.last_idx = take(Bm * 4);
+  w.tok_pos = take(Tm * 4);
+  w.tok_slot = take(Tm * 4);
+  w.rope_tab = take(Tm * (size_t)(B.L[0].hd / 2) * 8);
+  w.x = take(Tm * B.d * 4);
+  w.h = take(Tm * B.d * es);
+  w.h_lo = take(Tm * B.d * es);
+  w.qkv = take(Tm * B.max_nqkv * es);
+  w.qkv32 = take(Tm * B.max_nqkv * 4);
+  w.kv_lo = take(Tm * 2 * (size_t)B.max_dkv * es);
+  w.attn = take(Tm * B.max_dq * es);
+  w.gu = take(Tm * 2 * (size_t)B.max_ffn * es);
+  w.act = take(Tm * (size_t)B.max_ffn * es);
+  w.attn_sched = take((size_t)(Tm / 128 + Bm + 1) * 8);
+  w.total = off;
+  return w;
+}
+}  // namespace
+
+extern "C" kvp_status kvp_train_workspace_bytes(const kvp_handle* h, int32_t max_batch, int64_t max_total_tokens, size_t* bytes) {
+  if (!h || !bytes || max_batch <= 0 || max_batch > KVP_MAX_BATCH || max_total_tokens < max_batch) return KVP_ERR_INVALID_ARG;
+  *bytes = train_ws_layout(h, max_batch, max_total_tokens).total;
+  return KVP_OK;
+}
+
+extern "C" kvp_status kvp_train_forward(kvp_handle* h, const int32_t* tokens, const int32_t* lengths, int32_t batch,
+                                        const kvp_cache* cache, void* workspace, size_t workspace_bytes, float* logits_out,
+                                        float* l1_k, float* l1_v, void* stream) {
+  CallShape cs;
+  kvp_status st = common_checks(h, lengths, batch, cache, workspace, 0, &cs);
+  if (st != KVP_OK) return st;
+  if (!tokens || !l1_k || !l1_v) return fail(h, KVP_ERR_INVALID_ARG, "NULL argument");
+  if (!h->ready_decode) return fail(h, KVP_ERR_NOT_LOADED, "kvp_load_weights has not supplied every required tensor");
+  const int T = cs.total, es = h->es;
+  TrainWs w = train_ws_layout(h, batch, T);
+  if (workspace_bytes < w.total) return fail(h, KVP_ERR_WORKSPACE, "workspace needs %zu bytes, got %zu", w.total, workspace_bytes);
+  char* ws = (char*)workspace;
+  cudaStream_t s = (cudaStream_t)stream;
+  int* status = (int*)(ws + w.status);
+  LaunchCtx ctx{s, &h->n_launch, status, h->opt.dtype};
+  const ModelPlan& B = h->base;
+  const char* P = h->packed;
+  cudaMemsetAsync(status, 0, MEGA_STATUS_BYTES, s);
+  cudaMemsetAsync(l1_k, 0, (size_t)B.n_layers * 4, s);
+  cudaMemsetAsync(l1_v, 0, (size_t)B.n_layers * 4, s);
+  int* cu_dev = (int*)(ws + w.cu);
+  int* tok_pos = (int*)(ws + w.tok_pos);
+  int* tok_slot = (int*)(ws + w.tok_slot);
+  float* x = (float*)(ws + w.x);
+  char* hbuf = ws + w.h;
+  char* qkv = ws + w.qkv;
+  const bool split = h->opt.dtype == KVP_BF16;
+  char* h_lo = split ? ws + w.h_lo : nullptr;
+  char* kv_lo = split ? ws + w.kv_lo : nullptr;
+  float* qkv32 = (float*)(ws + w.qkv32);
+  float2* rope_tab = (float2*)(ws + w.rope_tab);
+  char* attn = ws + w.attn;
+  char* gu = ws + w.gu;
+  char* act = ws + w.act;
+  int2* attn_sched = (int2*)(ws + w.attn_sched);
+  cudaError_t tc_err = cudaSuccess;
+  // token -> (sequence position, cache slot); seq_lens is rewritten with the same lengths the cache already holds
+  launch_build_index(ctx, cs.cu.data(), batch, T, cu_dev, tok_pos, tok_slot, (int*)(ws + w.last_idx), cache->block_table,
+                     cache->max_pages_per_seq, cache->n_pages, cache->seq_lens);
+  int max_nq = 1;
+  for (int i = 0; i < B.n_layers; ++i) max_nq = std::max(max_nq, B.L[i].nq);
+  const int attn_tiles = attn_tc_items(cs.cu.data(), batch, 2) * max_nq < h->n_sm ? 1 : 2;
+  const int attn_items = attn_tc_items(cs.cu.data(), batch, attn_tiles);
+  if (h->use_tc && h->opt.dtype == KVP_BF16 && (B.L[0].hd == 64 || B.L[0].hd == 128)) {
+    launch_rope_table(ctx, rope_tab, cs.max_len, B.L[0].hd, B.theta);
+    launch_attn_schedule(cu_dev, batch, attn_tiles, attn_sched, ctx.st, ctx.n_launch);
+  }
+  // pass 0: the base model's ordinary forward, for its own cache KV_B (consistency terms against the predicted one);
+  // pass 1: the forward whose attention reads the predicted cache, for the logits
+  for (int pass = 0; pass < 2; ++pass) {
+    if (pass == 1 && !logits_out) break;
+    launch_embed(ctx, tokens, nullptr, T, P + B.embed, B.vocab, B.d, x);
+    for (int i = 0; i < B.n_layers; ++i) {
+      const LayerPlan& L = B.L[i];
+      const bool last = pass == 0 && i == B.n_layers - 1;     // only this layer's keys and values are still needed
+      launch_rmsnorm(ctx, x, (const float*)(P + L.attn_norm), B.eps, T, B.d, hbuf, h->opt.dtype, h_lo);
+      const int col_begin = last ? L.dq : 0;
+      const int n_out = L.nqkv - col_begin, q_heads = last ? 0 : L.nq;
+      const float* qn = B.qk_norm ? (const float*)(P + L.q_norm) : nullptr;
+      const float* kn = B.qk_norm ? (const float*)(P + L.k_norm) : nullptr;
+      TcGemm tq{};
+      tq.A = (const bf16*)hbuf; tq.lda = B.d; tq.A2 = (const bf16*)h_lo; tq.lda2 = B.d; tq.split_begin = L.dq - col_begin;
+      tq.W = (const bf16*)(P + L.wqkv + (size_t)col_begin * B.d * es); tq.ldw = B.d; tq.M = T; tq.N = n_out; tq.K = B.d;
+      tq.epi = TC_QKV; tq.C = (bf16*)(qkv + (size_t)col_begin * es); tq.ldc = L.nqkv;
+      tq.C_lo = (bf16*)kv_lo; tq.ld_lo = 2 * L.dkv; tq.lo_col_begin = q_heads * L.hd;
+      tq.rot_cols = (q_heads + L.nkv) * L.hd; tq.hd = L.hd; tq.rope_tab = rope_tab; tq.tok_pos = tok_pos;
+      tq.q_gain = qn; tq.k_gain = kn; tq.q_cols = q_heads * L.hd; tq.eps = B.eps;
+      if (!try_tc(h, ctx, tq, KVP_CLASS_OTHER, &tc_err)) {
+        GemmArgs g{};
+        g.A = hbuf; g.lda = B.d; g.M = T; g.K = B.d; g.A2 = h_lo; g.lda2 = B.d; g.split_begin = L.dq - col_begin;
+        g.W = P + L.wqkv + (size_t)col_begin * B.d * es; g.ldw = B.d; g.N = n_out; g.C = qkv32; g.ldc = g.N;
+        launch_gemm_simt(ctx, g, EPI_STORE32);
+        launch_rope_split(ctx, qkv32, g.N, T, g.N / L.hd, q_heads + L.nkv, L.hd, tok_pos, B.theta, qkv + (size_t)col_begin * es,
+                          L.nqkv, kv_lo, 2 * L.dkv, q_heads, q_heads, qn, kn, B.eps);
+      }
+      if (pass == 0) {
+        launch_kv_l1(ctx, qkv, L.nqkv, L.dq, kv_lo, 2 * L.dkv, T, L.nkv, L.hd, tok_slot, cache->k_pools[i], cache->v_pools[i],
+                     l1_k + i, l1_v + i);
+        if (last) break;
+      } else {
+        launch_kv_take(ctx, qkv, L.nqkv, L.dq, T, L.nkv, L.hd, tok_slot, cache->k_pools[i], cache->v_pools[i]);
+      }
+      if (h->use_tc && split && attn_items <= 65535 && attn_tc_supported(L.hd, L.nqkv, qkv, L.dq, attn)) {
+        cudaError_t e = launch_attn_tc((const bf16*)qkv, L.nqkv, T, L.nq, L.nkv, L.hd, cu_dev, attn_sched, attn_items, attn_tiles,
+                                       (bf16*)attn, L.dq, ctx.status, ctx.st, ctx.n_launch);
+        if (e != cudaSuccess && tc_err == cudaSuccess) tc_err = e;
+      } else {
+        launch_attn_prefill_simt(ctx, qkv, L.nqkv, L.nq, L.nkv, L.hd, cu_dev, batch, T, attn, L.dq);
+      }
+      TcGemm to{};
+      to.A = (const bf16*)attn; to.lda = L.dq; to.W = (const bf16*)(P + L.wo); to.ldw = L.dq; to.M = T; to.N = B.d; to.K = L.dq;
+      to.epi = TC_RESID; to.X = x; to.ldx = B.d;
+      if (!try_tc(h, ctx, to, KVP_CLASS_OTHER, &tc_err)) {
+        GemmArgs o{};
+        o.A = attn; o.lda = L.dq; o.W = P + L.wo; o.ldw = L.dq; o.M = T; o.N = B.d; o.K = L.dq; o.X = x; o.ldx = B.d;
+        launch_gemm_simt(ctx, o, EPI_RESID);
+      }
+      launch_rmsnorm(ctx, x, (const float*)(P + L.ffn_norm), B.eps, T, B.d, hbuf, h->opt.dtype);
+      TcGemm tf{};
+      tf.A = (const bf16*)hbuf; tf.lda = B.d; tf.W = (const bf16*)(P + L.wgu); tf.ldw = B.d; tf.M = T; tf.N = 2 * L.ffn; tf.K = B.d;
+      tf.epi = TC_SWIGLU; tf.C = (bf16*)act; tf.ldc = L.ffn; tf.ffn = L.G == 64 ? L.ffn : 1;
+      if (!try_tc(h, ctx, tf, KVP_CLASS_OTHER, &tc_err)) {
+        GemmArgs f{};
+        f.A = hbuf; f.lda = B.d; f.W = P + L.wgu; f.ldw = B.d; f.M = T; f.N = 2 * L.ffn; f.K = B.d; f.C = gu; f.ldc = 2 * L.ffn;
+        launch_gemm_simt(ctx, f, EPI_STORE);
+        launch_swiglu(ctx, gu, T, L.ffn, L.G, act);
+      }
+      TcGemm td{};
+      td.A = (const bf16*)act; td.lda = L.ffn; td.W = (const bf16*)(P + L.wd); td.ldw = L.ffn; td.M = T; td.N = B.d; td.K = L.ffn;
+      td.epi = TC_RESID; td.X = x; td.ldx = B.d;
+      if (!try_tc(h, ctx, td, KVP_CLASS_OTHER, &tc_err)) {
+        GemmArgs d{};
+        d.A = act; d.lda = L.ffn; d.W = P + L.wd; d.ldw = L.ffn; d.M = T; d.N = B.d; d.K = L.ffn; d.X = x; d.ldx = B.d;
+        launch_gemm_simt(ctx, d, EPI_RESID);
+      }
+    }
+  }
+  if (logits_out) {      // logits of every position: final norm, LM head (accumulated onto zeros by the residual epilogue)
+    launch_rmsnorm(ctx, x, (const float*)(P + B.final_norm), B.eps, T, B.d, hbuf, h->opt.dtype);
+    cudaMemsetAsync(logits_out, 0, (size_t)T * B.vocab * 4, s);
+    TcGemm tl{};
+    tl.A = (const bf16*)hbuf; tl.lda = B.d; tl.W = (const bf16*)(P + B.lm_head); tl.ldw = B.d; tl.M = T; tl.N = B.vocab; tl.K = B.d;
+    tl.epi = TC_RESID; tl.X = logits_out; tl.ldx = B.vocab;
+    if (!try_tc(h, ctx, tl, KVP_CLASS_OTHER, &tc_err)) {
+      GemmArgs g{};
+      g.A = hbuf; g.lda = B.d; g.W = P + B.lm_head; g.ldw = B.d; g.M = T; g.N = B.vocab; g.K = B.d; g.X = logits_out; g.ldx = B.vocab;
+      launch_gemm_simt(ctx, g, EPI_RESID);
+    }
+  }
+  if (tc_err != cudaSuccess) return fail(h, KVP_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(tc_err));
+  return check_cuda(h, "kvp_train_forward");
+}

@@ -166,6 +166,56 @@ def test_recorded_decode_step_replays_for_later_positions(lens):
         s.close()
 
 
+TRAIN_CASES = [
+    ("c1", None, "fanin"),                       # fp32, CUDA-core kernels
+    ("t_small_f32", [129, 40, 1], "fanin"),
+    ("t_small", [150, 37, 1, 64, 65], "fanin"),  # bf16, tensor-core GEMMs and attention, ragged
+    ("t_small", [300], "n002"),
+    ("t_hd128", [130, 70, 2], "fanin"),
+    ("t_scaled", [100, 33, 257], "fanin"),       # heterogeneous layers
+    ("t_small_qkn", [129, 40], "fanin"),         # query / key norm
+]
+
+
+@pytest.mark.parametrize("name,lens,regime", TRAIN_CASES, ids=lambda v: str(v).replace(" ", ""))
+def test_train_forward_matches_oracle(name, lens, regime):
+    """Training-time forward (Sec. 4.1): logits of every position from the base model on the predicted cache, and
+    the consistency terms mean |KV_hat - KV_B| per base layer (Sec. 4.3), against the oracle."""
+    import torch
+    pair = wl.pair(name)
+    W = wl.make_weights(pair, seed=6, regime=regime)
+    pr = wl.prompts(name, seed=6) if lens is None else wl.custom_prompts(pair.base.vocab, lens, seed=6)
+    lens = [int(x) for x in pr.lengths]
+    s = make_session(pair, W, pr)
+    tol = TOL[pair.dtype]
+    try:
+        toks = torch.from_numpy(pr.tokens).to(s.device)
+        s.prefill_predict(toks, lens)
+        logits, l1_k, l1_v = s.train_forward(toks, lens)
+        s.poll()
+        logits, l1_k, l1_v = logits.cpu().numpy(), l1_k.cpu().numpy(), l1_v.cpu().numpy()
+        assert s.cache.seq_lens[:pr.batch].cpu().tolist() == lens
+        nb = pair.base.n_layers
+        abs_k, abs_v, cnt = np.zeros(nb), np.zeros(nb), np.zeros(nb)
+        t0 = 0
+        for b in range(pr.batch):
+            ref_logits, ak, av, n = orc.train_forward(pair, W, pr.seq(b))
+            abs_k += ak; abs_v += av; cnt += n
+            got = logits[t0:t0 + lens[b]]
+            assert rel_fro(got, ref_logits) <= tol, f"seq {b}: logits {rel_fro(got, ref_logits):.3e}"
+            # the last row is the inference path's first step (also checked there); every row must hold on its own
+            worst = max(rel_fro(got[t], ref_logits[t]) for t in range(lens[b]))
+            assert worst <= 2 * tol, f"seq {b}: worst row {worst:.3e}"
+            t0 += lens[b]
+        # the predicted cache is rounded to the run dtype before it is compared: one bf16 rounding of O(1) entries
+        slack = 4e-3 if pair.dtype == "bf16" else 1e-5
+        for i in range(nb):
+            for got, ref in ((l1_k[i], abs_k[i] / cnt[i]), (l1_v[i], abs_v[i] / cnt[i])):
+                assert abs(got - ref) <= slack * max(ref, 1e-3) + 1e-6, f"layer {i}: {got} vs {ref}"
+    finally:
+        s.close()
+
+
 def test_sequence_alone_equals_sequence_in_batch():
     import torch
     pair = wl.pair("t_small")
