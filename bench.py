@@ -153,6 +153,8 @@ def main():
     ap.add_argument("--workload", default="c2", choices=["c1", "c2", "c3", "c4", "c5", "qa", "lp75", "lp50", "lp25"])
     ap.add_argument("--impl", default="kvp", choices=["kvp", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--train-forward", action="store_true",
+                    help="also time the training-time forward (base model over the whole prompt on the predicted cache)")
     ap.add_argument("--decode-steps", type=int, default=16, help="generation steps timed after the TTFT measurement (0 = none)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "kvp" else args.warmup
@@ -278,6 +280,29 @@ def main():
         gms = max_over_ranks(g0.elapsed_time(g1) / args.decode_steps, dist, dev)
         decode.update({"graph_ms_per_step": gms, "graph_tok_per_s": world * pr.batch / (gms * 1e-3)})
 
+    # ---- training-time forward (Sec. 4.1 "Training"): secondary figure, on request ----
+    train = None
+    if args.train_forward:
+        step()
+        for _ in range(2):
+            sess.train_forward(toks, lens)
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        n_tf = max(3, min(args.steps, 10))
+        t0.record(stream)
+        for _ in range(n_tf):
+            sess.train_forward(toks, lens)
+        t1.record(stream)
+        torch.cuda.synchronize()
+        sess.poll()
+        tms = max_over_ranks(t0.elapsed_time(t1) / n_tf, dist, dev)
+        tf = wl.train_forward_flops(pair, lens)
+        pk = measured_peaks()
+        pk_tf = (pk["bf16_tflops_sustained"] or pk["bf16_tflops"]) / (16.0 if pair.dtype == "f32" else 1.0)
+        train = {"ms": tms, "tok_per_s": world * work["tokens"] / (tms * 1e-3), "tflops": tf / (tms * 1e-3) / 1e12,
+                 "algorithmic_tflop": tf / 1e12, "frac_of_tensor_peak": tf / (tms * 1e-3) / 1e12 / pk_tf,
+                 "peak": pk_tf, "peak_source": pk["source"]}
+
     # ---- per-kernel-class device times (separate pass: events around every launch) ----
     kvp.kvp_timing_enable(sess.h, True)
     for _ in range(args.steps):
@@ -335,6 +360,7 @@ def main():
         "roofline": roofline,
         "tensor_frac_stage12": tensor_frac,
         "decode": decode,
+        "train_forward": train,
         "clocks": clocks,
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

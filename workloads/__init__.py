@@ -404,3 +404,20 @@ def algorithmic_work(p: PairCfg, lengths: Sequence[int]) -> Dict[str, float]:
                 tensor_flops=gemm + attn + pred, cache_bytes=cache_bytes,
                 step_weight_bytes=step_w, step_bytes=step_w + cache_bytes,
                 step_flops=step_flops)
+
+
+def train_forward_flops(p: PairCfg, lengths: Sequence[int]) -> float:
+    """FLOPs of the training-time forward after the predicted cache exists: the base model's ordinary forward up to
+    the last layer's K/V projection (the target cache), and its forward on the predicted cache with the LM head
+    over every position; causal attention counts L(L+1)/2 pairs."""
+    lens = [int(x) for x in lengths]
+    T = sum(lens)
+    pairs = sum(l * (l + 1) // 2 for l in lens)
+    d = p.base.d_model
+    f = 0.0
+    n = p.base.n_layers
+    for i, lc in enumerate(p.base.layers):
+        full = 2.0 * T * (d * (lc.d_q + 2 * lc.d_kv) + lc.d_q * d + 3 * d * lc.ffn_dim) + 4.0 * lc.d_q * pairs
+        f += full                                             # forward on the predicted cache
+        f += full if i < n - 1 else 2.0 * T * d * 2 * lc.d_kv   # ordinary forward
+    return f + 2.0 * T * d * p.base.vocab
