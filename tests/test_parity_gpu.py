@@ -301,10 +301,23 @@ def test_error_paths_report_status_and_keep_the_context_usable():
         s.cache.block_table.copy_(keep)
         s.prefill_predict(toks, lens)                              # and the handle still works afterwards
         s.poll()
+        # training-time forward: same argument checks; without a logits buffer only the consistency terms are computed
+        l1 = torch.empty(pair.base.n_layers, dtype=torch.float32, device=s.device)
+        with pytest.raises(kvp.KvpError) as e:
+            kvp.kvp_train_forward(s.h, toks, lens, s.cache, small, None, l1, l1.clone(), s.stream)
+        assert e.value.status == -8
+        _, k_only, v_only = s.train_forward(toks, lens, want_logits=False)
+        _, k_both, v_both = s.train_forward(toks, lens, want_logits=True)
+        s.poll()
+        assert torch.allclose(k_only, k_both, rtol=1e-3) and torch.allclose(v_only, v_both, rtol=1e-3)   # fp32 atomic sums: order varies
+        assert bool((k_only > 0).all()) and bool((v_only > 0).all())
         h2 = kvp.kvp_create(pair.aux, pair.base, pair.layer_map, pair.dtype)
         with pytest.raises(kvp.KvpError) as e:
             kvp.kvp_prefill_predict(h2, toks, lens, s.cache, s.workspace, s.logits, s.first, s.stream)
         assert e.value.status == -4
+        with pytest.raises(kvp.KvpError) as e:
+            kvp.kvp_train_forward(h2, toks, lens, s.cache, s.workspace, None, l1, l1.clone(), s.stream)
+        assert e.value.status in (-4, -8)
         kvp.kvp_destroy(h2)
     finally:
         s.close()
