@@ -172,6 +172,7 @@ void launch_argmax(const LaunchCtx&, const float* logits, int batch, int vocab, 
 void launch_add_int(const LaunchCtx&, int* v, int n, int delta);
 int step_attn_splits(int batch, int nkv, int max_keys);
 // bandwidth-bound variant for the bf16 cache (pages fetched with bulk asynchronous copies)
+int step_attn_ring_splits(int nq, int nkv, int hd, int batch, int max_keys, int upper);
 bool step_attn_ring_supported(int dtype, int nq, int nkv, int hd, const void* kpool, const void* vpool);
 cudaError_t launch_step_attn_ring(const LaunchCtx&, const float* q, int ldq, int nq, int nkv, int hd, float theta,
                                   const void* kpool, const void* vpool, const int* block_table, int max_pages_per_seq,

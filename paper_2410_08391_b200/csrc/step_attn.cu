@@ -1,15 +1,24 @@
-// Single-query GQA attention of the base step over the paged bf16 cache, bandwidth-bound variant.
+// Single-query GQA attention of the base step over the paged bf16 cache, bandwidth-bound variants.
 //
-// grid (key-range split, kv head, sequence); a CTA of 64 * group threads serves the `group` query
-// heads that share one kv head and walks its range of cache pages.  A page of one kv head is one
-// contiguous block (64 keys x head_dim), so K and V pages are fetched whole with bulk asynchronous
-// copies into a ring of shared-memory stages, several pages ahead of the arithmetic: the HBM
-// latency is covered by copies in flight, not by resident warps.
-//   scores   thread = (key, head): dot product of the key's row with the head's query; the row's
-//            16-byte pieces are visited in an order rotated by the key index, which keeps the
-//            row-per-thread reads free of bank conflicts without padding the copied page
+// grid (key-range split, kv head, sequence); a CTA serves the `group` query heads that share one
+// kv head and walks its range of cache pages.  A page of one kv head is one contiguous block
+// (64 keys x head_dim), so K and V pages are fetched whole with bulk asynchronous copies into a
+// ring of shared-memory stages, several pages ahead of the arithmetic: the HBM latency is covered
+// by copies in flight, not by resident warps.
+//
+// step_attn_ring_wide_kernel (up to 4 query heads per kv head): every cached element is read from
+// shared memory ONCE and used for all heads of the group, because the shared-memory port, not
+// HBM, bounds a kernel that re-reads a page per head.
+//   scores   DS lanes share a key: each holds its slice of the group's queries in registers for
+//            the whole kernel, reads its 16-byte pieces of the key row (pieces interleaved over
+//            the lanes and visited in an order rotated by the key index: conflict-free), and the
+//            DS partial dot products per head are added with shuffles
 //   softmax  one warp per head over the page's 64 scores, running max / sum in shared memory
-//   values   thread = (head, pair of dims): sum over the page's keys
+//   values   thread = (pair of dims, block of keys): one 4-byte read of V and one broadcast read
+//            of the key's probabilities feed 2 x group multiply-adds; the key blocks are summed
+//            through shared memory once, after the last page
+// step_attn_ring_wide_kernel (5 to 8 heads per kv head): thread = (key, head) for the scores and
+// (pair of dims, head) for the values.
 // With more than one split, partial (o, m, l) per (sequence, q head, split) go to `part`.
 // The wait on a page's copies is bounded; on expiry the CTA flags DEV_TIMEOUT and leaves.
 #include <math.h>
@@ -44,7 +53,7 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
 }
 
 template <int HD>
-__global__ void __launch_bounds__(512) step_attn_ring_kernel(const float* __restrict__ q, int ldq, int nq, int nkv,
+__global__ void __launch_bounds__(512) step_attn_ring_wide_kernel(const float* __restrict__ q, int ldq, int nq, int nkv,
                                                              const __grid_constant__ InvFreq inv,
                                                              const bf16* __restrict__ kpool, const bf16* __restrict__ vpool,
                                                              const int* __restrict__ block_table, int mpps, int n_pages,
@@ -229,6 +238,263 @@ __global__ void __launch_bounds__(512) step_attn_ring_kernel(const float* __rest
   }
 }
 
+// ---- up to 4 query heads per kv head -------------------------------------------------------
+template <int HD, int GP>
+struct RingCfg {
+  static constexpr int DS = (HD * GP > 256) ? 8 : 4;       // lanes that share one key's dot products
+  static constexpr int NT = PAGE_TOKENS * DS;              // threads per CTA
+  static constexpr int CH = HD / 8;                        // 16-byte pieces per key row
+  static constexpr int CPT = CH / DS;                      // pieces per lane
+  static constexpr int NKQ = NT / (HD / 2);                // key blocks of the value sum
+  static constexpr int KPT = PAGE_TOKENS / NKQ;            // keys per block
+  static constexpr int PAGE_BYTES = PAGE_TOKENS * HD * 2;  // one K or V page of one kv head
+  // pages in flight: one 512-thread CTA per SM keeps 5 pages ahead, two 256-thread CTAs 2 or 4 each
+  static constexpr int STAGES = NT == 512 ? 6 : (HD == 64 ? 5 : 3);
+  static constexpr size_t SMEM = (size_t)STAGES * 2 * PAGE_BYTES + (size_t)(GP * HD + PAGE_TOKENS * GP + 3 * GP) * sizeof(float);
+};
+
+template <int HD, int GP>
+__global__ void __launch_bounds__(RingCfg<HD, GP>::NT, RingCfg<HD, GP>::NT == 512 ? 1 : 2)
+step_attn_ring_kernel(const float* __restrict__ q, int ldq, int nq, int nkv, const __grid_constant__ InvFreq inv,
+                      const bf16* __restrict__ kpool, const bf16* __restrict__ vpool, const int* __restrict__ block_table,
+                      int mpps, int n_pages, const int* __restrict__ seq_lens, int extra, int n_split,
+                      float* __restrict__ part, float* __restrict__ out, int* status, const float* __restrict__ q_gain,
+                      float eps) {
+  using Cfg = RingCfg<HD, GP>;
+  constexpr int DS = Cfg::DS, NT = Cfg::NT, CPT = Cfg::CPT, NKQ = Cfg::NKQ, KPT = Cfg::KPT, STG = Cfg::STAGES;
+  constexpr int PAGE_BYTES = Cfg::PAGE_BYTES;
+  extern __shared__ __align__(128) unsigned char sm_raw[];
+  unsigned char* ring = sm_raw;                                                  // [STG][K page | V page]
+  float* qs = reinterpret_cast<float*>(sm_raw + STG * 2 * PAGE_BYTES);           // [GP][HD], scaled, after RoPE
+  float* ps = qs + GP * HD;                                                      // [64 keys][GP]
+  float* m_run = ps + PAGE_TOKENS * GP;
+  float* l_run = m_run + GP;
+  float* alpha = l_run + GP;
+  __shared__ __align__(8) unsigned long long bars[STG];
+  __shared__ int s_ok;
+  __shared__ float rq[MAXG];
+  const int group = nq / nkv;                      // <= GP
+  const int sp = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int n_keys = seq_lens[b] + extra;
+  const int pos = n_keys - 1;
+  const int n_pg = (n_keys + PAGE_TOKENS - 1) / PAGE_TOKENS;
+  const int per = (n_pg + n_split - 1) / n_split;
+  const int pg0 = sp * per, pg1 = min(n_pg, pg0 + per);
+  const int n_it = max(pg1 - pg0, 0);
+
+  auto issue = [&](int it) {     // thread 0: start the copies of page pg0 + it into slot it % STG
+    const int pg = pg0 + it;
+    int page = pg < mpps ? block_table[(size_t)b * mpps + pg] : -1;
+    const uint32_t bar = smem_u32(&bars[it % STG]);
+    if (page < 0 || page >= n_pages) {   // never dereferenced: the slot completes empty and the page is skipped below
+      dev_flag(status, DEV_BAD_PAGE);
+      asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+      return;
+    }
+    const size_t off = ((size_t)page * nkv + kvh) * PAGE_TOKENS * HD;
+    const uint32_t dst = smem_u32(ring + (size_t)(it % STG) * 2 * PAGE_BYTES);
+    mbar_expect_tx(bar, 2 * PAGE_BYTES);
+    bulk_load(dst, kpool + off, PAGE_BYTES, bar);
+    bulk_load(dst + PAGE_BYTES, vpool + off, PAGE_BYTES, bar);
+  };
+
+  if (tid == 0) {
+    for (int s = 0; s < STG; ++s) mbar_init(smem_u32(&bars[s]), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    s_ok = 1;
+    for (int it = 0; it < min(STG - 1, n_it); ++it) issue(it);
+  }
+  // queries of the group: (query norm,) RoPE at the last position, scaled by 1/sqrt(hd); heads beyond the group are zero
+  if (q_gain) head_rnorm(q + (size_t)b * ldq + (size_t)kvh * group * HD, group, HD, eps, rq);
+  {
+    const float scale = rsqrtf((float)HD);
+    constexpr int half = HD / 2;
+    for (int i = tid; i < GP * half; i += NT) {
+      const int h = i / half, c = i - h * half;
+      float r1 = 0.f, r2 = 0.f;
+      if (h < group) {
+        const float* qh = q + (size_t)b * ldq + (size_t)(kvh * group + h) * HD;
+        float sn, cs;
+        rope_sincos(pos, inv.f[c], &sn, &cs);
+        float x1 = qh[c], x2 = qh[c + half];
+        if (q_gain) { x1 *= rq[h] * q_gain[c]; x2 *= rq[h] * q_gain[c + half]; }
+        r1 = (x1 * cs - x2 * sn) * scale;
+        r2 = (x2 * cs + x1 * sn) * scale;
+      }
+      qs[h * HD + c] = r1;
+      qs[h * HD + c + half] = r2;
+    }
+    if (tid < GP) { m_run[tid] = -INFINITY; l_run[tid] = 0.f; alpha[tid] = 1.f; }
+  }
+  __syncthreads();
+  // scores: lane dq of key `key` visits pieces dq + DS * ((i + key) % CPT), i = 0 .. CPT-1; its queries for
+  // exactly those pieces stay in registers, in visiting order
+  const int key = tid / DS, dq = tid % DS;
+  float qr[GP][CPT][8];
+#pragma unroll
+  for (int i = 0; i < CPT; ++i) {
+    const int c = dq + DS * ((i + key) % CPT);
+#pragma unroll
+    for (int g = 0; g < GP; ++g) {
+      const float4 a = *reinterpret_cast<const float4*>(qs + g * HD + c * 8), bq = *reinterpret_cast<const float4*>(qs + g * HD + c * 8 + 4);
+      qr[g][i][0] = a.x; qr[g][i][1] = a.y; qr[g][i][2] = a.z; qr[g][i][3] = a.w;
+      qr[g][i][4] = bq.x; qr[g][i][5] = bq.y; qr[g][i][6] = bq.z; qr[g][i][7] = bq.w;
+    }
+  }
+  // values: thread = (pair of dims d2, key block kq)
+  const int d2 = tid % (HD / 2), kq = tid / (HD / 2);
+  float acc[GP][2];
+#pragma unroll
+  for (int g = 0; g < GP; ++g) { acc[g][0] = 0.f; acc[g][1] = 0.f; }
+  bool ok = true;
+  for (int it = 0; it < n_it; ++it) {
+    __syncthreads();                              // slot (it - 1) % STG and ps are free again
+    if (tid == 0 && it + STG - 1 < n_it) issue(it + STG - 1);
+    {                                             // wait for this page's copies (every thread polls; bounded)
+      const uint32_t bar = smem_u32(&bars[it % STG]), parity = (it / STG) & 1;
+      bool got = false;
+      for (uint32_t spin = 0; spin < SPIN_LIMIT; ++spin) {
+        if (mbar_test(bar, parity)) { got = true; break; }
+        if ((spin & 1023u) == 1023u && *(volatile int*)&s_ok == 0) break;
+      }
+      if (!got) { s_ok = 0; dev_flag(status, DEV_TIMEOUT); }
+    }
+    ok = __syncthreads_and(*(volatile int*)&s_ok != 0);
+    if (!ok) break;
+    const int pg = pg0 + it;
+    const int page = pg < mpps ? block_table[(size_t)b * mpps + pg] : -1;
+    const int nk = (page >= 0 && page < n_pages) ? min(PAGE_TOKENS, n_keys - pg * PAGE_TOKENS) : 0;
+    const unsigned char* Ks = ring + (size_t)(it % STG) * 2 * PAGE_BYTES;
+    const unsigned char* Vs = Ks + PAGE_BYTES;
+    // ---- scores
+    {
+      float s[GP];
+#pragma unroll
+      for (int g = 0; g < GP; ++g) s[g] = 0.f;
+      const unsigned char* kr = Ks + key * (HD * 2);
+#pragma unroll
+      for (int i = 0; i < CPT; ++i) {
+        const int c = dq + DS * ((i + key) % CPT);
+        const uint4 u = *reinterpret_cast<const uint4*>(kr + c * 16);
+        const float k0 = __uint_as_float(u.x << 16), k1 = __uint_as_float(u.x & 0xffff0000u);
+        const float k2 = __uint_as_float(u.y << 16), k3 = __uint_as_float(u.y & 0xffff0000u);
+        const float k4 = __uint_as_float(u.z << 16), k5 = __uint_as_float(u.z & 0xffff0000u);
+        const float k6 = __uint_as_float(u.w << 16), k7 = __uint_as_float(u.w & 0xffff0000u);
+#pragma unroll
+        for (int g = 0; g < GP; ++g) {
+          float t0 = fmaf(k0, qr[g][i][0], s[g]), t1 = k1 * qr[g][i][1];
+          t0 = fmaf(k2, qr[g][i][2], t0); t1 = fmaf(k3, qr[g][i][3], t1);
+          t0 = fmaf(k4, qr[g][i][4], t0); t1 = fmaf(k5, qr[g][i][5], t1);
+          t0 = fmaf(k6, qr[g][i][6], t0); t1 = fmaf(k7, qr[g][i][7], t1);
+          s[g] = t0 + t1;
+        }
+      }
+      float mine = 0.f;                            // lane dq < GP keeps head dq's sum
+#pragma unroll
+      for (int g = 0; g < GP; ++g) {
+#pragma unroll
+        for (int off = 1; off < DS; off <<= 1) s[g] += __shfl_xor_sync(0xffffffffu, s[g], off);
+        if (dq == g) mine = s[g];
+      }
+      if (dq < GP) ps[key * GP + dq] = key < nk ? mine : -INFINITY;
+    }
+    __syncthreads();
+    // ---- running softmax statistics, one warp per head
+    if (warp < GP) {
+      const int hh = warp;
+      const float s0 = ps[lane * GP + hh], s1 = ps[(32 + lane) * GP + hh];
+      const float mt = warp_max(fmaxf(s0, s1));
+      const float m_old = m_run[hh];
+      const float mn = fmaxf(m_old, mt);
+      const float p0 = (mn == -INFINITY) ? 0.f : __expf(s0 - mn), p1 = (mn == -INFINITY) ? 0.f : __expf(s1 - mn);
+      const float sum = warp_sum(p0 + p1);
+      ps[lane * GP + hh] = p0; ps[(32 + lane) * GP + hh] = p1;
+      if (lane == 0) {
+        const float a = (mn == -INFINITY) ? 1.f : __expf(m_old - mn);
+        alpha[hh] = a; m_run[hh] = mn; l_run[hh] = l_run[hh] * a + sum;
+      }
+    }
+    __syncthreads();
+    // ---- values: keys beyond nk carry p = 0 but their rows are not initialised memory: they are not read
+    {
+#pragma unroll
+      for (int g = 0; g < GP; ++g) { const float a = alpha[g]; acc[g][0] *= a; acc[g][1] *= a; }
+      const uint32_t* vr = reinterpret_cast<const uint32_t*>(Vs) + d2;
+      const int s1 = min(nk, (kq + 1) * KPT);
+#pragma unroll 4
+      for (int s = kq * KPT; s < s1; ++s) {
+        const uint32_t u = vr[s * (HD / 2)];
+        const float v0 = __uint_as_float(u << 16), v1 = __uint_as_float(u & 0xffff0000u);
+        float pv[4];
+        if constexpr (GP == 4) {
+          const float4 t = *reinterpret_cast<const float4*>(ps + s * 4);
+          pv[0] = t.x; pv[1] = t.y; pv[2] = t.z; pv[3] = t.w;
+        } else if constexpr (GP == 2) {
+          const float2 t = *reinterpret_cast<const float2*>(ps + s * 2);
+          pv[0] = t.x; pv[1] = t.y;
+        } else {
+          pv[0] = ps[s];
+        }
+#pragma unroll
+        for (int g = 0; g < GP; ++g) { acc[g][0] = fmaf(pv[g], v0, acc[g][0]); acc[g][1] = fmaf(pv[g], v1, acc[g][1]); }
+      }
+    }
+  }
+  if (!ok) {      // copies may still be landing in this CTA's shared memory
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+    return;
+  }
+  __syncthreads();
+  // the key blocks' sums meet in shared memory (the ring is idle: every copy issued was waited for)
+  float* red = reinterpret_cast<float*>(ring);                                   // [NKQ][GP][HD]
+#pragma unroll
+  for (int g = 0; g < GP; ++g)
+    *reinterpret_cast<float2*>(red + ((size_t)(kq * GP + g) * HD + 2 * d2)) = make_float2(acc[g][0], acc[g][1]);
+  __syncthreads();
+  const int ldr = HD + 2;
+  for (int o = tid; o < group * HD; o += NT) {
+    const int g = o / HD, d = o - g * HD;
+    float v = 0.f;
+#pragma unroll
+    for (int k = 0; k < NKQ; ++k) v += red[(size_t)(k * GP + g) * HD + d];
+    const int qh = kvh * group + g;
+    if (n_split == 1) out[(size_t)b * nq * HD + (size_t)qh * HD + d] = v / l_run[g];
+    else part[(((size_t)b * nq + qh) * n_split + sp) * ldr + d] = v;
+  }
+  if (n_split > 1 && tid < group) {
+    float* pr = part + (((size_t)b * nq + kvh * group + tid) * n_split + sp) * ldr;
+    pr[HD] = m_run[tid]; pr[HD + 1] = l_run[tid];
+  }
+}
+
+template <int HD, int GP>
+cudaError_t go_ring(dim3 grid, cudaStream_t st, const float* q, int ldq, int nq, int nkv, const InvFreq& inv, const bf16* kpool,
+                    const bf16* vpool, const int* block_table, int mpps, int n_pages, const int* seq_lens, int extra, int n_split,
+                    float* part, float* out, int* status, const float* q_gain, float eps) {
+  using Cfg = RingCfg<HD, GP>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(step_attn_ring_kernel<HD, GP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::SMEM);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  step_attn_ring_kernel<HD, GP><<<grid, Cfg::NT, Cfg::SMEM, st>>>(q, ldq, nq, nkv, inv, kpool, vpool, block_table, mpps, n_pages, seq_lens,
+                                                                  extra, n_split, part, out, status, q_gain, eps);
+  return cudaGetLastError();
+}
+
+template <int HD>
+cudaError_t go_ring_hd(int group, dim3 grid, cudaStream_t st, const float* q, int ldq, int nq, int nkv, const InvFreq& inv,
+                       const bf16* kpool, const bf16* vpool, const int* block_table, int mpps, int n_pages, const int* seq_lens,
+                       int extra, int n_split, float* part, float* out, int* status, const float* q_gain, float eps) {
+  if (group == 1)
+    return go_ring<HD, 1>(grid, st, q, ldq, nq, nkv, inv, kpool, vpool, block_table, mpps, n_pages, seq_lens, extra, n_split, part, out, status, q_gain, eps);
+  if (group == 2)
+    return go_ring<HD, 2>(grid, st, q, ldq, nq, nkv, inv, kpool, vpool, block_table, mpps, n_pages, seq_lens, extra, n_split, part, out, status, q_gain, eps);
+  return go_ring<HD, 4>(grid, st, q, ldq, nq, nkv, inv, kpool, vpool, block_table, mpps, n_pages, seq_lens, extra, n_split, part, out, status, q_gain, eps);
+}
+
 template <int HD>
 cudaError_t go(dim3 grid, int threads, cudaStream_t st, const float* q, int ldq, int nq, int nkv, const InvFreq& inv, const bf16* kpool,
                const bf16* vpool, const int* block_table, int mpps, int n_pages, const int* seq_lens, int extra, int n_split,
@@ -236,16 +502,35 @@ cudaError_t go(dim3 grid, int threads, cudaStream_t st, const float* q, int ldq,
   const size_t smem = (size_t)ST * 2 * PAGE_TOKENS * HD * 2 + (size_t)(MAXG * HD + MAXG * PAGE_TOKENS + 3 * MAXG) * sizeof(float);
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(step_attn_ring_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(step_attn_ring_wide_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  step_attn_ring_kernel<HD><<<grid, threads, smem, st>>>(q, ldq, nq, nkv, inv, kpool, vpool, block_table, mpps, n_pages, seq_lens, extra,
+  step_attn_ring_wide_kernel<HD><<<grid, threads, smem, st>>>(q, ldq, nq, nkv, inv, kpool, vpool, block_table, mpps, n_pages, seq_lens, extra,
                                                          n_split, part, out, status, q_gain, eps);
   return cudaGetLastError();
 }
 
 }  // namespace
+
+// Key-range splits for the ring kernels: at most `upper` (what the partial-result buffer was sized
+// for), chosen so that the CTAs fill whole waves of the SMs' resident slots: the cost of a launch is
+// waves x (pages per split + about two pages' worth of start-up).
+int step_attn_ring_splits(int nq, int nkv, int hd, int batch, int max_keys, int upper) {
+  const int group = nq / nkv;
+  int per_sm = 2;
+  if (group > 4) per_sm = 2;
+  else if (hd == 128 && group > 2) per_sm = 1;         // the 512-thread configuration
+  const int slots = 148 * per_sm, items = batch * nkv;
+  const int n_pg = (max_keys + PAGE_TOKENS - 1) / PAGE_TOKENS;
+  int best = 1; long long best_cost = -1;
+  for (int n = 1; n <= upper; ++n) {
+    const long long waves = ((long long)items * n + slots - 1) / slots;
+    const long long cost = waves * ((n_pg + n - 1) / n + 2);
+    if (best_cost < 0 || cost < best_cost) { best = n; best_cost = cost; }
+  }
+  return best;
+}
 
 bool step_attn_ring_supported(int dtype, int nq, int nkv, int hd, const void* kpool, const void* vpool) {
   const int group = nq / nkv;
@@ -260,6 +545,14 @@ cudaError_t launch_step_attn_ring(const LaunchCtx& ctx, const float* q, int ldq,
   dim3 grid(n_split, nkv, batch);
   const int threads = 64 * (nq / nkv);
   ++*ctx.n_launch;
+  const int group = nq / nkv;
+  if (group <= 4) {
+    if (hd == 64)
+      return go_ring_hd<64>(group, grid, ctx.st, q, ldq, nq, nkv, inv, (const bf16*)kpool, (const bf16*)vpool, block_table, mpps, n_pages,
+                            seq_lens, extra, n_split, part, out, ctx.status, q_gain, eps);
+    return go_ring_hd<128>(group, grid, ctx.st, q, ldq, nq, nkv, inv, (const bf16*)kpool, (const bf16*)vpool, block_table, mpps, n_pages,
+                           seq_lens, extra, n_split, part, out, ctx.status, q_gain, eps);
+  }
   if (hd == 64)
     return go<64>(grid, threads, ctx.st, q, ldq, nq, nkv, inv, (const bf16*)kpool, (const bf16*)vpool, block_table, mpps, n_pages, seq_lens,
                   extra, n_split, part, out, ctx.status, q_gain, eps);

@@ -599,6 +599,7 @@ void launch_step_attn(const LaunchCtx& ctx, const float* q, int ldq, int nq, int
   int n_split = step_attn_splits(batch, nkv, max_keys);
   dim3 grid(n_split, nkv, batch);
   if (step_attn_ring_supported(ctx.dtype, nq, nkv, hd, kpool, vpool)) {
+    n_split = step_attn_ring_splits(nq, nkv, hd, batch, max_keys, n_split);
     launch_step_attn_ring(ctx, q, ldq, nq, nkv, hd, theta, kpool, vpool, block_table, mpps, n_pages, seq_lens, extra, batch, n_split, part, out, q_gain, eps);
     if (n_split > 1) {
       ++*ctx.n_launch;
