@@ -29,6 +29,7 @@ namespace {
 
 constexpr int ST = 3;                       // pages in flight per CTA (K and V each)
 constexpr int MAXG = 8;
+constexpr int MAX_IDS = 512;                // page ids a CTA keeps in shared memory
 constexpr uint32_t SPIN_LIMIT = 20u * 1000u * 1000u;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -250,7 +251,7 @@ struct RingCfg {
   static constexpr int PAGE_BYTES = PAGE_TOKENS * HD * 2;  // one K or V page of one kv head
   // pages in flight: one 512-thread CTA per SM keeps 5 pages ahead, two 256-thread CTAs 2 or 4 each
   static constexpr int STAGES = NT == 512 ? 6 : (HD == 64 ? 5 : 3);
-  static constexpr size_t SMEM = (size_t)STAGES * 2 * PAGE_BYTES + (size_t)(GP * HD + PAGE_TOKENS * GP + 3 * GP) * sizeof(float);
+  static constexpr size_t SMEM = (size_t)STAGES * 2 * PAGE_BYTES + (size_t)(GP * HD + 2 * PAGE_TOKENS * GP + 3 * GP) * sizeof(float);
 };
 
 template <int HD, int GP>
@@ -266,13 +267,15 @@ step_attn_ring_kernel(const float* __restrict__ q, int ldq, int nq, int nkv, con
   extern __shared__ __align__(128) unsigned char sm_raw[];
   unsigned char* ring = sm_raw;                                                  // [STG][K page | V page]
   float* qs = reinterpret_cast<float*>(sm_raw + STG * 2 * PAGE_BYTES);           // [GP][HD], scaled, after RoPE
-  float* ps = qs + GP * HD;                                                      // [64 keys][GP]
-  float* m_run = ps + PAGE_TOKENS * GP;
+  float* ps = qs + GP * HD;                                                      // [64 keys][GP] probabilities
+  float* ss = ps + PAGE_TOKENS * GP;                                             // [64 keys][GP] scores
+  float* m_run = ss + PAGE_TOKENS * GP;                                          // exponent offset of each head
   float* l_run = m_run + GP;
   float* alpha = l_run + GP;
   __shared__ __align__(8) unsigned long long bars[STG];
   __shared__ int s_ok;
   __shared__ float rq[MAXG];
+  __shared__ int s_page[MAX_IDS];                  // page ids of this CTA's range (a global load per page would sit on the critical path)
   const int group = nq / nkv;                      // <= GP
   const int sp = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -283,9 +286,13 @@ step_attn_ring_kernel(const float* __restrict__ q, int ldq, int nq, int nkv, con
   const int pg0 = sp * per, pg1 = min(n_pg, pg0 + per);
   const int n_it = max(pg1 - pg0, 0);
 
-  auto issue = [&](int it) {     // thread 0: start the copies of page pg0 + it into slot it % STG
+  auto page_of = [&](int it) -> int {
+    if (it < MAX_IDS) return s_page[it];
     const int pg = pg0 + it;
-    int page = pg < mpps ? block_table[(size_t)b * mpps + pg] : -1;
+    return pg < mpps ? block_table[(size_t)b * mpps + pg] : -1;
+  };
+  auto issue = [&](int it) {     // thread 0: start the copies of page pg0 + it into slot it % STG
+    const int page = page_of(it);
     const uint32_t bar = smem_u32(&bars[it % STG]);
     if (page < 0 || page >= n_pages) {   // never dereferenced: the slot completes empty and the page is skipped below
       dev_flag(status, DEV_BAD_PAGE);
@@ -299,12 +306,18 @@ step_attn_ring_kernel(const float* __restrict__ q, int ldq, int nq, int nkv, con
     bulk_load(dst + PAGE_BYTES, vpool + off, PAGE_BYTES, bar);
   };
 
+  for (int i = tid; i < min(n_it, MAX_IDS); i += NT) {
+    const int pg = pg0 + i;
+    s_page[i] = pg < mpps ? block_table[(size_t)b * mpps + pg] : -1;
+  }
   if (tid == 0) {
     for (int s = 0; s < STG; ++s) mbar_init(smem_u32(&bars[s]), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     s_ok = 1;
-    for (int it = 0; it < min(STG - 1, n_it); ++it) issue(it);
   }
+  __syncthreads();
+  if (tid == 0)
+    for (int it = 0; it < min(STG - 1, n_it); ++it) issue(it);
   // queries of the group: (query norm,) RoPE at the last position, scaled by 1/sqrt(hd); heads beyond the group are zero
   if (q_gain) head_rnorm(q + (size_t)b * ldq + (size_t)kvh * group * HD, group, HD, eps, rq);
   {
@@ -347,6 +360,7 @@ step_attn_ring_kernel(const float* __restrict__ q, int ldq, int nq, int nkv, con
   float acc[GP][2];
 #pragma unroll
   for (int g = 0; g < GP; ++g) { acc[g][0] = 0.f; acc[g][1] = 0.f; }
+  float l_part = 0.f;                              // lane dq < GP: this key slot's share of head dq's sum of probabilities
   bool ok = true;
   for (int it = 0; it < n_it; ++it) {
     __syncthreads();                              // slot (it - 1) % STG and ps are free again
@@ -363,7 +377,7 @@ step_attn_ring_kernel(const float* __restrict__ q, int ldq, int nq, int nkv, con
     ok = __syncthreads_and(*(volatile int*)&s_ok != 0);
     if (!ok) break;
     const int pg = pg0 + it;
-    const int page = pg < mpps ? block_table[(size_t)b * mpps + pg] : -1;
+    const int page = page_of(it);
     const int nk = (page >= 0 && page < n_pages) ? min(PAGE_TOKENS, n_keys - pg * PAGE_TOKENS) : 0;
     const unsigned char* Ks = ring + (size_t)(it % STG) * 2 * PAGE_BYTES;
     const unsigned char* Vs = Ks + PAGE_BYTES;
@@ -397,29 +411,43 @@ step_attn_ring_kernel(const float* __restrict__ q, int ldq, int nq, int nkv, con
         for (int off = 1; off < DS; off <<= 1) s[g] += __shfl_xor_sync(0xffffffffu, s[g], off);
         if (dq == g) mine = s[g];
       }
-      if (dq < GP) ps[key * GP + dq] = key < nk ? mine : -INFINITY;
-    }
-    __syncthreads();
-    // ---- running softmax statistics, one warp per head
-    if (warp < GP) {
-      const int hh = warp;
-      const float s0 = ps[lane * GP + hh], s1 = ps[(32 + lane) * GP + hh];
-      const float mt = warp_max(fmaxf(s0, s1));
-      const float m_old = m_run[hh];
-      const float mn = fmaxf(m_old, mt);
-      const float p0 = (mn == -INFINITY) ? 0.f : __expf(s0 - mn), p1 = (mn == -INFINITY) ? 0.f : __expf(s1 - mn);
-      const float sum = warp_sum(p0 + p1);
-      ps[lane * GP + hh] = p0; ps[(32 + lane) * GP + hh] = p1;
-      if (lane == 0) {
-        const float a = (mn == -INFINITY) ? 1.f : __expf(m_old - mn);
-        alpha[hh] = a; m_run[hh] = mn; l_run[hh] = l_run[hh] * a + sum;
+      // Probabilities are taken against the head's current offset m_run straight away.  Only when a score
+      // exceeds the offset by more than 8 (always on the first page) does the block take the slow path
+      // below: new offset = running maximum, everything accumulated so far rescaled.
+      float pr = 0.f;
+      bool grow = false;
+      if (dq < GP) {
+        if (key >= nk) mine = -INFINITY;
+        const float mr = m_run[dq];
+        grow = mine > mr + 8.f;
+        pr = (mine == -INFINITY || grow) ? 0.f : __expf(mine - mr);
+        ss[key * GP + dq] = mine;
+        ps[key * GP + dq] = pr;
       }
+      if (__syncthreads_or(grow)) {
+        if (warp < GP) {
+          const int hh = warp;
+          const float mt = warp_max(fmaxf(ss[lane * GP + hh], ss[(32 + lane) * GP + hh]));
+          if (lane == 0) {
+            const float m_old = m_run[hh], mn = fmaxf(m_old, mt);
+            alpha[hh] = (m_old == -INFINITY) ? (mn == -INFINITY ? 1.f : 0.f) : __expf(m_old - mn);
+            m_run[hh] = mn;
+          }
+        }
+        __syncthreads();
+        if (dq < GP) {
+          pr = (mine == -INFINITY) ? 0.f : __expf(mine - m_run[dq]);
+          ps[key * GP + dq] = pr;
+          l_part *= alpha[dq];
+        }
+#pragma unroll
+        for (int g = 0; g < GP; ++g) { const float al = alpha[g]; acc[g][0] *= al; acc[g][1] *= al; }
+        __syncthreads();
+      }
+      l_part += pr;
     }
-    __syncthreads();
     // ---- values: keys beyond nk carry p = 0 but their rows are not initialised memory: they are not read
     {
-#pragma unroll
-      for (int g = 0; g < GP; ++g) { const float a = alpha[g]; acc[g][0] *= a; acc[g][1] *= a; }
       const uint32_t* vr = reinterpret_cast<const uint32_t*>(Vs) + d2;
       const int s1 = min(nk, (kq + 1) * KPT);
 #pragma unroll 4
@@ -446,6 +474,13 @@ step_attn_ring_kernel(const float* __restrict__ q, int ldq, int nq, int nkv, con
     return;
   }
   __syncthreads();
+  if (dq < GP) ps[key * GP + dq] = l_part;         // the heads' sums of probabilities
+  __syncthreads();
+  if (tid < GP) {
+    float l = 0.f;
+    for (int i = 0; i < PAGE_TOKENS; ++i) l += ps[i * GP + tid];
+    l_run[tid] = l;
+  }
   // the key blocks' sums meet in shared memory (the ring is idle: every copy issued was waited for)
   float* red = reinterpret_cast<float*>(ring);                                   // [NKQ][GP][HD]
 #pragma unroll
