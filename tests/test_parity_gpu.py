@@ -55,6 +55,14 @@ CASES = [
     ("t_hd128_qkn", [40, 9, 130, 17, 64, 65, 3, 90, 128], "fanin"),
     ("t_small_qkn", [4200, 70], "fanin"),
     ("t_small_qkn", [1, 2, 3, 5, 8, 13, 21, 34, 55, 89] * 13, "fanin"),
+    # other group sizes of the step attention over the bf16 cache (1, 2 and 8 query heads per kv head), with more
+    # than 4 sequences and with a small batch over a long cache
+    ("t_mha", [40, 9, 130, 17, 64, 65], "fanin"),
+    ("t_g2", [40, 9, 130, 17, 64, 65], "fanin"),
+    ("t_g8", [40, 9, 130, 17, 64, 65], "fanin"),
+    ("t_mha", [4130, 3], "fanin"),
+    ("t_g2", [4130], "n002"),
+    ("t_g8", [4130, 64], "fanin"),
 ]
 
 
@@ -79,7 +87,10 @@ def test_prefill_predict_matches_oracle(name, lens, regime):
                                               ("c1", "n002", [64]), ("t_small", "n002", [70, 63, 5, 64, 1, 30]),
                                               ("t_small_qkn", "fanin", [70, 63, 5]),
                                               ("t_small_qkn_f32", "fanin", [70, 5]),
-                                              ("t_hd128_qkn", "fanin", [70, 63, 5, 64, 1, 30])],
+                                              ("t_hd128_qkn", "fanin", [70, 63, 5, 64, 1, 30]),
+                                              ("t_mha", "fanin", [70, 63, 5, 64, 1, 30]),
+                                              ("t_g2", "fanin", [70, 63, 5, 64, 1, 30]),
+                                              ("t_g8", "fanin", [70, 63, 5, 64, 1, 30])],
                          ids=lambda v: str(v).replace(" ", ""))
 def test_decode_steps_match_oracle(name, regime, lens):
     import torch

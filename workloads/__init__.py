@@ -172,6 +172,18 @@ def pair(name: str) -> PairCfg:
         aux = layerwise_scaled_model(4, 256, 4, 8, 64, 1500, 0.5, 2.0)
         base = layerwise_scaled_model(6, 384, 4, 12, 64, 1500, 0.5, 2.0)
         return PairCfg("t_scaled", aux, base, (0, 0, 1, 1, 2, 3))
+    if name == "t_mha":       # one query head per kv head (head_dim 64)
+        aux = uniform_model(2, 192, 3, 3, 64, 320, 1000)
+        base = uniform_model(4, 256, 4, 4, 64, 448, 1000)
+        return PairCfg("t_mha", aux, base, (0, 0, 1, 1))
+    if name == "t_g2":        # two query heads per kv head, head_dim 128
+        aux = uniform_model(2, 256, 2, 1, 128, 512, 1000)
+        base = uniform_model(3, 512, 4, 2, 128, 1024, 1000)
+        return PairCfg("t_g2", aux, base, (0, 1, 1))
+    if name == "t_g8":        # eight query heads per kv head (the widest group the step kernels take)
+        aux = uniform_model(2, 192, 4, 1, 64, 320, 1000)
+        base = uniform_model(3, 512, 8, 1, 64, 1024, 1000)
+        return PairCfg("t_g8", aux, base, (0, 1, 1))
     if name == "t_bias":      # predictor with bias terms
         p = pair("t_small")
         return PairCfg("t_bias", p.aux, p.base, p.layer_map, predictor_bias=True)
