@@ -164,7 +164,8 @@ void launch_step_gemv(const LaunchCtx&, const void* W, int ldw, int N, int K, co
 void launch_step_attn(const LaunchCtx&, const float* q, int ldq, int nq, int nkv, int hd, float theta,
                       const void* kpool, const void* vpool, const int* block_table,
                       int max_pages_per_seq, int n_pages, const int* seq_lens, int extra, int batch,
-                      int max_keys, float* part, float* out, const float* q_gain = nullptr, float eps = 0.f);
+                      int max_keys, float* part, float* out, const float* q_gain = nullptr, float eps = 0.f,
+                      int* split_done = nullptr /* [batch * nkv] ints: lets the attention kernel merge its own key-range splits */);
 void launch_step_append(const LaunchCtx&, const float* qkv, int nq, int nkv, int hd, float theta,
                         void* kpool, void* vpool, const int* block_table, int max_pages_per_seq,
                         int n_pages, const int* seq_lens, int batch, const float* k_gain = nullptr, float eps = 0.f);
@@ -177,4 +178,4 @@ bool step_attn_ring_supported(int dtype, int nq, int nkv, int hd, const void* kp
 cudaError_t launch_step_attn_ring(const LaunchCtx&, const float* q, int ldq, int nq, int nkv, int hd, float theta,
                                   const void* kpool, const void* vpool, const int* block_table, int max_pages_per_seq,
                                   int n_pages, const int* seq_lens, int extra, int batch, int n_split, float* part, float* out,
-                                  const float* q_gain = nullptr, float eps = 0.f);
+                                  const float* q_gain = nullptr, float eps = 0.f, int* split_done = nullptr);

@@ -259,7 +259,7 @@ void base_layer_step(kvp_handle* h, const LaunchCtx& ctx, int i, const kvp_cache
                        cache->max_pages_per_seq, cache->n_pages, cache->seq_lens, batch, kn, B.eps));
   KVP_TIMED(KVP_CLASS_STEP_ATTN, launch_step_attn(ctx, qkvb, n_out, L.nq, L.nkv, L.hd, B.theta, cache->k_pools[i], cache->v_pools[i], cache->block_table,
                    cache->max_pages_per_seq, cache->n_pages, cache->seq_lens, generation ? 1 : 0, batch, max_keys,
-                   (float*)(ws + w.part), ab, qn, B.eps));
+                   (float*)(ws + w.part), ab, qn, B.eps, (int*)(ws + w.attn_done)));
   if (tc) {
     float* gub = (float*)(ws + w.gub);
     step_proj_tc(h, ctx, w, ws, PREP_PLAIN, ab, L.dq, L.dq, batch, nullptr, 0, P + L.wo, B.d, xb, B.d, false, err);

@@ -260,7 +260,7 @@ step_attn_ring_kernel(const float* __restrict__ q, int ldq, int nq, int nkv, con
                       const bf16* __restrict__ kpool, const bf16* __restrict__ vpool, const int* __restrict__ block_table,
                       int mpps, int n_pages, const int* __restrict__ seq_lens, int extra, int n_split,
                       float* __restrict__ part, float* __restrict__ out, int* status, const float* __restrict__ q_gain,
-                      float eps) {
+                      float eps, int* __restrict__ split_done) {
   using Cfg = RingCfg<HD, GP>;
   constexpr int DS = Cfg::DS, NT = Cfg::NT, CPT = Cfg::CPT, NKQ = Cfg::NKQ, KPT = Cfg::KPT, STG = Cfg::STAGES;
   constexpr int PAGE_BYTES = Cfg::PAGE_BYTES;
@@ -501,12 +501,40 @@ step_attn_ring_kernel(const float* __restrict__ q, int ldq, int nq, int nkv, con
     float* pr = part + (((size_t)b * nq + kvh * group + tid) * n_split + sp) * ldr;
     pr[HD] = m_run[tid]; pr[HD + 1] = l_run[tid];
   }
+  // With a counter per (sequence, kv head) (zero at launch) the CTA that finishes the group's last split merges the
+  // partial results on the spot; without one a separate kernel does it.
+  if (n_split > 1 && split_done) {
+    __shared__ int s_last;
+    __threadfence();                               // this CTA's partial results are visible before it counts itself done
+    __syncthreads();
+    if (tid == 0) s_last = atomicAdd(split_done + b * nkv + kvh, 1) == n_split - 1;
+    __syncthreads();
+    if (s_last) {
+      __threadfence();
+      for (int o = tid; o < group * HD; o += NT) {
+        const int g = o / HD, d = o - g * HD;
+        const int qh = kvh * group + g;
+        const float* pr = part + ((size_t)b * nq + qh) * n_split * ldr;
+        float mm = -INFINITY;
+        for (int s = 0; s < n_split; ++s) mm = fmaxf(mm, __ldcg(pr + (size_t)s * ldr + HD));
+        float ll = 0.f, v = 0.f;
+        for (int s = 0; s < n_split; ++s) {
+          const float* r = pr + (size_t)s * ldr;
+          const float ms = __ldcg(r + HD);
+          const float f = (ms == -INFINITY) ? 0.f : __expf(ms - mm);
+          ll = fmaf(__ldcg(r + HD + 1), f, ll);
+          v = fmaf(__ldcg(r + d), f, v);
+        }
+        out[(size_t)b * nq * HD + (size_t)qh * HD + d] = v / ll;
+      }
+    }
+  }
 }
 
 template <int HD, int GP>
 cudaError_t go_ring(dim3 grid, cudaStream_t st, const float* q, int ldq, int nq, int nkv, const InvFreq& inv, const bf16* kpool,
                     const bf16* vpool, const int* block_table, int mpps, int n_pages, const int* seq_lens, int extra, int n_split,
-                    float* part, float* out, int* status, const float* q_gain, float eps) {
+                    float* part, float* out, int* status, const float* q_gain, float eps, int* split_done) {
   using Cfg = RingCfg<HD, GP>;
   static bool attr_set = false;
   if (!attr_set) {
@@ -515,19 +543,19 @@ cudaError_t go_ring(dim3 grid, cudaStream_t st, const float* q, int ldq, int nq,
     attr_set = true;
   }
   step_attn_ring_kernel<HD, GP><<<grid, Cfg::NT, Cfg::SMEM, st>>>(q, ldq, nq, nkv, inv, kpool, vpool, block_table, mpps, n_pages, seq_lens,
-                                                                  extra, n_split, part, out, status, q_gain, eps);
+                                                                  extra, n_split, part, out, status, q_gain, eps, split_done);
   return cudaGetLastError();
 }
 
 template <int HD>
 cudaError_t go_ring_hd(int group, dim3 grid, cudaStream_t st, const float* q, int ldq, int nq, int nkv, const InvFreq& inv,
                        const bf16* kpool, const bf16* vpool, const int* block_table, int mpps, int n_pages, const int* seq_lens,
-                       int extra, int n_split, float* part, float* out, int* status, const float* q_gain, float eps) {
+                       int extra, int n_split, float* part, float* out, int* status, const float* q_gain, float eps, int* split_done) {
   if (group == 1)
-    return go_ring<HD, 1>(grid, st, q, ldq, nq, nkv, inv, kpool, vpool, block_table, mpps, n_pages, seq_lens, extra, n_split, part, out, status, q_gain, eps);
+    return go_ring<HD, 1>(grid, st, q, ldq, nq, nkv, inv, kpool, vpool, block_table, mpps, n_pages, seq_lens, extra, n_split, part, out, status, q_gain, eps, split_done);
   if (group == 2)
-    return go_ring<HD, 2>(grid, st, q, ldq, nq, nkv, inv, kpool, vpool, block_table, mpps, n_pages, seq_lens, extra, n_split, part, out, status, q_gain, eps);
-  return go_ring<HD, 4>(grid, st, q, ldq, nq, nkv, inv, kpool, vpool, block_table, mpps, n_pages, seq_lens, extra, n_split, part, out, status, q_gain, eps);
+    return go_ring<HD, 2>(grid, st, q, ldq, nq, nkv, inv, kpool, vpool, block_table, mpps, n_pages, seq_lens, extra, n_split, part, out, status, q_gain, eps, split_done);
+  return go_ring<HD, 4>(grid, st, q, ldq, nq, nkv, inv, kpool, vpool, block_table, mpps, n_pages, seq_lens, extra, n_split, part, out, status, q_gain, eps, split_done);
 }
 
 template <int HD>
@@ -574,7 +602,7 @@ bool step_attn_ring_supported(int dtype, int nq, int nkv, int hd, const void* kp
 
 cudaError_t launch_step_attn_ring(const LaunchCtx& ctx, const float* q, int ldq, int nq, int nkv, int hd, float theta, const void* kpool,
                                   const void* vpool, const int* block_table, int mpps, int n_pages, const int* seq_lens, int extra,
-                                  int batch, int n_split, float* part, float* out, const float* q_gain, float eps) {
+                                  int batch, int n_split, float* part, float* out, const float* q_gain, float eps, int* split_done) {
   InvFreq inv;
   fill_inv_freq(&inv, hd, theta);
   dim3 grid(n_split, nkv, batch);
@@ -584,9 +612,9 @@ cudaError_t launch_step_attn_ring(const LaunchCtx& ctx, const float* q, int ldq,
   if (group <= 4) {
     if (hd == 64)
       return go_ring_hd<64>(group, grid, ctx.st, q, ldq, nq, nkv, inv, (const bf16*)kpool, (const bf16*)vpool, block_table, mpps, n_pages,
-                            seq_lens, extra, n_split, part, out, ctx.status, q_gain, eps);
+                            seq_lens, extra, n_split, part, out, ctx.status, q_gain, eps, split_done);
     return go_ring_hd<128>(group, grid, ctx.st, q, ldq, nq, nkv, inv, (const bf16*)kpool, (const bf16*)vpool, block_table, mpps, n_pages,
-                           seq_lens, extra, n_split, part, out, ctx.status, q_gain, eps);
+                           seq_lens, extra, n_split, part, out, ctx.status, q_gain, eps, split_done);
   }
   if (hd == 64)
     return go<64>(grid, threads, ctx.st, q, ldq, nq, nkv, inv, (const bf16*)kpool, (const bf16*)vpool, block_table, mpps, n_pages, seq_lens,

@@ -592,7 +592,7 @@ int step_attn_splits(int batch, int nkv, int max_keys) {
 void launch_step_attn(const LaunchCtx& ctx, const float* q, int ldq, int nq, int nkv, int hd, float theta,
                       const void* kpool, const void* vpool, const int* block_table, int mpps, int n_pages,
                       const int* seq_lens, int extra, int batch, int max_keys, float* part, float* out, const float* q_gain,
-                      float eps) {
+                      float eps, int* split_done) {
   // every sequence attends to seq_lens[b] + extra keys; max_keys bounds that count (host copy).
   InvFreq inv;
   fill_inv_freq(&inv, hd, theta);
@@ -600,8 +600,12 @@ void launch_step_attn(const LaunchCtx& ctx, const float* q, int ldq, int nq, int
   dim3 grid(n_split, nkv, batch);
   if (step_attn_ring_supported(ctx.dtype, nq, nkv, hd, kpool, vpool)) {
     n_split = step_attn_ring_splits(nq, nkv, hd, batch, max_keys, n_split);
-    launch_step_attn_ring(ctx, q, ldq, nq, nkv, hd, theta, kpool, vpool, block_table, mpps, n_pages, seq_lens, extra, batch, n_split, part, out, q_gain, eps);
-    if (n_split > 1) {
+    // up to 4 heads per kv head: the CTA that finishes a group's last split merges it (counters cleared here)
+    const bool fused = split_done && n_split > 1 && nq / nkv <= 4;
+    if (fused) cudaMemsetAsync(split_done, 0, (size_t)batch * nkv * sizeof(int), ctx.st);
+    launch_step_attn_ring(ctx, q, ldq, nq, nkv, hd, theta, kpool, vpool, block_table, mpps, n_pages, seq_lens, extra, batch, n_split, part, out,
+                          q_gain, eps, fused ? split_done : nullptr);
+    if (n_split > 1 && !fused) {
       ++*ctx.n_launch;
       step_attn_merge_kernel<<<dim3(nq, batch), 64, 0, ctx.st>>>(part, nq, hd, n_split, out);
     }
