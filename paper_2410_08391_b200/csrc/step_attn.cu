@@ -6,20 +6,25 @@
 // ring of shared-memory stages, several pages ahead of the arithmetic: the HBM latency is covered
 // by copies in flight, not by resident warps.
 //
-// step_attn_ring_wide_kernel (up to 4 query heads per kv head): every cached element is read from
+// step_attn_ring_kernel (up to 4 query heads per kv head): every cached element is read from
 // shared memory ONCE and used for all heads of the group, because the shared-memory port, not
 // HBM, bounds a kernel that re-reads a page per head.
 //   scores   DS lanes share a key: each holds its slice of the group's queries in registers for
 //            the whole kernel, reads its 16-byte pieces of the key row (pieces interleaved over
 //            the lanes and visited in an order rotated by the key index: conflict-free), and the
 //            DS partial dot products per head are added with shuffles
-//   softmax  one warp per head over the page's 64 scores, running max / sum in shared memory
+//   softmax  a key's lane takes exp(score - offset) against the head's current exponent offset at
+//            once; only when a score exceeds the offset by more than 8 (always on the first page)
+//            does the block move the offset to the running maximum and rescale what it has summed
 //   values   thread = (pair of dims, block of keys): one 4-byte read of V and one broadcast read
 //            of the key's probabilities feed 2 x group multiply-adds; the key blocks are summed
 //            through shared memory once, after the last page
+//   The page ids of the CTA's range are staged in shared memory once.
 // step_attn_ring_wide_kernel (5 to 8 heads per kv head): thread = (key, head) for the scores and
-// (pair of dims, head) for the values.
-// With more than one split, partial (o, m, l) per (sequence, q head, split) go to `part`.
+// (pair of dims, head) for the values, one warp per head for a per-page softmax.
+// With more than one split, partial (o, m, l) per (sequence, q head, split) go to `part`; given a
+// zeroed counter per (sequence, kv head), the CTA of step_attn_ring_kernel that finishes a group's
+// last split merges them, otherwise a separate kernel does.
 // The wait on a page's copies is bounded; on expiry the CTA flags DEV_TIMEOUT and leaves.
 #include <math.h>
 
