@@ -19,7 +19,8 @@
 //   values   thread = (pair of dims, block of keys): one 4-byte read of V and one broadcast read
 //            of the key's probabilities feed 2 x group multiply-adds; the key blocks are summed
 //            through shared memory once, after the last page
-//   The page ids of the CTA's range are staged in shared memory once.
+//   The page ids of the CTA's range are staged in shared memory once; a page costs one block
+//   barrier (the vote on the offset).
 // step_attn_ring_wide_kernel (5 to 8 heads per kv head): thread = (key, head) for the scores and
 // (pair of dims, head) for the values, one warp per head for a per-page softmax.
 // With more than one split, partial (o, m, l) per (sequence, q head, split) go to `part`; given a
@@ -256,7 +257,7 @@ struct RingCfg {
   static constexpr int PAGE_BYTES = PAGE_TOKENS * HD * 2;  // one K or V page of one kv head
   // pages in flight: one 512-thread CTA per SM keeps 5 pages ahead, two 256-thread CTAs 2 or 4 each
   static constexpr int STAGES = NT == 512 ? 6 : (HD == 64 ? 5 : 3);
-  static constexpr size_t SMEM = (size_t)STAGES * 2 * PAGE_BYTES + (size_t)(GP * HD + 2 * PAGE_TOKENS * GP + 3 * GP) * sizeof(float);
+  static constexpr size_t SMEM = (size_t)STAGES * 2 * PAGE_BYTES + (size_t)(GP * HD + 3 * PAGE_TOKENS * GP + 3 * GP) * sizeof(float);
 };
 
 template <int HD, int GP>
@@ -272,8 +273,8 @@ step_attn_ring_kernel(const float* __restrict__ q, int ldq, int nq, int nkv, con
   extern __shared__ __align__(128) unsigned char sm_raw[];
   unsigned char* ring = sm_raw;                                                  // [STG][K page | V page]
   float* qs = reinterpret_cast<float*>(sm_raw + STG * 2 * PAGE_BYTES);           // [GP][HD], scaled, after RoPE
-  float* ps = qs + GP * HD;                                                      // [64 keys][GP] probabilities
-  float* ss = ps + PAGE_TOKENS * GP;                                             // [64 keys][GP] scores
+  float* ps_buf = qs + GP * HD;                                                  // 2 x [64 keys][GP] probabilities (alternating pages)
+  float* ss = ps_buf + 2 * PAGE_TOKENS * GP;                                     // [64 keys][GP] scores
   float* m_run = ss + PAGE_TOKENS * GP;                                          // exponent offset of each head
   float* l_run = m_run + GP;
   float* alpha = l_run + GP;
@@ -367,9 +368,11 @@ step_attn_ring_kernel(const float* __restrict__ q, int ldq, int nq, int nkv, con
   for (int g = 0; g < GP; ++g) { acc[g][0] = 0.f; acc[g][1] = 0.f; }
   float l_part = 0.f;                              // lane dq < GP: this key slot's share of head dq's sum of probabilities
   bool ok = true;
+  // One block barrier per page: a page's probabilities go to the buffer the page before last used, and the
+  // slot of page it - 1 is refilled after the barrier of page it, which every thread passes only once it
+  // is through with page it - 1.
   for (int it = 0; it < n_it; ++it) {
-    __syncthreads();                              // slot (it - 1) % STG and ps are free again
-    if (tid == 0 && it + STG - 1 < n_it) issue(it + STG - 1);
+    float* ps = ps_buf + (it & 1) * PAGE_TOKENS * GP;
     {                                             // wait for this page's copies (every thread polls; bounded)
       const uint32_t bar = smem_u32(&bars[it % STG]), parity = (it / STG) & 1;
       bool got = false;
@@ -379,8 +382,6 @@ step_attn_ring_kernel(const float* __restrict__ q, int ldq, int nq, int nkv, con
       }
       if (!got) { s_ok = 0; dev_flag(status, DEV_TIMEOUT); }
     }
-    ok = __syncthreads_and(*(volatile int*)&s_ok != 0);
-    if (!ok) break;
     const int pg = pg0 + it;
     const int page = page_of(it);
     const int nk = (page >= 0 && page < n_pages) ? min(PAGE_TOKENS, n_keys - pg * PAGE_TOKENS) : 0;
@@ -429,7 +430,13 @@ step_attn_ring_kernel(const float* __restrict__ q, int ldq, int nq, int nkv, con
         ss[key * GP + dq] = mine;
         ps[key * GP + dq] = pr;
       }
-      if (__syncthreads_or(grow)) {
+      const int any_grow = __syncthreads_or(grow);
+      if (*(volatile int*)&s_ok == 0) { ok = false; break; }      // a wait ran out (same answer in every thread: read after the barrier)
+      if (tid == 0 && it + STG - 1 < n_it) {
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the block's reads of that slot come before the copy's writes
+        issue(it + STG - 1);
+      }
+      if (any_grow) {
         if (warp < GP) {
           const int hh = warp;
           const float mt = warp_max(fmaxf(ss[lane * GP + hh], ss[(32 + lane) * GP + hh]));
@@ -479,11 +486,11 @@ step_attn_ring_kernel(const float* __restrict__ q, int ldq, int nq, int nkv, con
     return;
   }
   __syncthreads();
-  if (dq < GP) ps[key * GP + dq] = l_part;         // the heads' sums of probabilities
+  if (dq < GP) ps_buf[key * GP + dq] = l_part;     // the heads' sums of probabilities
   __syncthreads();
   if (tid < GP) {
     float l = 0.f;
-    for (int i = 0; i < PAGE_TOKENS; ++i) l += ps[i * GP + tid];
+    for (int i = 0; i < PAGE_TOKENS; ++i) l += ps_buf[i * GP + tid];
     l_run[tid] = l;
   }
   // the key blocks' sums meet in shared memory (the ring is idle: every copy issued was waited for)
