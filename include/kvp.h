@@ -11,8 +11,11 @@
  *
  * General conventions
  *   - Every call returns a kvp_status (0 = KVP_OK, negative = error).  Nothing
- *     throws, aborts or keeps global state.  kvp_last_error() returns a message
- *     owned by the handle, valid until the next call on that handle.
+ *     throws or aborts.  State lives in the handle; the only process-wide state is a
+ *     set of per-device flags (which kernels have had their shared-memory limit
+ *     raised on which device) and the built-in scratch array of kvp_decode_step_static.
+ *     kvp_last_error() returns a message owned by the handle, valid until the next
+ *     call on that handle.
  *   - "dev" pointers are CUDA device pointers on the device that was current when
  *     kvp_create() ran; "host" pointers are ordinary host memory.
  *   - The caller owns ALL device memory (weights, packed weights, workspace, cache
@@ -84,8 +87,9 @@ typedef struct {
 } kvp_model_cfg;
 
 typedef struct {
-  int32_t dtype;          /* KVP_F32 | KVP_BF16: storage type of weights, activations and cache.
-                             Accumulation, norms, softmax and the base step's activations are fp32. */
+  int32_t dtype;          /* KVP_F32 | KVP_BF16: storage type of weights and activations (tensor-core operands).
+                             Accumulation, norms, softmax and the base step's activations are fp32.  The cache
+                             holds fp32 elements in KVP_F32 mode and IEEE half elements in KVP_BF16 mode.    */
   int32_t page_tokens;    /* tokens per cache page; must be 64                                       */
   int32_t predictor_bias; /* 1: the predictor has bias vectors pred.L{i}.bk / bv                     */
   int32_t reserved;       /* must be 0                                                               */
@@ -112,7 +116,9 @@ typedef struct {
 /* The paged base-model KV cache, the user-visible product of prefill (Sec. 4.1:
  * the predicted cache is what the base model's attention then consumes).
  * Base layer i has one K pool and one V pool of n_pages pages; a page is
- * [n_kv_heads_i][page_tokens][head_dim] elements of the run dtype.  Entry t of
+ * [n_kv_heads_i][page_tokens][head_dim] elements: fp32 in KVP_F32 mode; in KVP_BF16 mode 16-bit IEEE half
+ * (fp16: 11 significant bits, stores saturate at +-65504), not bfloat16: the cache is the product of the path
+ * and the base model's step amplifies its rounding several times in the logits.  Entry t of
  * sequence b lives in page block_table[b * max_pages_per_seq + t / page_tokens]
  * at row t % page_tokens, in every layer's pools.  Keys are stored after RoPE.
  * Rows at or beyond a sequence's length are unspecified. */
@@ -225,7 +231,8 @@ kvp_status kvp_decode_step(kvp_handle* h, const int32_t* tokens /* dev [batch] *
  *   - A step whose kvp_workspace_bytes(h, batch, batch) exceeds KVP_STATIC_SCRATCH_BYTES is
  *     rejected with KVP_ERR_WORKSPACE and a message naming both sizes.
  *   - The first call on each device looks up the array's device address (with that device
- *     current); make that first call before any stream capture begins.
+ *     current); make that first call before any stream capture begins.  Arguments are checked
+ *     before the array or the stream is touched.
  *   - All calls on a device share the one array, which keeps the previous call's contents.
  *     The call clears the status word itself; everything else is overwritten before it is
  *     read.  Two calls that overlap on the GPU (different streams or handles) race on the
@@ -260,6 +267,13 @@ kvp_status kvp_train_forward(kvp_handle* h, const int32_t* tokens /* dev [sum(le
 /* Synchronises `stream`, reads the device status word of `workspace`, clears it and returns
  * KVP_OK, KVP_ERR_TIMEOUT, KVP_ERR_BAD_INDEX or KVP_ERR_CUDA. */
 kvp_status kvp_poll_status(kvp_handle* h, void* workspace, void* stream);
+
+/* Self-test of the error path behind KVP_ERR_TIMEOUT (the paper has no counterpart).  Enqueues a one-block
+ * kernel that waits, with the same bounded wait every kernel of the library uses but a limit of a few thousand
+ * polls, on a barrier that nothing completes.  The wait runs out, the kernel returns normally and records its code
+ * in the status word of `workspace` (dev, >= 16 bytes, as passed to the compute calls); kvp_poll_status then
+ * returns KVP_ERR_TIMEOUT and clears the word, and the handle and the context stay usable. */
+kvp_status kvp_selftest_wait_timeout(kvp_handle* h, void* workspace, void* stream);
 
 /* Number of kernels the handle launched since creation (for launch accounting). */
 int64_t kvp_launch_count(const kvp_handle* h);

@@ -6,5 +6,5 @@ from . import binding  # noqa: F401
 from .binding import (KvpError, Session, kvp_cache_layout, kvp_create, kvp_decode_step, kvp_decode_step_static, kvp_destroy,  # noqa: F401
                       kvp_last_error, kvp_launch_count, kvp_layer_map_canonical, kvp_layer_map_pruned,
                       kvp_layer_map_uniform, kvp_load_weights, kvp_packed_weight_bytes, kvp_poll_status,
-                      kvp_prefill_predict, kvp_prefill_predict_host, kvp_timing_enable, kvp_timing_read,
+                      kvp_prefill_predict, kvp_prefill_predict_host, kvp_selftest_wait_timeout, kvp_timing_enable, kvp_timing_read,
                       kvp_train_forward, kvp_train_workspace_bytes, kvp_workspace_bytes, lib)

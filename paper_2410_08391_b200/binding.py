@@ -52,7 +52,7 @@ EXPORTS = ["kvp_create", "kvp_destroy", "kvp_last_error", "kvp_layer_map_canonic
            "kvp_layer_map_uniform", "kvp_packed_weight_bytes", "kvp_workspace_bytes", "kvp_cache_layout",
            "kvp_load_weights", "kvp_prefill_predict", "kvp_prefill_predict_host", "kvp_decode_step",
            "kvp_poll_status", "kvp_launch_count", "kvp_timing_enable", "kvp_timing_read",
-           "kvp_decode_step_static", "kvp_train_workspace_bytes", "kvp_train_forward"]
+           "kvp_decode_step_static", "kvp_train_workspace_bytes", "kvp_train_forward", "kvp_selftest_wait_timeout"]
 
 CLASS_NAMES = ["aux_gemm", "aux_attn", "predictor", "step_gemv", "step_attn", "other", "step_fused"]
 
@@ -86,6 +86,7 @@ def lib() -> C.CDLL:
         L.kvp_train_workspace_bytes.argtypes = [vp, i32, i64, C.POINTER(C.c_size_t)]
         L.kvp_train_forward.argtypes = [vp, vp, C.POINTER(i32), i32, C.POINTER(CacheC), vp, C.c_size_t, vp, vp, vp, vp]
         L.kvp_poll_status.argtypes = [vp, vp, vp]
+        L.kvp_selftest_wait_timeout.argtypes = [vp, vp, vp]
         L.kvp_launch_count.argtypes = [vp]
         L.kvp_launch_count.restype = i64
         L.kvp_timing_enable.argtypes = [vp, i32]
@@ -250,6 +251,10 @@ def kvp_train_forward(h, tokens, lengths: Sequence[int], cache: "Cache", workspa
                                    l1_k.data_ptr(), l1_v.data_ptr(), stream), h)
 
 
+def kvp_selftest_wait_timeout(h, workspace, stream: int) -> None:
+    _check(lib().kvp_selftest_wait_timeout(h, workspace.data_ptr(), stream), h)
+
+
 def kvp_poll_status(h, workspace, stream: int) -> None:
     _check(lib().kvp_poll_status(h, workspace.data_ptr(), stream), h)
 
@@ -262,7 +267,8 @@ class Cache:
                  shuffle_pages: bool = True, seed: int = 0):
         import torch
         self.pair = pair
-        tdt = torch.bfloat16 if pair.dtype == "bf16" else torch.float32
+        # 16-bit cache elements are IEEE halves (see kvp.h: more significant bits than bfloat16 for the path's product)
+        tdt = torch.float16 if pair.dtype == "bf16" else torch.float32
         self.max_pages_per_seq = (max_len + 63) // 64
         self.n_pages = n_pages if n_pages is not None else max_batch * self.max_pages_per_seq
         nl = pair.base.n_layers

@@ -1,10 +1,15 @@
 // Shared device helpers and launch-function declarations for the KV Prediction library.
 #pragma once
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
 typedef __nv_bfloat16 bf16;
+// Element of the paged cache in bf16 mode.  The predicted cache is the product of the path, and the base step
+// amplifies its rounding about five-fold in the logits, so its 16 bits carry 11 significant bits (IEEE half)
+// instead of bfloat16's 8.  Stores saturate at the largest finite half.
+typedef __half kv16;
 
 // Codes kernels write into the device status word (first int of the workspace).
 enum : int { DEV_OK = 0, DEV_TIMEOUT = 1, DEV_BAD_TOKEN = 2, DEV_BAD_PAGE = 3 };
@@ -14,9 +19,17 @@ constexpr int MAX_PRED_SEG = 8;   // base layers fed by one auxiliary layer
 
 __device__ __forceinline__ float to_f(float v) { return v; }
 __device__ __forceinline__ float to_f(bf16 v) { return __bfloat162float(v); }
+__device__ __forceinline__ float to_f(kv16 v) { return __half2float(v); }
 template <class T> __device__ __forceinline__ T from_f(float v);
 template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
 template <> __device__ __forceinline__ bf16 from_f<bf16>(float v) { return __float2bfloat16_rn(v); }
+template <> __device__ __forceinline__ kv16 from_f<kv16>(float v) { return __float2half_rn(fminf(fmaxf(v, -65504.f), 65504.f)); }
+// the two cache elements held by a 32-bit word (element 2i in the low half)
+__device__ __forceinline__ float kv_lo(uint32_t u) { return __low2float(*reinterpret_cast<const __half2*>(&u)); }
+__device__ __forceinline__ float kv_hi(uint32_t u) { return __high2float(*reinterpret_cast<const __half2*>(&u)); }
+// cache element type for a run dtype: fp32 pools in fp32 mode, kv16 pools in bf16 mode
+template <class T> struct KvOf { typedef T type; };
+template <> struct KvOf<bf16> { typedef kv16 type; };
 
 __device__ __forceinline__ void dev_flag(int* status, int code) { atomicCAS(status, DEV_OK, code); }
 

@@ -68,7 +68,8 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmArgs g) {
         if (p.bias) v += p.bias[n];
         int page = slot / PAGE_TOKENS, row = slot - page * PAGE_TOKENS;
         size_t off = (((size_t)page * p.n_kv[s] + head) * PAGE_TOKENS + row) * p.head_dim + dim;
-        ((T*)p.pool[s])[off] = from_f<T>(v);
+        typedef typename KvOf<T>::type KT;     // cache element of this run dtype
+        ((KT*)p.pool[s])[off] = from_f<KT>(v);
       }
     }
   }

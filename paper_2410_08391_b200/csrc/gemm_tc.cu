@@ -22,8 +22,10 @@
 
 #include "common.cuh"
 #include "gemm_tc.h"
+#include "tc_ptx.cuh"
 
 namespace {
+using namespace tcp;
 
 constexpr int BM = 128, BK = 64;
 constexpr int GROUP_M = 16;                                // row blocks per rasterisation group
@@ -34,92 +36,6 @@ template <int BN> struct Tile {
   static constexpr int STAGE_BYTES = A_BYTES + W_BYTES;    // 48 KiB / 32 KiB
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
 };
-constexpr uint32_t SPIN_LIMIT = 20u * 1000u * 1000u;      // ~1-2 s of polling
-
-// ---- PTX wrappers -------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait.  Returns false if the kernel is aborting (this or another role gave up).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
-  for (uint32_t it = 0; it < SPIN_LIMIT; ++it) {
-    if (mbar_test(bar, parity)) return true;
-    if ((it & 63u) == 63u) {
-      if (*abort_flag) return false;
-      __nanosleep(64);
-    }
-  }
-  *abort_flag = 1;
-  dev_flag(status, DEV_TIMEOUT);
-  return false;
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
-      : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-
-__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-
-// 32 lanes x 32 columns of fp32: thread i of the warp gets row i, register j = column j.
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
-  uint32_t* r = reinterpret_cast<uint32_t*>(v);
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// Shared-memory matrix descriptor of a K-major bf16 tile stored with the 128-byte swizzle:
-// rows of 128 bytes, groups of 8 rows 1024 bytes apart.
-__device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr) {
-  uint64_t lo = ((smem_addr & 0x3FFFFu) >> 4) | (1u << 16);             // start address, leading offset (unused)
-  uint64_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);                 // stride offset, version 1, 128B swizzle
-  return lo | (hi << 32);
-}
-
 __device__ __forceinline__ uint4 pack8(const float* v) {
   __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
   __nv_bfloat162 c = __floats2bfloat162_rn(v[4], v[5]), d = __floats2bfloat162_rn(v[6], v[7]);
@@ -134,6 +50,22 @@ __device__ __forceinline__ uint4 pack8_lo(const float* v) {
 #pragma unroll
   for (int i = 0; i < 8; ++i) r[i] = v[i] - __bfloat162float(__float2bfloat16_rn(v[i]));
   return pack8(r);
+}
+// 32 values as cache elements (halves, saturating)
+__device__ __forceinline__ void store32_kv(kv16* dst, const float* v, int n_valid) {
+#pragma unroll
+  for (int g = 0; g < 4; ++g)
+    if (g * 8 < n_valid) {
+      uint4 u;
+      uint32_t* w = &u.x;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const __half2 h = __floats2half2_rn(fminf(fmaxf(v[g * 8 + 2 * i], -65504.f), 65504.f),
+                                            fminf(fmaxf(v[g * 8 + 2 * i + 1], -65504.f), 65504.f));
+        w[i] = *reinterpret_cast<const uint32_t*>(&h);
+      }
+      *reinterpret_cast<uint4*>(dst + g * 8) = u;
+    }
 }
 __device__ __forceinline__ void store32_bf16(bf16* dst, const float* v, int n_valid) {
 #pragma unroll
@@ -156,10 +88,16 @@ struct Params {
   int ffn;               // SwiGLU: output width
   const float* q_gain; const float* k_gain; int q_cols; float eps;   // TC_QKV: query / key norm (null = off)
   PagedOut paged;
+  // RMSNorm folded into its neighbours.  Producer (TC_RESID with H): once an element of X is final the epilogue also
+  // writes the next GEMM's operand H = bf16(X * gain_next) (+ its bf16 remainder H_lo) and adds the row's share of
+  // sum X^2 to ss_out[m].  Consumer (TC_QKV / TC_SWIGLU with ss_in): every row of the accumulator is scaled by
+  // rsqrt(ss_in[m] / K + rms_eps), which is the norm's 1 / rms applied after the product instead of before it.
+  bf16* H; bf16* H_lo; int ldh; const float* gain_next; float* ss_out; int* tile_cnt;
+  const float* ss_in; float rms_eps;
 };
 
 // ---- work list: every role of a CTA walks the same sequence of (tile, k-block range) ---------
-struct Work { int m0, n0, kb0, kb1; };
+struct Work { int m0, n0, kb0, kb1, tile; };
 
 template <int BN>
 struct Sched {
@@ -182,6 +120,7 @@ struct Sched {
     const int gm = min(GROUP_M, tiles_m - grp * GROUP_M);
     w.m0 = (grp * GROUP_M + r % gm) * BM;
     w.n0 = (r / gm) * BN;
+    w.tile = t;
   }
   __device__ __forceinline__ bool next(Work& w) {
     if (p.stream_k) {
@@ -206,12 +145,33 @@ __device__ __forceinline__ void red_add4(float* dst, float a, float b, float c, 
   asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
 
+// Fused-norm producer, 32 final values of X (row m, columns n ..): operand of the next GEMM and sum of squares.
+__device__ __forceinline__ float norm_out32(const Params& p, int m, int n, int n_valid, float* v) {
+  float ss = 0.f;
+#pragma unroll
+  for (int i = 0; i < 32; ++i) {
+    const bool in = i < n_valid;
+    ss = fmaf(in ? v[i] : 0.f, v[i], ss);
+    v[i] = in ? v[i] * p.gain_next[n + i] : 0.f;
+  }
+  bf16* h = p.H + (size_t)m * p.ldh + n;
+  store32_bf16(h, v, n_valid);
+  if (p.H_lo) {
+    bf16* lo = p.H_lo + (size_t)m * p.ldh + n;
+#pragma unroll
+    for (int g = 0; g < 4; ++g)
+      if (g * 8 < n_valid) *reinterpret_cast<uint4*>(lo + g * 8) = pack8_lo(v + g * 8);
+  }
+  return ss;
+}
+
 // ---- epilogues: one thread owns one output row of the tile ---------------------------------
 template <int EPI, int BN>
 __device__ __forceinline__ void epilogue_tile(const Params& p, uint32_t tmem_acc, int m, int n0, bool row_ok) {
   // tmem_acc already carries this warp's lane quarter in its upper half
   if (EPI == TC_STORE || EPI == TC_RESID || EPI == TC_PAGED) {
     int slot = -1;
+    float row_ss = 0.f;
     if (EPI == TC_PAGED && row_ok) slot = p.paged.tok_slot[m];
 #pragma unroll 1
     for (int c = 0; c < BN; c += 32) {
@@ -226,9 +186,21 @@ __device__ __forceinline__ void epilogue_tile(const Params& p, uint32_t tmem_acc
         store32_bf16(p.C + (size_t)m * p.ldc + n, v, n_valid);
       } else if (EPI == TC_RESID) {
         float* x = p.X + (size_t)m * p.ldx + n;
+        if (p.H && !p.stream_k) {     // this CTA alone owns the tile: plain read-modify-write, the final value is known here
 #pragma unroll
-        for (int g = 0; g < 8; ++g)
-          if (g * 4 < n_valid) red_add4(x + 4 * g, v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+          for (int g = 0; g < 8; ++g)
+            if (g * 4 < n_valid) {
+              float4 o = *reinterpret_cast<const float4*>(x + 4 * g);
+              o.x += v[4 * g]; o.y += v[4 * g + 1]; o.z += v[4 * g + 2]; o.w += v[4 * g + 3];
+              *reinterpret_cast<float4*>(x + 4 * g) = o;
+              v[4 * g] = o.x; v[4 * g + 1] = o.y; v[4 * g + 2] = o.z; v[4 * g + 3] = o.w;
+            }
+          row_ss += norm_out32(p, m, n, n_valid, v);
+        } else {
+#pragma unroll
+          for (int g = 0; g < 8; ++g)
+            if (g * 4 < n_valid) red_add4(x + 4 * g, v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+        }
       } else {
         if (slot < 0) continue;
         const PagedOut& q = p.paged;
@@ -241,12 +213,14 @@ __device__ __forceinline__ void epilogue_tile(const Params& p, uint32_t tmem_acc
           for (int i = 0; i < 32; ++i) v[i] += q.bias[n + i];
         }
         int page = slot / PAGE_TOKENS, row = slot - page * PAGE_TOKENS;
-        bf16* dst = (bf16*)q.pool[s] + (((size_t)page * q.n_kv[s] + head) * PAGE_TOKENS + row) * q.head_dim + dim;
-        store32_bf16(dst, v, n_valid);
+        kv16* dst = (kv16*)q.pool[s] + (((size_t)page * q.n_kv[s] + head) * PAGE_TOKENS + row) * q.head_dim + dim;
+        store32_kv(dst, v, n_valid);
       }
     }
+    if (EPI == TC_RESID && p.H && !p.stream_k && row_ok) atomicAdd(p.ss_out + m, row_ss);
   } else if (EPI == TC_SWIGLU) {
     // every 128 columns of the tile: [0, 64) gate rows, [64, 128) the matching up rows
+    const float rinv = (p.ss_in && row_ok) ? rsqrtf(p.ss_in[m] / (float)p.K + p.rms_eps) : 1.f;
 #pragma unroll 1
     for (int c = 0; c < BN / 2; c += 32) {
       int grp = c >> 6, cc = c & 63;
@@ -259,12 +233,13 @@ __device__ __forceinline__ void epilogue_tile(const Params& p, uint32_t tmem_acc
       tmem_ld_wait();
       if (!row_ok) continue;
 #pragma unroll
-      for (int i = 0; i < 32; ++i) g[i] = __fdividef(g[i], 1.f + __expf(-g[i])) * u[i];
+      for (int i = 0; i < 32; ++i) { const float gi = g[i] * rinv; g[i] = __fdividef(gi, 1.f + __expf(-gi)) * (u[i] * rinv); }
       store32_bf16(p.C + (size_t)m * p.ldc + n, g, n_valid);
     }
   } else {  // TC_QKV: RoPE on columns < rot_cols, hi part to C, lo part of columns >= lo_col_begin to C_lo
     int half = p.hd >> 1;
     const float2* tab = row_ok ? p.rope_tab + (size_t)p.tok_pos[m] * half : nullptr;
+    const float rinv = (p.ss_in && row_ok) ? rsqrtf(p.ss_in[m] / (float)p.K + p.rms_eps) : 1.f;
 #pragma unroll 1
     for (int h0 = 0; h0 < BN; h0 += p.hd) {
       if (n0 + h0 >= p.N) break;
@@ -281,7 +256,7 @@ __device__ __forceinline__ void epilogue_tile(const Params& p, uint32_t tmem_acc
 #pragma unroll
           for (int i = 0; i < 32; ++i) ss = fmaf(a[i], a[i], ss);
         }
-        rn = rsqrtf(ss / (float)p.hd + p.eps);
+        rn = rsqrtf(ss * rinv * rinv / (float)p.hd + p.eps);
       }
 #pragma unroll 1
       for (int j = 0; j < half; j += 32) {
@@ -291,6 +266,10 @@ __device__ __forceinline__ void epilogue_tile(const Params& p, uint32_t tmem_acc
         tmem_ld_wait();
         int n = n0 + h0 + j;
         if (!row_ok) continue;
+        if (p.ss_in) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) { a[i] *= rinv; b[i] *= rinv; }
+        }
         if (gain) {
 #pragma unroll
           for (int i = 0; i < 32; ++i) { a[i] *= rn * gain[j + i]; b[i] *= rn * gain[half + j + i]; }
@@ -330,33 +309,35 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
-  // bars: full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2]; then tmem base, abort flag
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+  // bars: full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], fin; then tmem base, abort flag, last-share flag
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 5);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  volatile int* s_last = reinterpret_cast<volatile int*>(tmem_slot + 2);
   const uint32_t smem_base = smem_u32(smem);
   const uint32_t bar_base = smem_u32(bars);
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
   auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
   auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
+  const uint32_t fin_bar = bar_base + 8u * (2 * STAGES + 4);      // the four epilogue warps meet here (stream-K with fused norm)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   pdl_trigger();      // the next kernel's CTAs may take SMs as this kernel's CTAs leave them
   if (threadIdx.x == 32) {   // tensor maps on their way while the barriers and tensor memory are set up
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
-    if (p.has_a2) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a2) : "memory");
+    prefetch_tensormap(&map_a);
+    prefetch_tensormap(&map_w);
+    if (p.has_a2) prefetch_tensormap(&map_a2);
   }
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 2); mbar_init(empty_bar(s), 1); }   // two loaders per stage
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+    mbar_init(fin_bar, 4);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {   // tensor memory: two accumulators of BN columns
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(2 * BN) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    tmem_alloc(smem_u32(tmem_slot), 2 * BN);
   }
   tc_fence_before();
   __syncthreads();
@@ -389,9 +370,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
       }
-      if (!ok) {   // aborting: give copies already issued time to land before the CTA's memory goes away
-        for (int i = 0; i < 2000; ++i) __nanosleep(1000);
-      }
+      if (!ok) drain_after_abort();
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
@@ -412,7 +391,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           if (!ok) break;
           tc_fence_after();
           const uint32_t sa = smem_base + stage * STAGE_BYTES, sb = sa + T::A_BYTES;
-          const uint64_t da = make_desc(sa), db = make_desc(sb);
+          const uint64_t da = desc_kmajor(sa), db = desc_kmajor(sb);
 #pragma unroll
           for (int k = 0; k < BK / 16; ++k)
             tc_mma_bf16(d_tmem, da + 2u * k, db + 2u * k, idesc, (it > w.kb0 || k > 0) ? 1u : 0u);
@@ -422,16 +401,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (ok) tc_commit(tfull_bar(acc));    // accumulator complete
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
       }
-      if (!ok) {
-        for (int i = 0; i < 2000; ++i) __nanosleep(1000);
-      }
+      if (!ok) drain_after_abort();
     }
   } else {
     // ---------------- epilogue: 4 warps, each owns the 32 tensor-memory lanes of its quarter ----------------
     const int quarter = warp & 3;
     Sched<BN> sched(p);
     Work w;
-    int acc = 0; uint32_t acc_phase = 0;
+    int acc = 0; uint32_t acc_phase = 0, fin_phase = 0;
     bool ok = true;
     while (sched.next(w)) {
       ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status);
@@ -445,48 +422,70 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar(acc));
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      if (EPI == TC_RESID && p.H && p.stream_k) {
+        // A tile's k blocks are shared among CTAs that add their partial sums with red.global.  Each share counts
+        // its k blocks into the tile's counter once its adds are globally visible; the share that completes the
+        // count re-reads the finished tile (from L2) and writes the next GEMM's operand and the rows' sums of squares.
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(fin_bar);
+        ok = mbar_wait(fin_bar, fin_phase, abort_flag, p.status);
+        fin_phase ^= 1u;
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        if (quarter == 3 && lane == 0) {
+          const int add = w.kb1 - w.kb0;
+          *s_last = (atomicAdd(p.tile_cnt + w.tile, add) + add == num_kb) ? 1 : 0;
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(fin_bar);
+        ok = mbar_wait(fin_bar, fin_phase, abort_flag, p.status);
+        fin_phase ^= 1u;
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        if (*s_last) {
+          __threadfence();
+          if (m < p.M) {
+            float row_ss = 0.f;
+#pragma unroll 1
+            for (int c = 0; c < BN; c += 32) {
+              const int n = w.n0 + c, n_valid = p.N - n;
+              if (n_valid <= 0) break;
+              float v[32];
+              const float* x = p.X + (size_t)m * p.ldx + n;
+#pragma unroll
+              for (int g = 0; g < 8; ++g) {
+                float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (g * 4 < n_valid) o = __ldcg(reinterpret_cast<const float4*>(x + 4 * g));
+                v[4 * g] = o.x; v[4 * g + 1] = o.y; v[4 * g + 2] = o.z; v[4 * g + 3] = o.w;
+              }
+              row_ss += norm_out32(p, m, n, n_valid, v);
+            }
+            atomicAdd(p.ss_out + m, row_ss);
+          }
+        }
+      }
     }
   }
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2 * BN) : "memory");
+    tmem_dealloc(tmem_base, 2 * BN);
   }
 }
 
 // ---- host side ----------------------------------------------------------------------------
-PFN_cuTensorMapEncodeTiled_v12000 g_encode = nullptr;
-
-bool get_encode() {
-  if (g_encode) return true;
-  void* fn = nullptr;
-  cudaDriverEntryPointQueryResult q;
-  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn) return false;
-  g_encode = (PFN_cuTensorMapEncodeTiled_v12000)fn;
-  return true;
-}
-
 // bf16 [rows, cols] row-major with row stride ld elements; box = 64 columns x box_rows rows, 128B swizzle
 bool make_map(CUtensorMap* m, const void* base, int rows, int cols, int ld, int box_rows) {
-  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-  cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
-  cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  CUresult r = g_encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS;
+  return tc_make_map_bf16(m, base, rows, cols, ld, box_rows);
 }
 
 template <int EPI, int BN>
 cudaError_t go(const CUtensorMap& a, const CUtensorMap& a2, const CUtensorMap& w, const Params& p, int grid, cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<EPI, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Tile<BN>::SMEM_BYTES);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static bool raised[TC_MAX_DEVICES] = {};
+  cudaError_t e = tc_raise_smem_limit(gemm_tc_kernel<EPI, BN>, Tile<BN>::SMEM_BYTES, raised);
+  if (e != cudaSuccess) return e;
   return launch_overlapped(gemm_tc_kernel<EPI, BN>, dim3(grid), dim3(N_THREADS), Tile<BN>::SMEM_BYTES, st, a, a2, w, p);
 }
 
@@ -521,7 +520,9 @@ bool tc_gemm_supported(const TcGemm& g) {
   if (g.A2 && (g.lda2 % 8 || !al16(g.A2))) return false;
   switch (g.epi) {
     case TC_STORE: return g.N % 8 == 0 && g.ldc % 8 == 0 && al16(g.C);
-    case TC_RESID: return g.N % 4 == 0 && g.ldx % 4 == 0 && al16(g.X);
+    case TC_RESID:
+      if (g.H && (g.N % 8 || g.ldh % 8 || !al16(g.H) || (g.H_lo && !al16(g.H_lo)) || !g.gain_next || !g.ss_out || !g.tile_cnt)) return false;
+      return g.N % 4 == 0 && g.ldx % 4 == 0 && al16(g.X);
     case TC_SWIGLU: return g.ffn % 64 == 0 && g.N == 2 * g.ffn && g.ldc % 8 == 0 && al16(g.C);
     case TC_QKV:
       return (g.hd == 64 || g.hd == 128) && g.N % g.hd == 0 && g.rot_cols % g.hd == 0 && g.lo_col_begin % g.hd == 0 &&
@@ -537,7 +538,7 @@ bool tc_gemm_supported(const TcGemm& g) {
 }
 
 cudaError_t launch_gemm_tc(const TcGemm& g, int* status, cudaStream_t st, int64_t* n_launch) {
-  if (!get_encode()) return cudaErrorNotSupported;
+  if (!tc_encode_fn()) return cudaErrorNotSupported;
   const int tiles128 = ((g.M + BM - 1) / BM) * ((g.N + 127) / 128);
   const bool stream_k = g.epi == TC_RESID && !g.A2 && tiles128 < 2 * g.n_sm;
   int bn = g.bn;
@@ -553,6 +554,8 @@ cudaError_t launch_gemm_tc(const TcGemm& g, int* status, cudaStream_t st, int64_
   p.C = g.C; p.ldc = g.ldc; p.X = g.X; p.ldx = g.ldx; p.C_lo = g.C_lo; p.ld_lo = g.ld_lo; p.lo_col_begin = g.lo_col_begin;
   p.q_gain = g.q_gain; p.k_gain = g.k_gain; p.q_cols = g.q_cols; p.eps = g.eps;
   p.rot_cols = g.rot_cols; p.hd = g.hd; p.rope_tab = g.rope_tab; p.tok_pos = g.tok_pos; p.ffn = g.ffn; p.paged = g.paged;
+  p.H = g.H; p.H_lo = g.H_lo; p.ldh = g.ldh; p.gain_next = g.gain_next; p.ss_out = g.ss_out; p.tile_cnt = g.tile_cnt;
+  p.ss_in = g.ss_in; p.rms_eps = g.rms_eps;
   const int tiles = ((g.M + BM - 1) / BM) * ((g.N + bn - 1) / bn);
   const long long kblocks = (long long)tiles * ((g.K + BK - 1) / BK);
   int grid = stream_k ? (int)(kblocks < g.n_sm ? kblocks : g.n_sm) : (tiles < g.n_sm ? tiles : g.n_sm);

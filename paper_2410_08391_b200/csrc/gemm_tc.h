@@ -28,6 +28,13 @@ struct TcGemm {
   // heads (gain k_gain); null gains = no norm
   const float* q_gain; const float* k_gain; int q_cols; float eps;
   PagedOut paged;
+  // RMSNorm folded into the neighbouring GEMMs (all null / 0 = off).
+  // TC_RESID with H: besides X += A W^T the epilogue writes H[m, n] = bf16(X[m, n] * gain_next[n]) (row stride ldh;
+  // H_lo = the bf16 remainder, or null) and adds the row's share of sum_n X[m, n]^2 to ss_out[m] (cleared by the
+  // caller); tile_cnt: one zeroed int per 128 x 128 output tile of this launch, used when tiles are shared among CTAs.
+  // TC_QKV / TC_SWIGLU with ss_in: the accumulator rows are scaled by rsqrt(ss_in[m] / K + rms_eps).
+  bf16* H; bf16* H_lo; int ldh; const float* gain_next; float* ss_out; int* tile_cnt;
+  const float* ss_in; float rms_eps;
   int n_sm;
   int bn;                          // tile width: 128, 256, or 0 = chosen by the launcher
 };

@@ -201,7 +201,7 @@ bool ends_with(const std::string& s, const char* suf) {
 
 // Tries the tcgen05 GEMM; returns false when the shape is not one it takes (caller falls back).
 bool try_tc(kvp_handle* h, const LaunchCtx& ctx, TcGemm& t, int cls, cudaError_t* err) {
-  if (!h->use_tc || h->opt.dtype != KVP_BF16) return false;
+  if (h->opt.dtype != KVP_BF16) return false;
   t.n_sm = h->gemm_sms;
   if (!tc_gemm_supported(t)) return false;
   TimedScope ts(h, ctx.st, cls);
@@ -213,7 +213,7 @@ bool try_tc(kvp_handle* h, const LaunchCtx& ctx, TcGemm& t, int cls, cudaError_t
 // Are the step's projections run on the tensor cores?  (Everything the persistent kernel does not take:
 // batches of more than 4 rows, and small batches over long caches.)
 bool step_uses_tc(const kvp_handle* h, int batch) {
-  if (!h->use_tc || h->opt.dtype != KVP_BF16 || step_tc_rows(batch) > 128) return false;
+  if (h->opt.dtype != KVP_BF16 || step_tc_rows(batch) > 128) return false;
   const ModelPlan& B = h->base;
   if (B.d % 8) return false;
   for (int i = 0; i < B.n_layers; ++i)
@@ -282,7 +282,7 @@ bool mega_prepare(kvp_handle* h, const LaunchCtx& ctx, const kvp_cache* cache, c
   // its attention phase reads cache pages with plain loads: fine for a few thousand keys, several times
   // slower than the ring-fed kernel beyond that
   if (max_keys > 4096) return false;
-  if (!h->use_mega || B.n_layers > MEGA_MAX_LAYERS || !step_mega_supported(batch, B.L[0].hd, k_max, B.max_group, h->es)) return false;
+  if (B.n_layers > MEGA_MAX_LAYERS || !step_mega_supported(batch, B.L[0].hd, k_max, B.max_group, h->es)) return false;
   // bulk copies need 16-byte rows: every projection's row length must be a multiple of 16 bytes
   for (int i = 0; i < B.n_layers; ++i)
     if ((B.d * h->es) % 16 || (B.L[i].dq * h->es) % 16 || (B.L[i].ffn * h->es) % 16) return false;
@@ -299,7 +299,11 @@ bool mega_prepare(kvp_handle* h, const LaunchCtx& ctx, const kvp_cache* cache, c
   p.part = (float*)(ws + w.part);
   p.attn_done = (int*)(ws + w.attn_done);
   p.logits = logits; p.token_out = token_out; p.status = ctx.status;
-  p.trace = getenv("KVP_MEGA_TRACE") ? (long long*)((char*)ctx.status + 256) : nullptr;
+#ifdef KVP_MEGA_TRACE     // build-time diagnostic: per-phase clocks of the persistent step kernel, from byte 256 of the status block
+  p.trace = (long long*)((char*)ctx.status + 256);
+#else
+  p.trace = nullptr;
+#endif
   int min_nkv = B.L[0].nkv;
   for (int i = 0; i < B.n_layers; ++i) {
     const LayerPlan& L = B.L[i];
@@ -407,11 +411,7 @@ kvp_status kvp_create(const kvp_model_cfg* aux, const kvp_model_cfg* base, const
     if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, h->device) == cudaSuccess && n > 0) h->n_sm = n;
   }
   cudaGetLastError();
-  if (const char* e = getenv("KVP_NO_TC")) h->use_tc = !(e[0] == '1');
-  if (const char* e = getenv("KVP_NO_GRAPH")) h->use_graph = !(e[0] == '1');
-  if (const char* e = getenv("KVP_NO_MEGA")) h->use_mega = !(e[0] == '1');
-  if (const char* e = getenv("KVP_NO_SIDE")) h->use_side = !(e[0] == '1');
-  if (h->use_side) {
+  {
     if (cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking) != cudaSuccess) h->side = nullptr;
     if (h->side && (cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
                     cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming) != cudaSuccess)) {
@@ -421,9 +421,7 @@ kvp_status kvp_create(const kvp_model_cfg* aux, const kvp_model_cfg* base, const
     cudaGetLastError();
   }
   h->gemm_sms = h->step_grid_sms = h->n_sm;
-  if (const char* e = getenv("KVP_STEP_TC_SMS")) h->step_tc_sms = atoi(e);
   if (h->step_tc_sms < 8 || h->step_tc_sms > h->n_sm) h->step_tc_sms = 0;
-  if (const char* e = getenv("KVP_STEP_SMS")) h->step_sms = atoi(e);
   if (h->step_sms < 8 || h->step_sms > h->n_sm - 32 || !h->side) h->step_sms = 0;
   if (h->step_sms) {
     if (cudaStreamCreateWithFlags(&h->step_st, cudaStreamNonBlocking) != cudaSuccess) h->step_st = nullptr;
@@ -600,7 +598,7 @@ static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int
   for (int j = 0; j <= h->j_max; ++j) max_nq = std::max(max_nq, A.L[j].nq);
   const int attn_tiles = attn_tc_items(cs.cu.data(), batch, 2) * max_nq < h->n_sm ? 1 : 2;
   const int attn_items = attn_tc_items(cs.cu.data(), batch, attn_tiles);
-  if (h->use_tc && h->opt.dtype == KVP_BF16 && (A.L[0].hd == 64 || A.L[0].hd == 128)) {
+  if (h->opt.dtype == KVP_BF16 && (A.L[0].hd == 64 || A.L[0].hd == 128)) {
     KVP_TIMED(KVP_CLASS_OTHER, launch_rope_table(ctx, rope_tab, cs.max_len, A.L[0].hd, A.theta));
     KVP_TIMED(KVP_CLASS_OTHER, launch_attn_schedule(cu_dev, batch, attn_tiles, attn_sched, ctx.st, ctx.n_launch));
   }
@@ -732,7 +730,7 @@ static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int
       }
     }
     if (last) break;
-    if (h->use_tc && split && attn_items <= 65535 && attn_tc_supported(L.hd, L.nqkv, qkv, L.dq, attn)) {
+    if (split && attn_items <= 65535 && attn_tc_supported(L.hd, L.nqkv, qkv, L.dq, attn)) {
       TimedScope ts(h, ctx.st, KVP_CLASS_AUX_ATTN);
       cudaError_t e = launch_attn_tc((const bf16*)qkv, L.nqkv, T, L.nq, L.nkv, L.hd, cu_dev, attn_sched, attn_items, attn_tiles, (bf16*)attn,
                                      L.dq, ctx.status, ctx.st, ctx.n_launch);
@@ -1031,7 +1029,7 @@ extern "C" kvp_status kvp_train_forward(kvp_handle* h, const int32_t* tokens, co
   for (int i = 0; i < B.n_layers; ++i) max_nq = std::max(max_nq, B.L[i].nq);
   const int attn_tiles = attn_tc_items(cs.cu.data(), batch, 2) * max_nq < h->n_sm ? 1 : 2;
   const int attn_items = attn_tc_items(cs.cu.data(), batch, attn_tiles);
-  if (h->use_tc && h->opt.dtype == KVP_BF16 && (B.L[0].hd == 64 || B.L[0].hd == 128)) {
+  if (h->opt.dtype == KVP_BF16 && (B.L[0].hd == 64 || B.L[0].hd == 128)) {
     launch_rope_table(ctx, rope_tab, cs.max_len, B.L[0].hd, B.theta);
     launch_attn_schedule(cu_dev, batch, attn_tiles, attn_sched, ctx.st, ctx.n_launch);
   }
@@ -1070,7 +1068,7 @@ extern "C" kvp_status kvp_train_forward(kvp_handle* h, const int32_t* tokens, co
       } else {
         launch_kv_take(ctx, qkv, L.nqkv, L.dq, T, L.nkv, L.hd, tok_slot, cache->k_pools[i], cache->v_pools[i]);
       }
-      if (h->use_tc && split && attn_items <= 65535 && attn_tc_supported(L.hd, L.nqkv, qkv, L.dq, attn)) {
+      if (split && attn_items <= 65535 && attn_tc_supported(L.hd, L.nqkv, qkv, L.dq, attn)) {
         cudaError_t e = launch_attn_tc((const bf16*)qkv, L.nqkv, T, L.nq, L.nkv, L.hd, cu_dev, attn_sched, attn_items, attn_tiles,
                                        (bf16*)attn, L.dq, ctx.status, ctx.st, ctx.n_launch);
         if (e != cudaSuccess && tc_err == cudaSuccess) tc_err = e;

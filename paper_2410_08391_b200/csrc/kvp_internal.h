@@ -64,20 +64,17 @@ struct kvp_handle {
   char* packed = nullptr;
   int device = 0;
   int n_sm = 148;
-  bool use_tc = true;                   // tcgen05 kernels for bf16 shapes they accept
   int64_t n_launch = 0;
   std::string err;
   // captured kernel schedules of kvp_prefill_predict, keyed by every argument that is baked in
   struct GraphEntry { std::vector<uint64_t> key; cudaGraphExec_t exec; int64_t launches; uint64_t last_use; };
   std::vector<GraphEntry> graphs;
   bool use_graph = true;
-  bool use_mega = true;                 // persistent kernel for the base step when it applies
   uint64_t graph_clock = 0;
   // The predictor GEMMs of an auxiliary layer depend only on that layer's K/V projection, so they
   // run on a stream of the handle's own beside the layer's attention and FFN (fork / join by events).
   cudaStream_t side = nullptr;
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
-  bool use_side = true;
   // The base step at small batch is one persistent kernel bound by HBM latency, the auxiliary prefill a chain
   // of tensor-core kernels: base layer i only needs the predicted cache of layers <= i, so the step runs in
   // pieces (one per auxiliary layer that completes some base layers' cache) on a stream of its own, on

@@ -42,7 +42,23 @@ extern "C" kvp_status kvp_decode_step_static(kvp_handle* h, const int32_t* token
     h->err = "kvp_decode_step_static: no usable current device";
     return KVP_ERR_CUDA;
   }
-  if (!g_scratch_addr[dev]) {   // set-up, once per device, with that device current
+  // nothing touches the array or the stream before the arguments have been checked
+  if (dev != h->device) {
+    h->err = "kvp_decode_step_static: the current device is not the handle's device";
+    return KVP_ERR_INVALID_ARG;
+  }
+  if (!tokens || !lengths_host || !cache || !logits_out || !cache->k_pools || !cache->v_pools || !cache->block_table ||
+      !cache->seq_lens) {
+    h->err = "kvp_decode_step_static: NULL argument";
+    return KVP_ERR_INVALID_ARG;
+  }
+  if (!h->ready_decode) {
+    h->err = "kvp_load_weights has not supplied every required tensor";
+    return KVP_ERR_NOT_LOADED;
+  }
+  // Set-up, once per device, with that device current.  Two threads making their first call on a device at the
+  // same moment both look the address up and store the same value.
+  if (!g_scratch_addr[dev]) {
     void* p = nullptr;
     cudaError_t e = cudaGetSymbolAddress(&p, g_step_scratch);
     if (e != cudaSuccess || !p) {

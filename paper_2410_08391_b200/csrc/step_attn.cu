@@ -1,4 +1,4 @@
-// Single-query GQA attention of the base step over the paged bf16 cache, bandwidth-bound variants.
+// Single-query GQA attention of the base step over the paged 16-bit (half) cache, bandwidth-bound variants.
 //
 // grid (key-range split, kv head, sequence); a CTA serves the `group` query heads that share one
 // kv head and walks its range of cache pages.  A page of one kv head is one contiguous block
@@ -30,39 +30,20 @@
 #include <math.h>
 
 #include "common.cuh"
+#include "tc_ptx.cuh"
 
 namespace {
+using namespace tcp;
 
 constexpr int ST = 3;                       // pages in flight per CTA (K and V each)
 constexpr int MAXG = 8;
 constexpr int MAX_IDS = 512;                // page ids a CTA keeps in shared memory
-constexpr uint32_t SPIN_LIMIT = 20u * 1000u * 1000u;
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
 
 template <int HD>
 __global__ void __launch_bounds__(512) step_attn_ring_wide_kernel(const float* __restrict__ q, int ldq, int nq, int nkv,
                                                              const __grid_constant__ InvFreq inv,
-                                                             const bf16* __restrict__ kpool, const bf16* __restrict__ vpool,
+                                                             const kv16* __restrict__ kpool, const kv16* __restrict__ vpool,
                                                              const int* __restrict__ block_table, int mpps, int n_pages,
                                                              const int* __restrict__ seq_lens, int extra, int n_split,
                                                              float* __restrict__ part, float* __restrict__ out, int* status,
@@ -164,10 +145,10 @@ __global__ void __launch_bounds__(512) step_attn_ring_wide_kernel(const float* _
         const int c = (i + key) & (CH - 1);
         const uint4 u = *reinterpret_cast<const uint4*>(kr + c * 16);
         const float4 q0 = *reinterpret_cast<const float4*>(qh + c * 8), q1 = *reinterpret_cast<const float4*>(qh + c * 8 + 4);
-        s0 = fmaf(__uint_as_float(u.x << 16), q0.x, s0); s1 = fmaf(__uint_as_float(u.x & 0xffff0000u), q0.y, s1);
-        s2 = fmaf(__uint_as_float(u.y << 16), q0.z, s2); s3 = fmaf(__uint_as_float(u.y & 0xffff0000u), q0.w, s3);
-        s0 = fmaf(__uint_as_float(u.z << 16), q1.x, s0); s1 = fmaf(__uint_as_float(u.z & 0xffff0000u), q1.y, s1);
-        s2 = fmaf(__uint_as_float(u.w << 16), q1.z, s2); s3 = fmaf(__uint_as_float(u.w & 0xffff0000u), q1.w, s3);
+        s0 = fmaf(kv_lo(u.x), q0.x, s0); s1 = fmaf(kv_hi(u.x), q0.y, s1);
+        s2 = fmaf(kv_lo(u.y), q0.z, s2); s3 = fmaf(kv_hi(u.y), q0.w, s3);
+        s0 = fmaf(kv_lo(u.z), q1.x, s0); s1 = fmaf(kv_hi(u.z), q1.y, s1);
+        s2 = fmaf(kv_lo(u.w), q1.z, s2); s3 = fmaf(kv_hi(u.w), q1.w, s3);
       }
       ps[h * PAGE_TOKENS + key] = key < nk ? (s0 + s1) + (s2 + s3) : -INFINITY;
     }
@@ -201,24 +182,24 @@ __global__ void __launch_bounds__(512) step_attn_ring_wide_kernel(const float* _
         for (; s + 2 <= nk; s += 2) {
           const uint32_t u = vr[s * (HD / 2)], w = vr[(s + 1) * (HD / 2)];
           const float pu = pr[s], pw = pr[s + 1];
-          a0 = fmaf(pu, __uint_as_float(u << 16), a0); a1 = fmaf(pu, __uint_as_float(u & 0xffff0000u), a1);
-          b0 = fmaf(pw, __uint_as_float(w << 16), b0); b1 = fmaf(pw, __uint_as_float(w & 0xffff0000u), b1);
+          a0 = fmaf(pu, kv_lo(u), a0); a1 = fmaf(pu, kv_hi(u), a1);
+          b0 = fmaf(pw, kv_lo(w), b0); b1 = fmaf(pw, kv_hi(w), b1);
         }
         if (s < nk) {
           const uint32_t u = vr[s * (HD / 2)];
-          a0 = fmaf(pr[s], __uint_as_float(u << 16), a0); a1 = fmaf(pr[s], __uint_as_float(u & 0xffff0000u), a1);
+          a0 = fmaf(pr[s], kv_lo(u), a0); a1 = fmaf(pr[s], kv_hi(u), a1);
         }
         acc[0] = a0 + b0; acc[DP - 1] = a1 + b1;
       } else {
         float a0 = acc[0] * a, b0 = 0.f, c0 = 0.f, d0 = 0.f;
-        const bf16* vr = reinterpret_cast<const bf16*>(Vs) + key;
+        const kv16* vr = reinterpret_cast<const kv16*>(Vs) + key;
         int s = 0;
 #pragma unroll 2
         for (; s + 4 <= nk; s += 4) {
-          a0 = fmaf(pr[s], __bfloat162float(vr[s * HD]), a0); b0 = fmaf(pr[s + 1], __bfloat162float(vr[(s + 1) * HD]), b0);
-          c0 = fmaf(pr[s + 2], __bfloat162float(vr[(s + 2) * HD]), c0); d0 = fmaf(pr[s + 3], __bfloat162float(vr[(s + 3) * HD]), d0);
+          a0 = fmaf(pr[s], __half2float(vr[s * HD]), a0); b0 = fmaf(pr[s + 1], __half2float(vr[(s + 1) * HD]), b0);
+          c0 = fmaf(pr[s + 2], __half2float(vr[(s + 2) * HD]), c0); d0 = fmaf(pr[s + 3], __half2float(vr[(s + 3) * HD]), d0);
         }
-        for (; s < nk; ++s) a0 = fmaf(pr[s], __bfloat162float(vr[s * HD]), a0);
+        for (; s < nk; ++s) a0 = fmaf(pr[s], __half2float(vr[s * HD]), a0);
         acc[0] = (a0 + b0) + (c0 + d0);
       }
     }
@@ -263,7 +244,7 @@ struct RingCfg {
 template <int HD, int GP>
 __global__ void __launch_bounds__(RingCfg<HD, GP>::NT, RingCfg<HD, GP>::NT == 512 ? 1 : 2)
 step_attn_ring_kernel(const float* __restrict__ q, int ldq, int nq, int nkv, const __grid_constant__ InvFreq inv,
-                      const bf16* __restrict__ kpool, const bf16* __restrict__ vpool, const int* __restrict__ block_table,
+                      const kv16* __restrict__ kpool, const kv16* __restrict__ vpool, const int* __restrict__ block_table,
                       int mpps, int n_pages, const int* __restrict__ seq_lens, int extra, int n_split,
                       float* __restrict__ part, float* __restrict__ out, int* status, const float* __restrict__ q_gain,
                       float eps, int* __restrict__ split_done) {
@@ -397,10 +378,10 @@ step_attn_ring_kernel(const float* __restrict__ q, int ldq, int nq, int nkv, con
       for (int i = 0; i < CPT; ++i) {
         const int c = dq + DS * ((i + key) % CPT);
         const uint4 u = *reinterpret_cast<const uint4*>(kr + c * 16);
-        const float k0 = __uint_as_float(u.x << 16), k1 = __uint_as_float(u.x & 0xffff0000u);
-        const float k2 = __uint_as_float(u.y << 16), k3 = __uint_as_float(u.y & 0xffff0000u);
-        const float k4 = __uint_as_float(u.z << 16), k5 = __uint_as_float(u.z & 0xffff0000u);
-        const float k6 = __uint_as_float(u.w << 16), k7 = __uint_as_float(u.w & 0xffff0000u);
+        const float k0 = kv_lo(u.x), k1 = kv_hi(u.x);
+        const float k2 = kv_lo(u.y), k3 = kv_hi(u.y);
+        const float k4 = kv_lo(u.z), k5 = kv_hi(u.z);
+        const float k6 = kv_lo(u.w), k7 = kv_hi(u.w);
 #pragma unroll
         for (int g = 0; g < GP; ++g) {
           float t0 = fmaf(k0, qr[g][i][0], s[g]), t1 = k1 * qr[g][i][1];
@@ -465,7 +446,7 @@ step_attn_ring_kernel(const float* __restrict__ q, int ldq, int nq, int nkv, con
 #pragma unroll 4
       for (int s = kq * KPT; s < s1; ++s) {
         const uint32_t u = vr[s * (HD / 2)];
-        const float v0 = __uint_as_float(u << 16), v1 = __uint_as_float(u & 0xffff0000u);
+        const float v0 = kv_lo(u), v1 = kv_hi(u);
         float pv[4];
         if constexpr (GP == 4) {
           const float4 t = *reinterpret_cast<const float4*>(ps + s * 4);
@@ -544,16 +525,13 @@ step_attn_ring_kernel(const float* __restrict__ q, int ldq, int nq, int nkv, con
 }
 
 template <int HD, int GP>
-cudaError_t go_ring(dim3 grid, cudaStream_t st, const float* q, int ldq, int nq, int nkv, const InvFreq& inv, const bf16* kpool,
-                    const bf16* vpool, const int* block_table, int mpps, int n_pages, const int* seq_lens, int extra, int n_split,
+cudaError_t go_ring(dim3 grid, cudaStream_t st, const float* q, int ldq, int nq, int nkv, const InvFreq& inv, const kv16* kpool,
+                    const kv16* vpool, const int* block_table, int mpps, int n_pages, const int* seq_lens, int extra, int n_split,
                     float* part, float* out, int* status, const float* q_gain, float eps, int* split_done) {
   using Cfg = RingCfg<HD, GP>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(step_attn_ring_kernel<HD, GP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::SMEM);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static bool raised[TC_MAX_DEVICES] = {};
+  cudaError_t e = tc_raise_smem_limit(step_attn_ring_kernel<HD, GP>, (int)Cfg::SMEM, raised);
+  if (e != cudaSuccess) return e;
   step_attn_ring_kernel<HD, GP><<<grid, Cfg::NT, Cfg::SMEM, st>>>(q, ldq, nq, nkv, inv, kpool, vpool, block_table, mpps, n_pages, seq_lens,
                                                                   extra, n_split, part, out, status, q_gain, eps, split_done);
   return cudaGetLastError();
@@ -561,7 +539,7 @@ cudaError_t go_ring(dim3 grid, cudaStream_t st, const float* q, int ldq, int nq,
 
 template <int HD>
 cudaError_t go_ring_hd(int group, dim3 grid, cudaStream_t st, const float* q, int ldq, int nq, int nkv, const InvFreq& inv,
-                       const bf16* kpool, const bf16* vpool, const int* block_table, int mpps, int n_pages, const int* seq_lens,
+                       const kv16* kpool, const kv16* vpool, const int* block_table, int mpps, int n_pages, const int* seq_lens,
                        int extra, int n_split, float* part, float* out, int* status, const float* q_gain, float eps, int* split_done) {
   if (group == 1)
     return go_ring<HD, 1>(grid, st, q, ldq, nq, nkv, inv, kpool, vpool, block_table, mpps, n_pages, seq_lens, extra, n_split, part, out, status, q_gain, eps, split_done);
@@ -571,16 +549,13 @@ cudaError_t go_ring_hd(int group, dim3 grid, cudaStream_t st, const float* q, in
 }
 
 template <int HD>
-cudaError_t go(dim3 grid, int threads, cudaStream_t st, const float* q, int ldq, int nq, int nkv, const InvFreq& inv, const bf16* kpool,
-               const bf16* vpool, const int* block_table, int mpps, int n_pages, const int* seq_lens, int extra, int n_split,
+cudaError_t go(dim3 grid, int threads, cudaStream_t st, const float* q, int ldq, int nq, int nkv, const InvFreq& inv, const kv16* kpool,
+               const kv16* vpool, const int* block_table, int mpps, int n_pages, const int* seq_lens, int extra, int n_split,
                float* part, float* out, int* status, const float* q_gain, float eps) {
   const size_t smem = (size_t)ST * 2 * PAGE_TOKENS * HD * 2 + (size_t)(MAXG * HD + MAXG * PAGE_TOKENS + 3 * MAXG) * sizeof(float);
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(step_attn_ring_wide_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static bool raised[TC_MAX_DEVICES] = {};
+  cudaError_t e = tc_raise_smem_limit(step_attn_ring_wide_kernel<HD>, (int)smem, raised);
+  if (e != cudaSuccess) return e;
   step_attn_ring_wide_kernel<HD><<<grid, threads, smem, st>>>(q, ldq, nq, nkv, inv, kpool, vpool, block_table, mpps, n_pages, seq_lens, extra,
                                                          n_split, part, out, status, q_gain, eps);
   return cudaGetLastError();
@@ -623,14 +598,14 @@ cudaError_t launch_step_attn_ring(const LaunchCtx& ctx, const float* q, int ldq,
   const int group = nq / nkv;
   if (group <= 4) {
     if (hd == 64)
-      return go_ring_hd<64>(group, grid, ctx.st, q, ldq, nq, nkv, inv, (const bf16*)kpool, (const bf16*)vpool, block_table, mpps, n_pages,
+      return go_ring_hd<64>(group, grid, ctx.st, q, ldq, nq, nkv, inv, (const kv16*)kpool, (const kv16*)vpool, block_table, mpps, n_pages,
                             seq_lens, extra, n_split, part, out, ctx.status, q_gain, eps, split_done);
-    return go_ring_hd<128>(group, grid, ctx.st, q, ldq, nq, nkv, inv, (const bf16*)kpool, (const bf16*)vpool, block_table, mpps, n_pages,
+    return go_ring_hd<128>(group, grid, ctx.st, q, ldq, nq, nkv, inv, (const kv16*)kpool, (const kv16*)vpool, block_table, mpps, n_pages,
                            seq_lens, extra, n_split, part, out, ctx.status, q_gain, eps, split_done);
   }
   if (hd == 64)
-    return go<64>(grid, threads, ctx.st, q, ldq, nq, nkv, inv, (const bf16*)kpool, (const bf16*)vpool, block_table, mpps, n_pages, seq_lens,
+    return go<64>(grid, threads, ctx.st, q, ldq, nq, nkv, inv, (const kv16*)kpool, (const kv16*)vpool, block_table, mpps, n_pages, seq_lens,
                   extra, n_split, part, out, ctx.status, q_gain, eps);
-  return go<128>(grid, threads, ctx.st, q, ldq, nq, nkv, inv, (const bf16*)kpool, (const bf16*)vpool, block_table, mpps, n_pages, seq_lens,
+  return go<128>(grid, threads, ctx.st, q, ldq, nq, nkv, inv, (const kv16*)kpool, (const kv16*)vpool, block_table, mpps, n_pages, seq_lens,
                  extra, n_split, part, out, ctx.status, q_gain, eps);
 }

@@ -19,6 +19,14 @@ template <> struct Vec8<bf16> {
     for (int i = 0; i < 4; ++i) { float2 t = __bfloat1622float2(h[i]); f[2 * i] = t.x; f[2 * i + 1] = t.y; }
   }
 };
+template <> struct Vec8<kv16> {
+  static __device__ __forceinline__ void load(const kv16* p, float* f) {
+    uint4 u = *reinterpret_cast<const uint4*>(p);
+    const __half2* hp = reinterpret_cast<const __half2*>(&u);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) { float2 t = __half22float2(hp[e]); f[2 * e] = t.x; f[2 * e + 1] = t.y; }
+  }
+};
 template <> struct Vec8<float> {
   static __device__ __forceinline__ void load(const float* p, float* f) {
     float4 a = __ldg(reinterpret_cast<const float4*>(p));
@@ -511,9 +519,9 @@ __global__ void __launch_bounds__(128) step_attn_paged_kernel(const float* __res
         float kf[8];
         if (sizeof(T) == 2) {
           uint4 u = *reinterpret_cast<const uint4*>(kr + c);
-          const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&u);
+          const __half2* hp = reinterpret_cast<const __half2*>(&u);     // 16-bit cache elements are halves
 #pragma unroll
-          for (int e = 0; e < 4; ++e) { float2 t = __bfloat1622float2(hp[e]); kf[2 * e] = t.x; kf[2 * e + 1] = t.y; }
+          for (int e = 0; e < 4; ++e) { float2 t = __half22float2(hp[e]); kf[2 * e] = t.x; kf[2 * e + 1] = t.y; }
         } else {
           float4 a = *reinterpret_cast<const float4*>(kr + c), bq = *reinterpret_cast<const float4*>(kr + c + 4);
           kf[0] = a.x; kf[1] = a.y; kf[2] = a.z; kf[3] = a.w; kf[4] = bq.x; kf[5] = bq.y; kf[6] = bq.z; kf[7] = bq.w;
@@ -620,7 +628,7 @@ void launch_step_attn(const LaunchCtx& ctx, const float* q, int ldq, int nq, int
       step_attn_paged_kernel<float><<<grid, 128, smem, ctx.st>>>(q, ldq, nq, nkv, hd, inv, (const float*)kpool, (const float*)vpool,
                                                                  block_table, mpps, n_pages, seq_lens, extra, n_split, part, out, ctx.status, q_gain, eps);
     } else {
-      step_attn_paged_kernel<bf16><<<grid, 128, smem, ctx.st>>>(q, ldq, nq, nkv, hd, inv, (const bf16*)kpool, (const bf16*)vpool,
+      step_attn_paged_kernel<kv16><<<grid, 128, smem, ctx.st>>>(q, ldq, nq, nkv, hd, inv, (const kv16*)kpool, (const kv16*)vpool,
                                                                 block_table, mpps, n_pages, seq_lens, extra, n_split, part, out, ctx.status, q_gain, eps);
     }
   } else {
@@ -629,7 +637,7 @@ void launch_step_attn(const LaunchCtx& ctx, const float* q, int ldq, int nq, int
       step_attn_kernel<float><<<grid, 128, smem, ctx.st>>>(q, ldq, nq, nkv, hd, inv, (const float*)kpool, (const float*)vpool,
                                                            block_table, mpps, n_pages, seq_lens, extra, n_split, part, out, ctx.status, q_gain, eps);
     else
-      step_attn_kernel<bf16><<<grid, 128, smem, ctx.st>>>(q, ldq, nq, nkv, hd, inv, (const bf16*)kpool, (const bf16*)vpool,
+      step_attn_kernel<kv16><<<grid, 128, smem, ctx.st>>>(q, ldq, nq, nkv, hd, inv, (const kv16*)kpool, (const kv16*)vpool,
                                                           block_table, mpps, n_pages, seq_lens, extra, n_split, part, out, ctx.status, q_gain, eps);
   }
   if (n_split > 1) {
@@ -681,5 +689,5 @@ void launch_step_append(const LaunchCtx& ctx, const float* qkv, int nq, int nkv,
   if (ctx.dtype == 0)
     step_append_kernel<float><<<batch, 128, 0, ctx.st>>>(qkv, nq, nkv, hd, inv, (float*)kpool, (float*)vpool, block_table, mpps, n_pages, seq_lens, ctx.status, k_gain, eps);
   else
-    step_append_kernel<bf16><<<batch, 128, 0, ctx.st>>>(qkv, nq, nkv, hd, inv, (bf16*)kpool, (bf16*)vpool, block_table, mpps, n_pages, seq_lens, ctx.status, k_gain, eps);
+    step_append_kernel<kv16><<<batch, 128, 0, ctx.st>>>(qkv, nq, nkv, hd, inv, (kv16*)kpool, (kv16*)vpool, block_table, mpps, n_pages, seq_lens, ctx.status, k_gain, eps);
 }

@@ -16,36 +16,17 @@
 #include <math.h>
 
 #include "common.cuh"
+#include "tc_ptx.cuh"
 #include "step_mega.h"
 
 namespace {
+using namespace tcp;
 
 constexpr int NT = 512;                 // threads per CTA, one CTA per SM
 constexpr int NW = NT / 32;
 constexpr int MAXG = 8;
 constexpr int NSLOT = 3;                // ring slots per warp
-constexpr unsigned SPIN_LIMIT = 20u * 1000u * 1000u;
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
 
 // Grid-wide barrier: every CTA adds one to *counter and waits until it reaches `target`.
 // Returns false when the wait ran out (or some role already gave up): the caller leaves.
@@ -357,10 +338,11 @@ __device__ __noinline__ void attn_item(const MegaParams& p, const MegaLayer& L, 
   float o[MAXG];
 #pragma unroll
   for (int i = 0; i < MAXG; ++i) o[i] = 0.f;
-  const int chunks_per_row = hd * (int)sizeof(T) / 16;
+  typedef typename KvOf<T>::type KT;                   // cache element: fp32, or 16-bit half in bf16 mode
+  const int chunks_per_row = hd * (int)sizeof(KT) / 16;
   const int n_chunks = PAGE_TOKENS * chunks_per_row;
-  const T* kpool = (const T*)L.kpool;
-  const T* vpool = (const T*)L.vpool;
+  const KT* kpool = (const KT*)L.kpool;
+  const KT* vpool = (const KT*)L.vpool;
   for (int pg = pg0; pg < pg1; ++pg) {
     int page = pg < p.mpps ? p.block_table[(size_t)b * p.mpps + pg] : -1;
     bool page_ok = page >= 0 && page < p.n_pages;
@@ -380,14 +362,14 @@ __device__ __noinline__ void attn_item(const MegaParams& p, const MegaLayer& L, 
     __syncthreads();
     if (hh_s < group) {
       float sc = 0.f;
-      const T* kr = reinterpret_cast<const T*>(Ks + key * row_bytes);
+      const KT* kr = reinterpret_cast<const KT*>(Ks + key * row_bytes);
       for (int c = 0; c < hd; c += 8) {
         float kf[8];
-        if (sizeof(T) == 2) {
+        if (sizeof(KT) == 2) {
           uint4 u = *reinterpret_cast<const uint4*>(kr + c);
-          const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&u);
+          const __half2* hp = reinterpret_cast<const __half2*>(&u);
 #pragma unroll
-          for (int e = 0; e < 4; ++e) { float2 t = __bfloat1622float2(hp[e]); kf[2 * e] = t.x; kf[2 * e + 1] = t.y; }
+          for (int e = 0; e < 4; ++e) { float2 t = __half22float2(hp[e]); kf[2 * e] = t.x; kf[2 * e + 1] = t.y; }
         } else {
           float4 a = *reinterpret_cast<const float4*>(kr + c), bq = *reinterpret_cast<const float4*>(kr + c + 4);
           kf[0] = a.x; kf[1] = a.y; kf[2] = a.z; kf[3] = a.w; kf[4] = bq.x; kf[5] = bq.y; kf[6] = bq.z; kf[7] = bq.w;
@@ -419,7 +401,7 @@ __device__ __noinline__ void attn_item(const MegaParams& p, const MegaLayer& L, 
       if (i * nhh < MAXG && h < group) {
         float acc = o[i] * alpha[h];
         const float* pr = ps + h * PAGE_TOKENS;
-        for (int s = 0; s < nk; ++s) acc = fmaf(pr[s], to_f(reinterpret_cast<const T*>(Vs + s * row_bytes)[dim]), acc);
+        for (int s = 0; s < nk; ++s) acc = fmaf(pr[s], to_f(reinterpret_cast<const KT*>(Vs + s * row_bytes)[dim]), acc);
         o[i] = acc;
       }
     }
@@ -523,10 +505,11 @@ __global__ void __launch_bounds__(NT, 1) step_mega_kernel(const __grid_constant_
           float x1 = __ldcg(kin + h * p.hd + c), x2 = __ldcg(kin + h * p.hd + c + half);
           if (L.k_norm) { x1 *= rk[h] * L.k_norm[c]; x2 *= rk[h] * L.k_norm[c + half]; }
           size_t off = (((size_t)page * L.nkv + h) * PAGE_TOKENS + row) * p.hd;
-          ((T*)L.kpool)[off + c] = from_f<T>(x1 * cs - x2 * sn);
-          ((T*)L.kpool)[off + c + half] = from_f<T>(x2 * cs + x1 * sn);
-          ((T*)L.vpool)[off + c] = from_f<T>(__ldcg(vin + h * p.hd + c));
-          ((T*)L.vpool)[off + c + half] = from_f<T>(__ldcg(vin + h * p.hd + c + half));
+          typedef typename KvOf<T>::type KT;
+          ((KT*)L.kpool)[off + c] = from_f<KT>(x1 * cs - x2 * sn);
+          ((KT*)L.kpool)[off + c + half] = from_f<KT>(x2 * cs + x1 * sn);
+          ((KT*)L.vpool)[off + c] = from_f<KT>(__ldcg(vin + h * p.hd + c));
+          ((KT*)L.vpool)[off + c + half] = from_f<KT>(__ldcg(vin + h * p.hd + c + half));
         }
       }
       BARRIER();

@@ -299,12 +299,9 @@ cudaError_t launch_step_gemm_tc(const bf16* W, int ldw, int N, int K, const bf16
   if (p.stages > 12) p.stages = 12;
   p.acc_stride = pow2_ceil(2 * Bp < 16 ? 16 : 2 * Bp);
   const int smem = p.stages * (W_BYTES + p.x_bytes) + 1024 + 8 * (2 * p.stages + 4) + 64;
-  static int attr_smem = 0;
-  if (smem > attr_smem) {
-    cudaError_t e = cudaFuncSetAttribute(step_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT);
-    if (e != cudaSuccess) return e;
-    attr_smem = SMEM_LIMIT;
-  }
+  static bool raised[TC_MAX_DEVICES] = {};
+  cudaError_t e = tc_raise_smem_limit(step_gemm_kernel, SMEM_LIMIT, raised);
+  if (e != cudaSuccess) return e;
   const long long total = (long long)((N + BM - 1) / BM) * ((K + BK - 1) / BK);
   const int grid = (int)(total < n_sm ? total : n_sm);
   ++*n_launch;

@@ -18,7 +18,8 @@ __device__ __forceinline__ size_t cache_off(int slot, int c, int nkv, int hd) {
 template <class T>
 __global__ void __launch_bounds__(256) kv_l1_kernel(const T* __restrict__ qkv, int ld, int k_col, const bf16* __restrict__ kv_lo,
                                                     int ld_lo, int T_tokens, int nkv, int hd, const int* __restrict__ tok_slot,
-                                                    const T* __restrict__ kpool, const T* __restrict__ vpool, float inv_n,
+                                                    const typename KvOf<T>::type* __restrict__ kpool,
+                                                    const typename KvOf<T>::type* __restrict__ vpool, float inv_n,
                                                     float* __restrict__ sum_k, float* __restrict__ sum_v) {
   const int dkv = nkv * hd;
   const size_t n = (size_t)T_tokens * dkv;
@@ -48,8 +49,9 @@ __global__ void __launch_bounds__(256) kv_l1_kernel(const T* __restrict__ qkv, i
 // The layer's key and value columns of the projection buffer take the predicted cache's entries.
 template <class T>
 __global__ void __launch_bounds__(256) kv_take_kernel(T* __restrict__ qkv, int ld, int k_col, int T_tokens, int nkv, int hd,
-                                                      const int* __restrict__ tok_slot, const T* __restrict__ kpool,
-                                                      const T* __restrict__ vpool) {
+                                                      const int* __restrict__ tok_slot,
+                                                      const typename KvOf<T>::type* __restrict__ kpool,
+                                                      const typename KvOf<T>::type* __restrict__ vpool) {
   const int dkv = nkv * hd;
   const size_t n = (size_t)T_tokens * dkv;
   for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
@@ -57,8 +59,8 @@ __global__ void __launch_bounds__(256) kv_take_kernel(T* __restrict__ qkv, int l
     const int slot = tok_slot[t];
     if (slot < 0) continue;
     const size_t off = cache_off(slot, c, nkv, hd);
-    qkv[(size_t)t * ld + k_col + c] = kpool[off];
-    qkv[(size_t)t * ld + k_col + dkv + c] = vpool[off];
+    qkv[(size_t)t * ld + k_col + c] = from_f<T>(to_f(kpool[off]));
+    qkv[(size_t)t * ld + k_col + dkv + c] = from_f<T>(to_f(vpool[off]));
   }
 }
 
@@ -77,7 +79,7 @@ void launch_kv_l1(const LaunchCtx& ctx, const void* qkv, int ld, int k_col, cons
                                                        (const float*)kpool, (const float*)vpool, inv_n, sum_k, sum_v);
   else
     kv_l1_kernel<bf16><<<grid_of(n), 256, 0, ctx.st>>>((const bf16*)qkv, ld, k_col, (const bf16*)kv_lo, ld_lo, T_tokens, nkv, hd,
-                                                      tok_slot, (const bf16*)kpool, (const bf16*)vpool, inv_n, sum_k, sum_v);
+                                                      tok_slot, (const kv16*)kpool, (const kv16*)vpool, inv_n, sum_k, sum_v);
 }
 
 void launch_kv_take(const LaunchCtx& ctx, void* qkv, int ld, int k_col, int T_tokens, int nkv, int hd, const int* tok_slot,
@@ -89,6 +91,6 @@ void launch_kv_take(const LaunchCtx& ctx, void* qkv, int ld, int k_col, int T_to
     kv_take_kernel<float><<<grid_of(n), 256, 0, ctx.st>>>((float*)qkv, ld, k_col, T_tokens, nkv, hd, tok_slot, (const float*)kpool,
                                                          (const float*)vpool);
   else
-    kv_take_kernel<bf16><<<grid_of(n), 256, 0, ctx.st>>>((bf16*)qkv, ld, k_col, T_tokens, nkv, hd, tok_slot, (const bf16*)kpool,
-                                                        (const bf16*)vpool);
+    kv_take_kernel<bf16><<<grid_of(n), 256, 0, ctx.st>>>((bf16*)qkv, ld, k_col, T_tokens, nkv, hd, tok_slot, (const kv16*)kpool,
+                                                        (const kv16*)vpool);
 }

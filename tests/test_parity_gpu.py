@@ -5,7 +5,8 @@ import pytest
 
 import workloads as wl
 from oracle import kvp_oracle as orc
-from parity_util import GAP, TOL, compare_prefill, make_session, rel_fro
+from parity_util import (GAP, TOL, ArgmaxTally, check_cache_layer, compare_prefill, compare_with_golden, load_golden,
+                         make_session, rel_fro, run_prefill)
 
 pytestmark = pytest.mark.gpu
 
@@ -73,12 +74,18 @@ def test_prefill_predict_matches_oracle(name, lens, regime):
     pr = wl.prompts(name, seed=1) if lens is None else wl.custom_prompts(pair.base.vocab, lens, seed=1)
     s = make_session(pair, W, pr)
     try:
-        # With 130 sequences some oracle top-2 gaps are certain to lie just above 1e-3, inside what the logits
-        # tolerance itself allows in bf16 (1e-2 of O(1) logits): there the first token is compared only where
-        # the gap is clear of that; the benchmark configurations keep the 1e-3 rule.
-        gap = 5e-2 if (pr.batch > 100 and pair.dtype == "bf16") else GAP
-        ek, ev, el, n = compare_prefill(s, pair, W, pr, gap=gap)
-        print(f"{name} {regime}: K {ek:.2e} V {ev:.2e} logits {el:.2e} argmax compared {n}/{pr.batch}")
+        ek, ev, el, tally = compare_prefill(s, pair, W, pr)
+        print(f"{name} {regime}: K {ek:.2e} V {ev:.2e} logits {el:.2e} argmax compared {tally.compared}/{pr.batch}")
+        # First token identical wherever the oracle's top-2 gap exceeds 1e-3.  A logits error inside the 1e-2 tolerance
+        # can still flip a near-tie (a flip needs gap < 2 max|err|), and among 130 sequences some gaps are certain to be
+        # that small: there, and only there, a flip is tolerated if the gap is below the logits tolerance itself, at most
+        # for 2 % of the sequences; every flip is printed.  All other cases and all benchmark configurations are strict.
+        if pr.batch > 100 and tally.mismatches:
+            print("first-token flips at near-ties: " + tally.report())
+            assert all(m["gap"] <= TOL[pair.dtype] for m in tally.mismatches), tally.report()
+            assert len(tally.mismatches) <= max(1, tally.compared // 50), tally.report()
+        else:
+            assert not tally.mismatches, tally.report()
     finally:
         s.close()
 
@@ -334,43 +341,90 @@ def test_error_paths_report_status_and_keep_the_context_usable():
         s.close()
 
 
-def test_config_2_full_size_matches_oracle():
-    """The benchmark's own workload (1.1B-shaped base, 270M-shaped aux, 1024-token prompt)."""
-    pair = wl.pair("c2")
-    W = wl.make_weights(pair, seed=0)
-    pr = wl.prompts("c2", seed=0)
+def test_bounded_wait_runs_out_and_is_reported_as_timeout():
+    """A device-side wait that nothing completes gives up after its limit: the kernel returns, the status word carries the
+    code, kvp_poll_status reports KVP_ERR_TIMEOUT, and the same handle then runs the whole path correctly."""
+    import torch
+    import paper_2410_08391_b200 as kvp
+    pair = wl.pair("t_small")
+    W = wl.make_weights(pair, seed=8, regime="fanin")
+    pr = wl.custom_prompts(pair.base.vocab, [70, 33], seed=8)
     s = make_session(pair, W, pr)
     try:
-        ek, ev, el, n = compare_prefill(s, pair, W, pr)
-        print(f"c2: K {ek:.2e} V {ev:.2e} logits {el:.2e} argmax compared {n}")
+        s.poll()
+        kvp.kvp_selftest_wait_timeout(s.h, s.workspace, s.stream)
+        with pytest.raises(kvp.KvpError) as e:
+            s.poll()
+        assert e.value.status == -7
+        s.poll()                                   # the word was cleared by the poll that reported it
+        ek, ev, el, tally = compare_prefill(s, pair, W, pr)
+        assert not tally.mismatches
     finally:
         s.close()
+
+
+def _full_size(name, seqs, golden=True):
+    """kvp_prefill_predict on a benchmark configuration in the launch configuration the benchmark times.  Every
+    sequence the stored oracle file follows is compared (logits, first token, sampled cache rows); `seqs` are followed
+    by the oracle here, whole cache included."""
+    pair = wl.pair(name)
+    W = wl.make_weights(pair, seed=0)
+    pr = wl.prompts(name, seed=0)
+    s = make_session(pair, W, pr)
+    try:
+        logits, first = run_prefill(s, pr)
+        lens = [int(x) for x in pr.lengths]
+        tol = TOL[pair.dtype]
+        g = load_golden(name) if golden else None
+        if golden:
+            assert g is not None, f"tests/golden/{name}_first_step.npz is missing (tests/golden/make_full_size_refs.py {name})"
+            el, er, tally, per_seq = compare_with_golden(s, pair, pr, logits, first, g)
+            print(f"{name}: {len(per_seq)} stored sequences, worst logits err {el:.2e}, worst sampled (token, head) slice {er:.2e}, "
+                  f"argmax compared {tally.compared}; per sequence: " + " ".join(f"{b}:{e:.1e}" for b, e in per_seq.items()))
+            assert not tally.mismatches, tally.report()
+        tally = ArgmaxTally()
+        ref = orc.prefill_predict(pair, W, pr, seqs)
+        for b, (kv_hat, ref_logits, _) in ref.items():
+            worst = 0.0
+            for i in range(pair.base.n_layers):
+                k, v = s.cache.gather(i, b, lens[b])
+                e1, e2, e3 = check_cache_layer(k, v, kv_hat[i][0], kv_hat[i][1], pair.base.layers[i].head_dim, tol, f"{name} seq {b} base layer {i}")
+                worst = max(worst, e1, e2)
+            e = rel_fro(logits[b], ref_logits)
+            assert e <= tol, f"{name} seq {b}: logits err {e:.3e}"
+            tally.add(b, first[b], logits[b], ref_logits)
+            print(f"{name} seq {b} ({lens[b]} tokens), whole cache: worst K/V layer err {worst:.2e}, logits {e:.2e}")
+        assert not tally.mismatches, tally.report()
+    finally:
+        s.close()
+
+
+def test_config_2_full_size_matches_oracle():
+    """The 1.1B-shaped base with the 270M-shaped auxiliary model on the 1024-token prompt."""
+    _full_size("c2", [0], golden=False)
 
 
 def test_paper_shaped_batch_full_size_sampled_sequences_match_oracle():
-    """64 prompts of 59 tokens (the TriviaQA 1-shot length of Sec. 6) on the 1.1B / 270M-shaped pair, in the launch
-    configuration the benchmark times (step pieces on their own stream, tensor-core step projections); the oracle
-    follows three sampled sequences."""
-    pair = wl.pair("qa")
-    W = wl.make_weights(pair, seed=0)
-    pr = wl.prompts("qa", seed=0)
-    s = make_session(pair, W, pr)
-    try:
-        ek, ev, el, n = compare_prefill(s, pair, W, pr, seqs=[0, 31, 63])
-        print(f"qa: K {ek:.2e} V {ev:.2e} logits {el:.2e} argmax compared {n}")
-    finally:
-        s.close()
+    """64 prompts of 59 tokens (the TriviaQA 1-shot length of Sec. 6) on the 1.1B / 270M-shaped pair (step pieces on
+    their own stream, tensor-core step projections); the oracle follows three sampled sequences."""
+    _full_size("qa", [0, 31, 63], golden=False)
 
 
 def test_layer_pruned_pair_full_size_sampled_sequences_match_oracle():
     """KVP-LP-0.25 of Table 1 (auxiliary = 7 of the base model's 28 layers) on the 64 x 59 batch."""
-    pair = wl.pair("lp25")
+    _full_size("lp25", [5, 40], golden=False)
+
+
+def test_prompt_length_sweep_batch_8_matches_oracle():
+    """The batch-8 prompt-length sweep of Sec. 6 (TTFT against prompt length) at one of its lengths, 8 x 256 tokens."""
+    pair = wl.pair("c2")
     W = wl.make_weights(pair, seed=0)
-    pr = wl.prompts("lp25", seed=0)
+    pr = wl.sweep_prompts(256, seed=0)
     s = make_session(pair, W, pr)
     try:
-        ek, ev, el, n = compare_prefill(s, pair, W, pr, seqs=[5, 40])
-        print(f"lp25: K {ek:.2e} V {ev:.2e} logits {el:.2e} argmax compared {n}")
+        ek, ev, el, tally = compare_prefill(s, pair, W, pr, seqs=[0, 7])
+        print(f"sweep8 256: K {ek:.2e} V {ev:.2e} logits {el:.2e} argmax compared {tally.compared}")
+        assert not tally.mismatches, tally.report()
     finally:
         s.close()
 
@@ -403,64 +457,64 @@ def test_train_forward_config_2_sampled_rows_match_oracle():
         s.close()
 
 
-def test_config_3_full_size_shortest_sequence_matches_oracle():
-    """3B-shaped base, 450M-shaped aux, 8 ragged prompts (25 240 tokens) in the launch configuration the
-    benchmark times; the oracle follows the shortest sequence, the batch-invariance test covers the rest."""
-    pair = wl.pair("c3")
-    W = wl.make_weights(pair, seed=0)
+def test_config_3_full_size_all_sequences_match_oracle():
+    """3B-shaped base, 450M-shaped auxiliary model, 8 ragged prompts (25 240 tokens): all 8 sequences against the
+    stored oracle results, the shortest one against the oracle run here with its whole cache."""
     pr = wl.prompts("c3", seed=0)
-    s = make_session(pair, W, pr)
-    try:
-        b = int(np.argmin(pr.lengths))
-        ek, ev, el, n = compare_prefill(s, pair, W, pr, seqs=[b])
-        print(f"c3 seq {b} ({int(pr.lengths[b])} tokens): K {ek:.2e} V {ev:.2e} logits {el:.2e} argmax compared {n}")
-    finally:
-        s.close()
+    _full_size("c3", [int(np.argmin(pr.lengths))])
 
 
-def test_config_4_full_size_one_sequence_matches_oracle():
-    """Layer-wise scaled pair, non-uniform map, 32 x 2048 tokens; the oracle follows sequence 0.
-    The logits bound is tight here for a reason that is not the kernels': rounding the oracle's own exact
-    predicted cache to bf16 (the cache format) and running the oracle's base step on it already moves the
-    logits by 9.3e-3 on sequence 5 and 7.0e-3 on C2 (oracle/cache_rounding_floor.py); K_hat and V_hat
-    themselves are within 6e-3."""
-    pair = wl.pair("c4")
-    W = wl.make_weights(pair, seed=0)
-    pr = wl.prompts("c4", seed=0)
-    s = make_session(pair, W, pr)
-    try:
-        ek, ev, el, n = compare_prefill(s, pair, W, pr, seqs=[0])
-        print(f"c4 seq 0: K {ek:.2e} V {ev:.2e} logits {el:.2e} argmax compared {n}")
-    finally:
-        s.close()
+def test_config_4_full_size_all_sequences_match_oracle():
+    """Layer-wise scaled pair, non-uniform map, 32 x 2048 tokens: all 32 sequences against the stored oracle results
+    (logits, first token, sampled cache rows); the sequence whose logits are the most sensitive to the cache's
+    storage rounding (largest stored `floor_f16`) is followed by the oracle here with its whole cache."""
+    g = load_golden("c4")
+    assert g is not None
+    _full_size("c4", [int(g["seqs"][int(np.argmax(g["floor_f16"]))])])
 
 
-def test_config_5_long_prompts_cache_prefix_matches_oracle():
-    """4 x 16 384 tokens.  The oracle cannot follow a whole sequence in reasonable time, but causality makes
-    the predicted cache entries of positions < n a function of the first n tokens alone: the oracle runs the
-    first 640 tokens of sequence 2 and its K_hat, V_hat are compared with rows 0..639 of the GPU's cache.
-    Logits are checked for what holds at any size: finite, and the first token is their argmax."""
-    import torch
+def test_config_5_long_prompts_match_oracle():
+    """4 x 16 384 tokens, the launch shape of the long-cache step (key-range splits over 256 pages).
+    (1) One whole sequence against the stored oracle run: first-step logits, first token, 24 sampled cache rows over the
+        whole length in every base layer.
+    (2) Every sequence: the GPU's own predicted cache is downloaded and the ORACLE's base step runs on it
+        (b <- B(I[-1], KV_B_hat), Fig. 2(b)); logits and first token of the GPU's step must match it.  This isolates the
+        step over 16 384 cached entries from the prefill.
+    (3) Causality makes cache rows < n a function of the first n tokens: the oracle runs the first 4096 tokens of another
+        sequence and every row of the GPU's cache prefix is compared, page tails included."""
     pair = wl.pair("c5")
     W = wl.make_weights(pair, seed=0)
     pr = wl.prompts("c5", seed=0)
     s = make_session(pair, W, pr)
+    tol = TOL[pair.dtype]
     try:
-        lens = [int(x) for x in pr.lengths]
-        logits, first = s.prefill_predict(torch.from_numpy(pr.tokens).to(s.device), lens)
-        s.poll()
-        logits, first = logits.cpu().numpy(), first.cpu().numpy()
+        logits, first = run_prefill(s, pr)
         assert np.isfinite(logits).all()
+        lens = [int(x) for x in pr.lengths]
+        g = load_golden("c5")
+        assert g is not None, "tests/golden/c5_first_step.npz is missing"
+        el, er, tally, per_seq = compare_with_golden(s, pair, pr, logits, first, g)
+        print(f"c5 stored sequence(s) {list(per_seq)}: logits err {el:.2e}, worst sampled (token, head) slice {er:.2e}, argmax compared {tally.compared}")
+        assert not tally.mismatches, tally.report()
+        tally = ArgmaxTally()
         for b in range(pr.batch):
-            assert int(first[b]) == int(np.argmax(logits[b]))
-        n = 640
-        kv_hat = orc.predict_kv(pair, W, orc.aux_prefill(pair, W, pr.seq(2)[:n]))
+            kv = []
+            for i in range(pair.base.n_layers):
+                k, v = s.cache.gather(i, b, lens[b])
+                kv.append((k.astype(np.float64), v.astype(np.float64)))
+            ref_logits = orc.base_first_step(pair, W, int(pr.seq(b)[-1]), kv)
+            e = rel_fro(logits[b], ref_logits)
+            print(f"c5 seq {b}: step on the GPU's own cache vs oracle step on the same cache: logits err {e:.2e}, gap {orc.top2_gap(ref_logits):.2e}")
+            assert e <= tol
+            tally.add(b, first[b], logits[b], ref_logits)
+        assert not tally.mismatches, tally.report()
+        n, b = 4096, 1
+        kv_hat = orc.predict_kv(pair, W, orc.aux_prefill(pair, W, pr.seq(b)[:n]))
         worst = 0.0
         for i in range(pair.base.n_layers):
-            k, v = s.cache.gather(i, 2, n)
-            e1, e2 = rel_fro(k, kv_hat[i][0]), rel_fro(v, kv_hat[i][1])
-            assert e1 <= TOL[pair.dtype] and e2 <= TOL[pair.dtype], (i, e1, e2)
+            k, v = s.cache.gather(i, b, n)
+            e1, e2, _ = check_cache_layer(k, v, kv_hat[i][0], kv_hat[i][1], pair.base.layers[i].head_dim, tol, f"c5 seq {b} prefix base layer {i}")
             worst = max(worst, e1, e2)
-        print(f"c5 seq 2 prefix {n}: worst K/V err {worst:.2e}")
+        print(f"c5 seq {b} prefix {n}: worst K/V err {worst:.2e}")
     finally:
         s.close()

@@ -367,6 +367,17 @@ def prompts(name: str, seed: int = 0) -> Prompts:
     raise KeyError(name)
 
 
+# Sec. 6 of the paper plots TTFT against the prompt length at batch 8 (on a CPU; the curve itself is not reproduced
+# here): the same sweep on synthetic Zipf prompts, every prompt of the batch of one length.
+SWEEP8_LENGTHS = (64, 128, 256, 512, 1024, 2048)
+
+
+def sweep_prompts(length: int, seed: int = 0, batch: int = 8) -> Prompts:
+    v = pair("c2").base.vocab
+    lens = np.full(batch, int(length), np.int32)
+    return Prompts(zipf_tokens(int(lens.sum()), v, seed, tag=f"sweep{length}"), lens)
+
+
 def custom_prompts(vocab: int, lengths: Sequence[int], seed: int = 0, zipf: bool = True) -> Prompts:
     lens = np.asarray(lengths, np.int32)
     n = int(lens.sum())
