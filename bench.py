@@ -220,7 +220,7 @@ class Bench:
         work = wl.algorithmic_work(pair, lens)
         decode_steps = max(args.decode_steps, 0) if full else 0
         sess = kvp.Session(pair, W, max_batch=pr.batch, max_total_tokens=pr.total, max_len=max(lens), device=dev,
-                           extra_len=2 * decode_steps + 4)
+                           extra_len=2 * decode_steps + 4, flags=args.opt_flags)
         toks = torch.from_numpy(pr.tokens).to(dev)
 
         def step():
@@ -407,6 +407,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--train-forward", action="store_true",
                     help="also time the training-time forward (base model over the whole prompt on the predicted cache)")
+    ap.add_argument("--opt-flags", type=int, default=0, help="kvp_options.flags: optional kernel variants (see include/kvp.h)")
     ap.add_argument("--decode-steps", type=int, default=16, help="generation steps timed after the TTFT measurement (0 = none)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "kvp" else args.warmup

@@ -92,8 +92,18 @@ typedef struct {
                              holds fp32 elements in KVP_F32 mode and IEEE half elements in KVP_BF16 mode.    */
   int32_t page_tokens;    /* tokens per cache page; must be 64                                       */
   int32_t predictor_bias; /* 1: the predictor has bias vectors pred.L{i}.bk / bv                     */
-  int32_t reserved;       /* must be 0                                                               */
+  int32_t flags;          /* 0, or a sum of KVP_OPT_* (kernel variants; results are the same within rounding) */
 } kvp_options;
+
+/* Kernel variants that are built and tested but are not the default schedule because they measured slower on the
+ * benchmark configurations (numbers in the design notes):
+ *   KVP_OPT_FUSED_KV_PRED  the K/V projection of an auxiliary layer and the KV predictor as ONE kernel (the predictor
+ *                          is the projection's epilogue; K_A / V_A reach it through shared memory), used for calls
+ *                          with at least one 128-token block per SM;
+ *   KVP_OPT_FUSED_NORM     RMSNorm folded into the GEMMs around it (the residual GEMM that completes x also writes
+ *                          bf16(x * gain) and the rows' sums of squares, the next GEMM scales its rows by 1 / rms),
+ *                          used where every output tile of the residual GEMMs belongs to one CTA. */
+enum { KVP_OPT_FUSED_KV_PRED = 1, KVP_OPT_FUSED_NORM = 2 };
 
 /* A named tensor handed to kvp_load_weights().  Names:
  *   "aux.embed" [vocab, d_A]
@@ -291,7 +301,8 @@ enum {
   KVP_CLASS_STEP_ATTN = 4,  /* base step: attention over the paged cache                  */
   KVP_CLASS_OTHER = 5,      /* norms, RoPE, SwiGLU, gathers, index, argmax                */
   KVP_CLASS_STEP_FUSED = 6, /* base step as one persistent kernel (batch <= 4)            */
-  KVP_N_CLASSES = 7
+  KVP_CLASS_KV_PRED = 7,    /* auxiliary K/V projection with the predictor as its epilogue */
+  KVP_N_CLASSES = 8
 };
 kvp_status kvp_timing_enable(kvp_handle* h, int32_t on);
 kvp_status kvp_timing_read(kvp_handle* h, double* ms, int64_t* launches);

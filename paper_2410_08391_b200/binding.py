@@ -35,7 +35,7 @@ class ModelCfgC(C.Structure):
 
 
 class OptionsC(C.Structure):
-    _fields_ = [("dtype", C.c_int32), ("page_tokens", C.c_int32), ("predictor_bias", C.c_int32), ("reserved", C.c_int32)]
+    _fields_ = [("dtype", C.c_int32), ("page_tokens", C.c_int32), ("predictor_bias", C.c_int32), ("flags", C.c_int32)]
 
 
 class TensorC(C.Structure):
@@ -54,7 +54,7 @@ EXPORTS = ["kvp_create", "kvp_destroy", "kvp_last_error", "kvp_layer_map_canonic
            "kvp_poll_status", "kvp_launch_count", "kvp_timing_enable", "kvp_timing_read",
            "kvp_decode_step_static", "kvp_train_workspace_bytes", "kvp_train_forward", "kvp_selftest_wait_timeout"]
 
-CLASS_NAMES = ["aux_gemm", "aux_attn", "predictor", "step_gemv", "step_attn", "other", "step_fused"]
+CLASS_NAMES = ["aux_gemm", "aux_attn", "predictor", "step_gemv", "step_attn", "other", "step_fused", "kv_pred"]
 
 _lib = None
 
@@ -132,11 +132,14 @@ def kvp_layer_map_uniform(n_base: int, n_aux: int) -> List[int]:
     return list(out)[:n_base]
 
 
+KVP_OPT_FUSED_KV_PRED, KVP_OPT_FUSED_NORM = 1, 2
+
+
 def kvp_create(aux, base, layer_map: Sequence[int], dtype: str = "bf16", predictor_bias: bool = False,
-               page_tokens: int = 64) -> int:
+               page_tokens: int = 64, flags: int = 0) -> int:
     a, _ka = _model_c(aux)
     b, _kb = _model_c(base)
-    opt = OptionsC(KVP_BF16 if dtype == "bf16" else KVP_F32, page_tokens, int(predictor_bias), 0)
+    opt = OptionsC(KVP_BF16 if dtype == "bf16" else KVP_F32, page_tokens, int(predictor_bias), int(flags))
     h = C.c_void_p()
     _check(lib().kvp_create(C.byref(a), C.byref(b), _i32arr(layer_map), C.byref(opt), C.byref(h)))
     return h.value
@@ -305,7 +308,7 @@ class Session:
     """Creates a handle for `pair`, uploads and packs weights, allocates workspace and cache."""
 
     def __init__(self, pair, weights: Dict[str, np.ndarray], max_batch: int, max_total_tokens: int, max_len: int,
-                 device="cuda:0", extra_len: int = 0):
+                 device="cuda:0", extra_len: int = 0, flags: int = 0):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("no CUDA device: the KV Prediction library has no CPU path")
@@ -313,7 +316,7 @@ class Session:
         self.pair = pair
         self.device = torch.device(device)
         torch.cuda.set_device(self.device)
-        self.h = kvp_create(pair.aux, pair.base, pair.layer_map, pair.dtype, pair.predictor_bias)
+        self.h = kvp_create(pair.aux, pair.base, pair.layer_map, pair.dtype, pair.predictor_bias, flags=flags)
         # The library replays a recorded CUDA graph per call, which the legacy default stream cannot record:
         # when that is the current stream the session works on a stream of its own and orders it against the
         # current stream around every call, so a caller still sees everything in the current stream's order.

@@ -36,12 +36,29 @@ template <int BN> struct Tile {
   static constexpr int STAGE_BYTES = A_BYTES + W_BYTES;    // 48 KiB / 32 KiB
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
 };
+// Fused-norm residual epilogue: each epilogue warp prefetches the residual stream's old values of its 32 rows,
+// 32 columns at a time, into a private ring of XS slots (TMA, 128-byte swizzle) while the main loop of the next
+// tile runs, so the read-modify-write of X never waits on memory.
+constexpr int XS = 2;
+constexpr int X_SLOT_BYTES = 32 * 32 * 4;
+constexpr int XRING_BYTES = 4 * XS * X_SLOT_BYTES;       // 32 KiB
 __device__ __forceinline__ uint4 pack8(const float* v) {
   __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
   __nv_bfloat162 c = __floats2bfloat162_rn(v[4], v[5]), d = __floats2bfloat162_rn(v[6], v[7]);
   uint4 u;
   u.x = *reinterpret_cast<uint32_t*>(&a); u.y = *reinterpret_cast<uint32_t*>(&b);
   u.z = *reinterpret_cast<uint32_t*>(&c); u.w = *reinterpret_cast<uint32_t*>(&d);
+  return u;
+}
+// 8 values as IEEE halves (saturating)
+__device__ __forceinline__ uint4 pack8_half(const float* v) {
+  uint4 u;
+  uint32_t* w = &u.x;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const __half2 h = __floats2half2_rn(fminf(fmaxf(v[2 * i], -65504.f), 65504.f), fminf(fmaxf(v[2 * i + 1], -65504.f), 65504.f));
+    w[i] = *reinterpret_cast<const uint32_t*>(&h);
+  }
   return u;
 }
 // bf16 rounding remainders of 8 values
@@ -83,16 +100,18 @@ struct Params {
   bf16* C; int ldc;
   float* X; int ldx;
   bf16* C_lo; int ld_lo; int lo_col_begin;
+  int lo_is_half;        // C_lo receives the whole value as an IEEE half instead of the bf16 remainder
+  int f16_operands;      // A and W hold IEEE halves (both operands of one MMA have the same type)
   int rot_cols; int hd;
   const float2* rope_tab; const int* tok_pos;
   int ffn;               // SwiGLU: output width
   const float* q_gain; const float* k_gain; int q_cols; float eps;   // TC_QKV: query / key norm (null = off)
   PagedOut paged;
-  // RMSNorm folded into its neighbours.  Producer (TC_RESID with H): once an element of X is final the epilogue also
-  // writes the next GEMM's operand H = bf16(X * gain_next) (+ its bf16 remainder H_lo) and adds the row's share of
-  // sum X^2 to ss_out[m].  Consumer (TC_QKV / TC_SWIGLU with ss_in): every row of the accumulator is scaled by
+  // RMSNorm folded into its neighbours.  Producer (TC_RESID with H; every tile owned by one CTA): the epilogue
+  // reads the old X (prefetched by TMA), stores X + acc, and also writes the next GEMM's operand
+  // H = bf16(X * gain_next) (+ its bf16 remainder H_lo) and adds the row's share of sum X^2 to ss_out[m].  Consumer (TC_QKV / TC_SWIGLU with ss_in): every row of the accumulator is scaled by
   // rsqrt(ss_in[m] / K + rms_eps), which is the norm's 1 / rms applied after the product instead of before it.
-  bf16* H; bf16* H_lo; int ldh; const float* gain_next; float* ss_out; int* tile_cnt;
+  bf16* H; bf16* H_lo; int ldh; const float* gain_next; float* ss_out;
   const float* ss_in; float rms_eps;
 };
 
@@ -171,7 +190,6 @@ __device__ __forceinline__ void epilogue_tile(const Params& p, uint32_t tmem_acc
   // tmem_acc already carries this warp's lane quarter in its upper half
   if (EPI == TC_STORE || EPI == TC_RESID || EPI == TC_PAGED) {
     int slot = -1;
-    float row_ss = 0.f;
     if (EPI == TC_PAGED && row_ok) slot = p.paged.tok_slot[m];
 #pragma unroll 1
     for (int c = 0; c < BN; c += 32) {
@@ -186,21 +204,9 @@ __device__ __forceinline__ void epilogue_tile(const Params& p, uint32_t tmem_acc
         store32_bf16(p.C + (size_t)m * p.ldc + n, v, n_valid);
       } else if (EPI == TC_RESID) {
         float* x = p.X + (size_t)m * p.ldx + n;
-        if (p.H && !p.stream_k) {     // this CTA alone owns the tile: plain read-modify-write, the final value is known here
 #pragma unroll
-          for (int g = 0; g < 8; ++g)
-            if (g * 4 < n_valid) {
-              float4 o = *reinterpret_cast<const float4*>(x + 4 * g);
-              o.x += v[4 * g]; o.y += v[4 * g + 1]; o.z += v[4 * g + 2]; o.w += v[4 * g + 3];
-              *reinterpret_cast<float4*>(x + 4 * g) = o;
-              v[4 * g] = o.x; v[4 * g + 1] = o.y; v[4 * g + 2] = o.z; v[4 * g + 3] = o.w;
-            }
-          row_ss += norm_out32(p, m, n, n_valid, v);
-        } else {
-#pragma unroll
-          for (int g = 0; g < 8; ++g)
-            if (g * 4 < n_valid) red_add4(x + 4 * g, v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
-        }
+        for (int g = 0; g < 8; ++g)
+          if (g * 4 < n_valid) red_add4(x + 4 * g, v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
       } else {
         if (slot < 0) continue;
         const PagedOut& q = p.paged;
@@ -217,7 +223,6 @@ __device__ __forceinline__ void epilogue_tile(const Params& p, uint32_t tmem_acc
         store32_kv(dst, v, n_valid);
       }
     }
-    if (EPI == TC_RESID && p.H && !p.stream_k && row_ok) atomicAdd(p.ss_out + m, row_ss);
   } else if (EPI == TC_SWIGLU) {
     // every 128 columns of the tile: [0, 64) gate rows, [64, 128) the matching up rows
     const float rinv = (p.ss_in && row_ok) ? rsqrtf(p.ss_in[m] / (float)p.K + p.rms_eps) : 1.f;
@@ -289,10 +294,18 @@ __device__ __forceinline__ void epilogue_tile(const Params& p, uint32_t tmem_acc
         store32_bf16(dst + half, b, 32);
         if (p.C_lo && n >= p.lo_col_begin) {
           bf16* lo = p.C_lo + (size_t)m * p.ld_lo + (n - p.lo_col_begin);
+          if (p.lo_is_half) {
 #pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            *reinterpret_cast<uint4*>(lo + g * 8) = pack8_lo(a + g * 8);
-            *reinterpret_cast<uint4*>(lo + half + g * 8) = pack8_lo(b + g * 8);
+            for (int g = 0; g < 4; ++g) {
+              *reinterpret_cast<uint4*>(lo + g * 8) = pack8_half(a + g * 8);
+              *reinterpret_cast<uint4*>(lo + half + g * 8) = pack8_half(b + g * 8);
+            }
+          } else {
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+              *reinterpret_cast<uint4*>(lo + g * 8) = pack8_lo(a + g * 8);
+              *reinterpret_cast<uint4*>(lo + half + g * 8) = pack8_lo(b + g * 8);
+            }
           }
         }
       }
@@ -303,23 +316,23 @@ __device__ __forceinline__ void epilogue_tile(const Params& p, uint32_t tmem_acc
 template <int EPI, int BN>
 __global__ void __launch_bounds__(N_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_a2,
-               const __grid_constant__ CUtensorMap map_w, const Params p) {
+               const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, const Params p) {
   using T = Tile<BN>;
   constexpr int STAGES = T::STAGES, STAGE_BYTES = T::STAGE_BYTES;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
-  // bars: full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], fin; then tmem base, abort flag, last-share flag
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 5);
+  constexpr int XR = EPI == TC_RESID ? XRING_BYTES : 0;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES + XR);
+  // bars: full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], x_full[4][XS]; then tmem base, abort flag
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4 + 4 * XS);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  volatile int* s_last = reinterpret_cast<volatile int*>(tmem_slot + 2);
   const uint32_t smem_base = smem_u32(smem);
   const uint32_t bar_base = smem_u32(bars);
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
   auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
   auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
-  const uint32_t fin_bar = bar_base + 8u * (2 * STAGES + 4);      // the four epilogue warps meet here (stream-K with fused norm)
+  auto xfull_bar = [&](int q, int s) { return bar_base + 8u * (2 * STAGES + 4 + q * XS + s); };
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   pdl_trigger();      // the next kernel's CTAs may take SMs as this kernel's CTAs leave them
@@ -332,7 +345,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 2); mbar_init(empty_bar(s), 1); }   // two loaders per stage
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
-    mbar_init(fin_bar, 4);
+    for (int q = 0; q < 4; ++q) for (int x = 0; x < XS; ++x) mbar_init(xfull_bar(q, x), 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -375,7 +388,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
-      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      // operand formats: bits 7-9 (A) and 10-12 (B): 1 = bf16, 0 = IEEE half
+      const uint32_t fmt = p.f16_operands ? 0u : ((1u << 7) | (1u << 10));
+      const uint32_t idesc = (1u << 4) | fmt | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
       Sched<BN> sched(p);
       Work w;
       int stage = 0; uint32_t phase = 0;
@@ -408,8 +423,27 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int quarter = warp & 3;
     Sched<BN> sched(p);
     Work w;
-    int acc = 0; uint32_t acc_phase = 0, fin_phase = 0;
+    int acc = 0; uint32_t acc_phase = 0;
     bool ok = true;
+    // fused norm (TC_RESID with H, every tile owned by one CTA): the old values of X arrive through this warp's ring
+    const bool fused = EPI == TC_RESID && p.H != nullptr;
+    const uint32_t xring = smem_base + STAGES * STAGE_BYTES + quarter * (XS * X_SLOT_BYTES);
+    Sched<BN> pre(p);
+    Work pw;
+    bool pre_ok = fused && pre.next(pw);
+    int pre_c = 0;
+    uint32_t x_issued = 0, x_used = 0;
+    auto prefetch_x = [&]() {      // next 32 x 32 block of X in (tile, column) order into the slot just freed
+      if (!pre_ok) return;
+      const int slot = x_issued % XS;
+      if (lane == 0) {
+        mbar_expect_tx(xfull_bar(quarter, slot), X_SLOT_BYTES);
+        tma_load_2d(xring + slot * X_SLOT_BYTES, &map_x, pw.n0 + pre_c * 32, pw.m0 + quarter * 32, xfull_bar(quarter, slot));
+      }
+      ++x_issued;
+      if (pw.n0 + (++pre_c) * 32 >= p.N || pre_c * 32 >= BN) { pre_ok = pre.next(pw); pre_c = 0; }
+    };
+    if (fused) for (int i = 0; i < XS; ++i) prefetch_x();
     while (sched.next(w)) {
       ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status);
       ok = __all_sync(0xffffffffu, ok);
@@ -417,55 +451,79 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       tc_fence_after();
       const int m = w.m0 + quarter * 32 + lane;
       const uint32_t tmem_acc = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
-      epilogue_tile<EPI, BN>(p, tmem_acc, m, w.n0, m < p.M);
+      if (fused) {
+        float row_ss = 0.f;
+#pragma unroll 1
+        for (int c = 0; c < BN && ok; c += 32) {
+          const int n = w.n0 + c, n_valid = p.N - n;
+          if (n_valid <= 0) break;
+          const int slot = x_used % XS;
+          ok = mbar_wait(xfull_bar(quarter, slot), (x_used / XS) & 1u, abort_flag, p.status);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          float v[32];
+          tmem_ld32(tmem_acc + c, v);
+          const uint32_t xrow = xring + slot * X_SLOT_BYTES + lane * 128;
+#pragma unroll
+          for (int g = 0; g < 8; ++g) {          // this thread's row of the slot: 16-byte pieces swizzled by the row
+            float4 o;
+            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(o.x), "=f"(o.y), "=f"(o.z), "=f"(o.w)
+                         : "r"(xrow + ((g ^ (lane & 7)) << 4)));
+            if (g == 0) tmem_ld_wait();
+            v[4 * g] += o.x; v[4 * g + 1] += o.y; v[4 * g + 2] += o.z; v[4 * g + 3] += o.w;
+          }
+          __syncwarp();
+          ++x_used;
+          prefetch_x();
+          if (m < p.M) {
+            float* x = p.X + (size_t)m * p.ldx + n;
+#pragma unroll
+            for (int g = 0; g < 8; ++g)
+              if (g * 4 < n_valid) *reinterpret_cast<float4*>(x + 4 * g) = make_float4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+            row_ss += norm_out32(p, m, n, n_valid, v);
+          }
+        }
+        if (!ok) break;
+        if (m < p.M) atomicAdd(p.ss_out + m, row_ss);
+      } else if (EPI == TC_RESID) {
+        // X += acc through the copy engine: a 32 x 32 block of the accumulator goes into one of this warp's slots
+        // (swizzled like a tensor tile) and leaves as ONE reduce-add of whole 128-byte rows, instead of 256 separate
+        // 16-byte atomics.  Rows and columns beyond the matrix are clipped by the tensor map.
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 32) {
+          const int n = w.n0 + c;
+          if (n >= p.N) break;
+          const int slot = x_used % XS;
+          if (x_used >= XS) {          // the reduce issued from this slot two blocks ago has read it
+            if (lane == 0) asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(XS - 1) : "memory");
+            __syncwarp();
+          }
+          float v[32];
+          tmem_ld32(tmem_acc + c, v);
+          tmem_ld_wait();
+          const uint32_t xrow = xring + slot * X_SLOT_BYTES + lane * 128;
+#pragma unroll
+          for (int g = 0; g < 8; ++g)
+            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(xrow + ((g ^ (lane & 7)) << 4)), "f"(v[4 * g]), "f"(v[4 * g + 1]),
+                         "f"(v[4 * g + 2]), "f"(v[4 * g + 3]) : "memory");
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          __syncwarp();
+          if (lane == 0) {
+            asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2}], [%3];"
+                         ::"l"(&map_x), "r"(n), "r"(w.m0 + quarter * 32), "r"(xring + slot * X_SLOT_BYTES) : "memory");
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+          }
+          ++x_used;
+        }
+      } else {
+        epilogue_tile<EPI, BN>(p, tmem_acc, m, w.n0, m < p.M);
+      }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar(acc));
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
-      if (EPI == TC_RESID && p.H && p.stream_k) {
-        // A tile's k blocks are shared among CTAs that add their partial sums with red.global.  Each share counts
-        // its k blocks into the tile's counter once its adds are globally visible; the share that completes the
-        // count re-reads the finished tile (from L2) and writes the next GEMM's operand and the rows' sums of squares.
-        __threadfence();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(fin_bar);
-        ok = mbar_wait(fin_bar, fin_phase, abort_flag, p.status);
-        fin_phase ^= 1u;
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        if (quarter == 3 && lane == 0) {
-          const int add = w.kb1 - w.kb0;
-          *s_last = (atomicAdd(p.tile_cnt + w.tile, add) + add == num_kb) ? 1 : 0;
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(fin_bar);
-        ok = mbar_wait(fin_bar, fin_phase, abort_flag, p.status);
-        fin_phase ^= 1u;
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        if (*s_last) {
-          __threadfence();
-          if (m < p.M) {
-            float row_ss = 0.f;
-#pragma unroll 1
-            for (int c = 0; c < BN; c += 32) {
-              const int n = w.n0 + c, n_valid = p.N - n;
-              if (n_valid <= 0) break;
-              float v[32];
-              const float* x = p.X + (size_t)m * p.ldx + n;
-#pragma unroll
-              for (int g = 0; g < 8; ++g) {
-                float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (g * 4 < n_valid) o = __ldcg(reinterpret_cast<const float4*>(x + 4 * g));
-                v[4 * g] = o.x; v[4 * g + 1] = o.y; v[4 * g + 2] = o.z; v[4 * g + 3] = o.w;
-              }
-              row_ss += norm_out32(p, m, n, n_valid, v);
-            }
-            atomicAdd(p.ss_out + m, row_ss);
-          }
-        }
-      }
     }
+    if (EPI == TC_RESID && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");    // this warp's reduces have completed
   }
   tc_fence_before();
   __syncthreads();
@@ -482,21 +540,22 @@ bool make_map(CUtensorMap* m, const void* base, int rows, int cols, int ld, int 
 }
 
 template <int EPI, int BN>
-cudaError_t go(const CUtensorMap& a, const CUtensorMap& a2, const CUtensorMap& w, const Params& p, int grid, cudaStream_t st) {
+cudaError_t go(const CUtensorMap& a, const CUtensorMap& a2, const CUtensorMap& w, const CUtensorMap& x, const Params& p, int grid, cudaStream_t st) {
+  constexpr int SMEM = Tile<BN>::SMEM_BYTES + (EPI == TC_RESID ? XRING_BYTES : 0);
   static bool raised[TC_MAX_DEVICES] = {};
-  cudaError_t e = tc_raise_smem_limit(gemm_tc_kernel<EPI, BN>, Tile<BN>::SMEM_BYTES, raised);
+  cudaError_t e = tc_raise_smem_limit(gemm_tc_kernel<EPI, BN>, SMEM, raised);
   if (e != cudaSuccess) return e;
-  return launch_overlapped(gemm_tc_kernel<EPI, BN>, dim3(grid), dim3(N_THREADS), Tile<BN>::SMEM_BYTES, st, a, a2, w, p);
+  return launch_overlapped(gemm_tc_kernel<EPI, BN>, dim3(grid), dim3(N_THREADS), SMEM, st, a, a2, w, x, p);
 }
 
 template <int BN>
-cudaError_t go_epi(int epi, const CUtensorMap& a, const CUtensorMap& a2, const CUtensorMap& w, const Params& p, int grid, cudaStream_t st) {
+cudaError_t go_epi(int epi, const CUtensorMap& a, const CUtensorMap& a2, const CUtensorMap& w, const CUtensorMap& x, const Params& p, int grid, cudaStream_t st) {
   switch (epi) {
-    case TC_STORE: return go<TC_STORE, BN>(a, a2, w, p, grid, st);
-    case TC_RESID: return go<TC_RESID, BN>(a, a2, w, p, grid, st);
-    case TC_SWIGLU: return go<TC_SWIGLU, BN>(a, a2, w, p, grid, st);
-    case TC_QKV: return go<TC_QKV, BN>(a, a2, w, p, grid, st);
-    default: return go<TC_PAGED, BN>(a, a2, w, p, grid, st);
+    case TC_STORE: return go<TC_STORE, BN>(a, a2, w, x, p, grid, st);
+    case TC_RESID: return go<TC_RESID, BN>(a, a2, w, x, p, grid, st);
+    case TC_SWIGLU: return go<TC_SWIGLU, BN>(a, a2, w, x, p, grid, st);
+    case TC_QKV: return go<TC_QKV, BN>(a, a2, w, x, p, grid, st);
+    default: return go<TC_PAGED, BN>(a, a2, w, x, p, grid, st);
   }
 }
 
@@ -513,6 +572,11 @@ double tile_cost(const TcGemm& g, int bn, bool stream_k) {
 
 }  // namespace
 
+bool tc_gemm_resid_can_fuse(int M, int N, int n_sm) {
+  // with fewer than two 128 x 128 tiles per SM the k loops are shared among CTAs and no CTA sees a final value
+  return ((M + BM - 1) / BM) * ((N + 127) / 128) >= 2 * n_sm;
+}
+
 bool tc_gemm_supported(const TcGemm& g) {
   auto al16 = [](const void* p) { return ((uintptr_t)p & 15) == 0; };
   if (g.M <= 0 || g.N <= 0 || g.K <= 0) return false;
@@ -521,7 +585,8 @@ bool tc_gemm_supported(const TcGemm& g) {
   switch (g.epi) {
     case TC_STORE: return g.N % 8 == 0 && g.ldc % 8 == 0 && al16(g.C);
     case TC_RESID:
-      if (g.H && (g.N % 8 || g.ldh % 8 || !al16(g.H) || (g.H_lo && !al16(g.H_lo)) || !g.gain_next || !g.ss_out || !g.tile_cnt)) return false;
+      if (g.H && (g.N % 8 || g.ldh % 8 || !al16(g.H) || (g.H_lo && !al16(g.H_lo)) || !g.gain_next || !g.ss_out || g.A2 ||
+                  !tc_gemm_resid_can_fuse(g.M, g.N, g.n_sm))) return false;
       return g.N % 4 == 0 && g.ldx % 4 == 0 && al16(g.X);
     case TC_SWIGLU: return g.ffn % 64 == 0 && g.N == 2 * g.ffn && g.ldc % 8 == 0 && al16(g.C);
     case TC_QKV:
@@ -543,24 +608,28 @@ cudaError_t launch_gemm_tc(const TcGemm& g, int* status, cudaStream_t st, int64_
   const bool stream_k = g.epi == TC_RESID && !g.A2 && tiles128 < 2 * g.n_sm;
   int bn = g.bn;
   if (bn != 128 && bn != 256) bn = tile_cost(g, 256, stream_k) <= tile_cost(g, 128, stream_k) ? 256 : 128;
-  CUtensorMap ma, ma2, mw;
+  CUtensorMap ma, ma2, mw, mx;
+  if (g.H && (stream_k || g.epi != TC_RESID)) return cudaErrorInvalidValue;     // see tc_gemm_resid_can_fuse()
   if (!make_map(&ma, g.A, g.M, g.K, g.lda, BM)) return cudaErrorInvalidValue;
   if (!make_map(&mw, g.W, g.N, g.K, g.ldw, bn)) return cudaErrorInvalidValue;
   if (g.A2) { if (!make_map(&ma2, g.A2, g.M, g.K, g.lda2, BM)) return cudaErrorInvalidValue; }
   else ma2 = ma;
+  if (g.epi == TC_RESID) { if (!tc_make_map_f32(&mx, g.X, g.M, g.N, g.ldx, 32)) return cudaErrorInvalidValue; }
+  else mx = ma;
   Params p{};
   p.M = g.M; p.N = g.N; p.K = g.K; p.split_begin = g.split_begin; p.has_a2 = g.A2 != nullptr; p.status = status;
   p.stream_k = stream_k ? 1 : 0;
   p.C = g.C; p.ldc = g.ldc; p.X = g.X; p.ldx = g.ldx; p.C_lo = g.C_lo; p.ld_lo = g.ld_lo; p.lo_col_begin = g.lo_col_begin;
   p.q_gain = g.q_gain; p.k_gain = g.k_gain; p.q_cols = g.q_cols; p.eps = g.eps;
   p.rot_cols = g.rot_cols; p.hd = g.hd; p.rope_tab = g.rope_tab; p.tok_pos = g.tok_pos; p.ffn = g.ffn; p.paged = g.paged;
-  p.H = g.H; p.H_lo = g.H_lo; p.ldh = g.ldh; p.gain_next = g.gain_next; p.ss_out = g.ss_out; p.tile_cnt = g.tile_cnt;
+  p.H = g.H; p.H_lo = g.H_lo; p.ldh = g.ldh; p.gain_next = g.gain_next; p.ss_out = g.ss_out;
   p.ss_in = g.ss_in; p.rms_eps = g.rms_eps;
+  p.lo_is_half = g.lo_is_half; p.f16_operands = g.f16_operands;
   const int tiles = ((g.M + BM - 1) / BM) * ((g.N + bn - 1) / bn);
   const long long kblocks = (long long)tiles * ((g.K + BK - 1) / BK);
   int grid = stream_k ? (int)(kblocks < g.n_sm ? kblocks : g.n_sm) : (tiles < g.n_sm ? tiles : g.n_sm);
   ++*n_launch;
-  return bn == 256 ? go_epi<256>(g.epi, ma, ma2, mw, p, grid, st) : go_epi<128>(g.epi, ma, ma2, mw, p, grid, st);
+  return bn == 256 ? go_epi<256>(g.epi, ma, ma2, mw, mx, p, grid, st) : go_epi<128>(g.epi, ma, ma2, mw, mx, p, grid, st);
 }
 
 // ---- RoPE table: tab[pos][c] = (cos, sin)(pos * theta^(-2c/hd)) -----------------------------

@@ -31,14 +31,17 @@ struct TcGemm {
   // RMSNorm folded into the neighbouring GEMMs (all null / 0 = off).
   // TC_RESID with H: besides X += A W^T the epilogue writes H[m, n] = bf16(X[m, n] * gain_next[n]) (row stride ldh;
   // H_lo = the bf16 remainder, or null) and adds the row's share of sum_n X[m, n]^2 to ss_out[m] (cleared by the
-  // caller); tile_cnt: one zeroed int per 128 x 128 output tile of this launch, used when tiles are shared among CTAs.
+  // caller).  Only where tc_gemm_resid_can_fuse() holds (every output tile computed by one CTA).
   // TC_QKV / TC_SWIGLU with ss_in: the accumulator rows are scaled by rsqrt(ss_in[m] / K + rms_eps).
-  bf16* H; bf16* H_lo; int ldh; const float* gain_next; float* ss_out; int* tile_cnt;
+  bf16* H; bf16* H_lo; int ldh; const float* gain_next; float* ss_out;
   const float* ss_in; float rms_eps;
+  int lo_is_half;                  // TC_QKV: C_lo receives the whole value as an IEEE half (not the bf16 remainder)
+  int f16_operands;                // A and W hold IEEE halves instead of bf16 (same 2 bytes; both operands alike)
   int n_sm;
   int bn;                          // tile width: 128, 256, or 0 = chosen by the launcher
 };
 
 bool tc_gemm_supported(const TcGemm& g);
+bool tc_gemm_resid_can_fuse(int M, int N, int n_sm);
 cudaError_t launch_gemm_tc(const TcGemm& g, int* status, cudaStream_t st, int64_t* n_launch);
 void launch_rope_table(const LaunchCtx& ctx, float2* tab, int n_pos, int hd, float theta);

@@ -38,6 +38,8 @@ void launch_pack_rows(const LaunchCtx& ctx, const void* src, int sdt, void* dst,
   if (sdt == 0 && ddt == 0) pack_rows_kernel<float, float><<<grid, 256, 0, ctx.st>>>((const float*)src, (float*)dst, rows, cols, map);
   else if (sdt == 0 && ddt == 1) pack_rows_kernel<float, bf16><<<grid, 256, 0, ctx.st>>>((const float*)src, (bf16*)dst, rows, cols, map);
   else if (sdt == 1 && ddt == 0) pack_rows_kernel<bf16, float><<<grid, 256, 0, ctx.st>>>((const bf16*)src, (float*)dst, rows, cols, map);
+  else if (sdt == 0 && ddt == 2) pack_rows_kernel<float, kv16><<<grid, 256, 0, ctx.st>>>((const float*)src, (kv16*)dst, rows, cols, map);
+  else if (sdt == 1 && ddt == 2) pack_rows_kernel<bf16, kv16><<<grid, 256, 0, ctx.st>>>((const bf16*)src, (kv16*)dst, rows, cols, map);
   else pack_rows_kernel<bf16, bf16><<<grid, 256, 0, ctx.st>>>((const bf16*)src, (bf16*)dst, rows, cols, map);
 }
 

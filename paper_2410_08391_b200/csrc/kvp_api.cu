@@ -12,6 +12,7 @@
 #include "attn_tc.h"
 #include "gemm_tc.h"
 #include "kvp_internal.h"
+#include "kvpred_tc.h"
 #include "step_mega.h"
 #include "step_tc.h"
 
@@ -148,6 +149,8 @@ WsLayout ws_layout(const kvp_handle* h, int64_t Bm, int64_t Tm) {
   w.gub = take(Bm * 2 * (size_t)B.max_ffn * 4);
   w.attn_sched = take((size_t)(Tm / 128 + Bm + 1) * 8);
   w.attn_done = take((size_t)Bm * B.max_nkv * 4);
+  // fused RMSNorm: per auxiliary layer two vectors of row sums of squares (one memset clears all)
+  w.norm_ss = take((size_t)2 * A.n_layers * Tm * 4);
   w.total = off;
   return w;
 }
@@ -389,7 +392,7 @@ kvp_status kvp_create(const kvp_model_cfg* aux, const kvp_model_cfg* base, const
   if (!aux || !base || !layer_map || !opt) return KVP_ERR_INVALID_ARG;
   if (validate_model(aux) || validate_model(base)) return KVP_ERR_SHAPE;
   if (opt->dtype != KVP_F32 && opt->dtype != KVP_BF16) return KVP_ERR_INVALID_ARG;
-  if (opt->page_tokens != PAGE_TOKENS || opt->reserved != 0) return KVP_ERR_INVALID_ARG;
+  if (opt->page_tokens != PAGE_TOKENS || (opt->flags & ~(KVP_OPT_FUSED_KV_PRED | KVP_OPT_FUSED_NORM)) != 0) return KVP_ERR_INVALID_ARG;
   if (opt->predictor_bias != 0 && opt->predictor_bias != 1) return KVP_ERR_INVALID_ARG;
   if (aux->vocab != base->vocab) return KVP_ERR_SHAPE;   // one token stream feeds both models
   if (unsupported_model(aux) || unsupported_model(base)) return KVP_ERR_UNSUPPORTED;
@@ -445,6 +448,12 @@ kvp_status kvp_create(const kvp_model_cfg* aux, const kvp_model_cfg* base, const
       ++g.n_seg;
     }
     int dout = g.col0[g.n_seg];
+    // The predictor's input has to carry more than bf16's 8 significant bits (the logits amplify its rounding).
+    // Where everything on its way runs on the tensor cores, K_A / V_A travel as IEEE halves and FK / FV are
+    // stored as halves (exact for |w| >= 2^-14, absolute error <= 2^-25 below): one MMA pass.  Otherwise K_A / V_A
+    // travel as a bf16 value plus its bf16 remainder and the matrices stay in the run dtype: two passes.
+    g.half_path = bf && (h->aux.L[j].hd == 64 || h->aux.L[j].hd == 128) && h->aux.d % 8 == 0 && g.din % 8 == 0 &&
+                  h->base.L[0].hd % 32 == 0;
     if (dout == 0) continue;
     g.fk = take((size_t)dout * g.din * h->es);
     g.fv = take((size_t)dout * g.din * h->es);
@@ -459,9 +468,10 @@ kvp_status kvp_create(const kvp_model_cfg* aux, const kvp_model_cfg* base, const
       int i = g.base_layer[s], dout = g.col0[s + 1] - g.col0[s];
       char b[64];
       snprintf(b, sizeof b, "pred.L%d.fk", i);
-      h->slots[b] = PackSlot{g.fk + (size_t)g.col0[s] * g.din * h->es, dout, g.din, opt->dtype, RowMap{0, 0, 0, 0}};
+      const int f_dtype = g.half_path ? 2 : opt->dtype;
+      h->slots[b] = PackSlot{g.fk + (size_t)g.col0[s] * g.din * h->es, dout, g.din, f_dtype, RowMap{0, 0, 0, 0}};
       snprintf(b, sizeof b, "pred.L%d.fv", i);
-      h->slots[b] = PackSlot{g.fv + (size_t)g.col0[s] * g.din * h->es, dout, g.din, opt->dtype, RowMap{0, 0, 0, 0}};
+      h->slots[b] = PackSlot{g.fv + (size_t)g.col0[s] * g.din * h->es, dout, g.din, f_dtype, RowMap{0, 0, 0, 0}};
       if (opt->predictor_bias) {
         snprintf(b, sizeof b, "pred.L%d.bk", i);
         h->slots[b] = PackSlot{g.bk + (size_t)g.col0[s] * 4, 1, dout, 0, RowMap{0, 0, 0, 0}};
@@ -591,6 +601,24 @@ static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int
 
   KVP_TIMED(KVP_CLASS_OTHER, launch_build_index(ctx, cs.cu.data(), batch, T, cu_dev, tok_pos, tok_slot, last_idx, cache->block_table,
                      cache->max_pages_per_seq, cache->n_pages, cache->seq_lens));
+  // RMSNorm is folded into the GEMMs around it wherever both neighbours run on the tensor cores: the residual GEMM
+  // that completes x writes bf16(x * gain) and the rows' sums of squares, the next GEMM scales its accumulator rows
+  // by 1 / rms.  fused_in[j][0 / 1]: layer j's QKV / gate-up projection takes its operand that way.
+  float* norm_ss = (float*)(ws + w.norm_ss);
+  // (the producer needs every output tile to belong to one CTA: enough tiles for the SMs the GEMMs of this call get)
+  const int sms_for_gemms = (h->side != nullptr && !h->timing && T <= 4096 && h->step_sms > 0) ? h->n_sm - h->step_sms : h->n_sm;
+  const bool can_fuse = (h->opt.flags & KVP_OPT_FUSED_NORM) != 0 && tc_gemm_resid_can_fuse(T, A.d, h->n_sm) &&
+                        tc_gemm_resid_can_fuse(T, A.d, sms_for_gemms);
+  if (can_fuse) cudaMemsetAsync(norm_ss, 0, (size_t)2 * A.n_layers * T * 4, s);
+  auto shape_ok = [&](int K, int N) { return can_fuse && h->opt.dtype == KVP_BF16 && K % 8 == 0 && N % 8 == 0 && A.d % 8 == 0; };
+  std::vector<char> fused_in(2 * (h->j_max + 1), 0);
+  for (int j = 0; j <= h->j_max; ++j) {
+    const LayerPlan& L = A.L[j];
+    const bool hd_ok = L.hd == 64 || L.hd == 128;
+    // QKV of layer j (j >= 1) is fed by layer j-1's down projection; gate/up of layer j by its own O projection
+    if (j >= 1 && hd_ok && shape_ok(A.d, L.nqkv) && shape_ok(A.L[j - 1].ffn, A.d)) fused_in[2 * j] = 1;
+    if (j < h->j_max && L.ffn % 64 == 0 && shape_ok(A.d, 2 * L.ffn) && shape_ok(L.dq, A.d)) fused_in[2 * j + 1] = 1;
+  }
   int2* attn_sched = (int2*)(ws + w.attn_sched);
   // two query tiles per CTA share their K/V tiles; with so few tokens that even the widest layer's pairs
   // would leave SMs idle, one tile per CTA finishes sooner
@@ -643,23 +671,65 @@ static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int
   for (int j = 0; j <= h->j_max; ++j) {
     const LayerPlan& L = A.L[j];
     const bool last = (j == h->j_max);   // only K and V of the last mapped layer are needed
-    KVP_TIMED(KVP_CLASS_OTHER, launch_rmsnorm(ctx, x, (const float*)(P + L.attn_norm), A.eps, T, A.d, hbuf, h->opt.dtype, h_lo));
-    int col_begin = last ? L.dq : 0;
-    const int n_out = L.nqkv - col_begin, q_heads = last ? 0 : L.nq;
-    if (pending_join) {   // the previous layer's predictor still reads the K/V buffers this projection overwrites
-      cudaStreamWaitEvent(s, h->ev_join, 0);
-      pending_join = false;
+    const bool qkv_fused = fused_in[2 * j] != 0, gu_fused = fused_in[2 * j + 1] != 0;
+    const bool next_fused = !last && fused_in[2 * (j + 1)] != 0;
+    if (!qkv_fused)
+      KVP_TIMED(KVP_CLASS_OTHER, launch_rmsnorm(ctx, x, (const float*)(P + L.attn_norm), A.eps, T, A.d, hbuf, h->opt.dtype, h_lo));
+    // predictor of this layer: K_hat_i = K_A,j FK_i^T, V_hat_i = V_A,j FV_i^T for every base layer i with j_i = j
+    const PredGroup& pg = h->groups[j];
+    const bool half_path = pg.half_path;
+    PagedOut paged[2];
+    for (int kv = 0; kv < 2; ++kv) {
+      PagedOut& q = paged[kv];
+      q.n_seg = pg.n_seg;
+      for (int sg = 0; sg <= pg.n_seg; ++sg) q.col0[sg] = pg.col0[sg];
+      for (int sg = 0; sg < pg.n_seg; ++sg) {
+        int i = pg.base_layer[sg];
+        q.n_kv[sg] = h->base.L[i].nkv;
+        q.pool[sg] = kv ? cache->v_pools[i] : cache->k_pools[i];
+      }
+      q.bias = h->opt.predictor_bias ? (const float*)(P + (kv ? pg.bv : pg.bk)) : nullptr;
+      q.tok_slot = tok_slot;
+      q.head_dim = h->base.L[0].hd;
     }
+    // With enough tokens to give every SM a work item, the K/V projection and the predictor are ONE kernel: the
+    // predictor is the projection's epilogue and K_A / V_A reach it through shared memory.
+    KvPred kp{};
+    kp.A = (const bf16*)hbuf; kp.lda = A.d; kp.A_lo = (const bf16*)h_lo; kp.lda_lo = A.d;
+    kp.Wkv = (const bf16*)(P + L.wqkv + (size_t)L.dq * A.d * es); kp.ldw = A.d; kp.M = T; kp.K = A.d;
+    kp.dkv = L.dkv; kp.hd = L.hd; kp.kv_begin = 0; kp.kv_end = 2;
+    if (qkv_fused) { kp.ss_in = norm_ss + (size_t)(2 * j) * T; kp.rms_eps = A.eps; }
+    kp.rope_tab = rope_tab; kp.tok_pos = tok_pos; kp.k_gain = A.qk_norm ? (const float*)(P + L.k_norm) : nullptr; kp.eps = A.eps;
+    kp.C = (bf16*)qkv; kp.ldc = L.nqkv; kp.k_col = L.dq;
+    kp.FK = P + pg.fk; kp.FV = P + pg.fv; kp.n_tot = pg.col0[pg.n_seg]; kp.paged[0] = paged[0]; kp.paged[1] = paged[1];
+    kp.n_sm = h->gemm_sms;
+    const bool fused_kv = (h->opt.flags & KVP_OPT_FUSED_KV_PRED) != 0 && half_path && split && pg.n_seg > 0 && 2 * ((T + 127) / 128) >= h->n_sm && kvpred_tc_supported(kp);
+    int col_begin = last ? L.dq : 0;
+    int n_out = L.nqkv - col_begin;
+    const int q_heads = last ? 0 : L.nq;
+    if (fused_kv) { col_begin = 0; n_out = L.dq; }      // the GEMM below projects the queries only
     TcGemm tq{};
     tq.A = (const bf16*)hbuf; tq.lda = A.d; tq.A2 = (const bf16*)h_lo; tq.lda2 = A.d; tq.split_begin = L.dq - col_begin;
     tq.W = (const bf16*)(P + L.wqkv + (size_t)col_begin * A.d * es); tq.ldw = A.d; tq.M = T; tq.N = n_out; tq.K = A.d;
     tq.epi = TC_QKV; tq.C = (bf16*)(qkv + (size_t)col_begin * es); tq.ldc = L.nqkv;
     tq.C_lo = (bf16*)kv_lo; tq.ld_lo = 2 * L.dkv; tq.lo_col_begin = q_heads * L.hd;
     tq.rot_cols = (q_heads + L.nkv) * L.hd; tq.hd = L.hd; tq.rope_tab = rope_tab; tq.tok_pos = tok_pos;
+    if (fused_kv) { tq.C_lo = nullptr; tq.rot_cols = q_heads * L.hd; tq.A2 = nullptr; }
     const float* qn = A.qk_norm ? (const float*)(P + L.q_norm) : nullptr;
     const float* kn = A.qk_norm ? (const float*)(P + L.k_norm) : nullptr;
     tq.q_gain = qn; tq.k_gain = kn; tq.q_cols = q_heads * L.hd; tq.eps = A.eps;
-    if (!try_tc(h, ctx, tq, KVP_CLASS_AUX_GEMM, &tc_err)) {
+    if (qkv_fused) { tq.ss_in = norm_ss + (size_t)(2 * j) * T; tq.rms_eps = A.eps; }
+    tq.lo_is_half = half_path ? 1 : 0;
+    if (fused_kv) {
+      TimedScope ts(h, ctx.st, KVP_CLASS_KV_PRED);
+      cudaError_t e = launch_kvpred_tc(kp, ctx.status, ctx.st, ctx.n_launch);
+      if (e != cudaSuccess && tc_err == cudaSuccess) tc_err = e;
+    }
+    if (fused_kv && last) {
+      // only keys and values of the last mapped layer are needed: nothing else to project
+    } else if (!try_tc(h, ctx, tq, KVP_CLASS_AUX_GEMM, &tc_err)) {
+      if (half_path && h->groups[j].n_seg > 0) return fail(h, KVP_ERR_CUDA, "internal: half-precision predictor input planned for a projection the tensor-core kernel refuses");
+      if (qkv_fused) return fail(h, KVP_ERR_CUDA, "internal: fused norm planned for a projection the tensor-core kernel refuses");
       GemmArgs g{};
       g.A = hbuf; g.lda = A.d; g.M = T; g.K = A.d;
       g.A2 = h_lo; g.lda2 = A.d;
@@ -670,8 +740,6 @@ static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int
       KVP_TIMED(KVP_CLASS_OTHER, launch_rope_split(ctx, qkv32, g.N, T, g.N / L.hd, q_heads + L.nkv, L.hd, tok_pos, A.theta,
                                                    qkv + (size_t)col_begin * es, L.nqkv, kv_lo, 2 * L.dkv, q_heads, q_heads, qn, kn, A.eps));
     }
-    // predictor: K_hat_i = K_A,j FK_i^T, V_hat_i = V_A,j FV_i^T for every base layer i with j_i = j
-    const PredGroup& pg = h->groups[j];
     if (pg.n_seg > 0) {
       LaunchCtx pctx = ctx;
       if (fork) {
@@ -680,26 +748,22 @@ static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int
         pctx.st = h->side;
       }
       const LaunchCtx& ctx = pctx;      // the predictor's launches go to the side stream
-      for (int kv = 0; kv < 2; ++kv) {
+      for (int kv = 0; kv < 2 && !fused_kv; ++kv) {
         GemmArgs p{};
         p.A = qkv + (size_t)(L.dq + kv * L.dkv) * es; p.lda = L.nqkv; p.M = T; p.K = L.dkv;
         if (split) { p.A2 = kv_lo + (size_t)(kv * L.dkv) * es; p.lda2 = 2 * L.dkv; p.split_begin = 0; }
         p.W = P + (kv ? pg.fv : pg.fk); p.ldw = L.dkv; p.N = pg.col0[pg.n_seg];
-        p.paged.n_seg = pg.n_seg;
-        for (int sg = 0; sg <= pg.n_seg; ++sg) p.paged.col0[sg] = pg.col0[sg];
-        for (int sg = 0; sg < pg.n_seg; ++sg) {
-          int i = pg.base_layer[sg];
-          p.paged.n_kv[sg] = h->base.L[i].nkv;
-          p.paged.pool[sg] = kv ? cache->v_pools[i] : cache->k_pools[i];
-        }
-        p.paged.bias = h->opt.predictor_bias ? (const float*)(P + (kv ? pg.bv : pg.bk)) : nullptr;
-        p.paged.tok_slot = tok_slot;
-        p.paged.head_dim = h->base.L[0].hd;
+        p.paged = paged[kv];
         TcGemm tp{};
         tp.A = (const bf16*)p.A; tp.lda = p.lda; tp.A2 = (const bf16*)p.A2; tp.lda2 = p.lda2; tp.split_begin = 0;
         tp.W = (const bf16*)p.W; tp.ldw = p.ldw; tp.M = T; tp.N = p.N; tp.K = p.K; tp.epi = TC_PAGED; tp.paged = p.paged;
-        if (!try_tc(h, ctx, tp, KVP_CLASS_PREDICTOR, &tc_err))
-          KVP_TIMED(KVP_CLASS_PREDICTOR, launch_gemm_simt(ctx, p, EPI_PAGED));
+        if (half_path) {     // K_A / V_A as halves (written by the projection's epilogue), FK / FV stored as halves: one pass
+          tp.A = (const bf16*)(kv_lo + (size_t)(kv * L.dkv) * es); tp.lda = 2 * L.dkv; tp.A2 = nullptr; tp.f16_operands = 1;
+        }
+        if (!try_tc(h, ctx, tp, KVP_CLASS_PREDICTOR, &tc_err)) {
+          if (half_path) tc_err = cudaErrorInvalidValue;    // the matrices are stored as halves: no other kernel reads them
+          else KVP_TIMED(KVP_CLASS_PREDICTOR, launch_gemm_simt(ctx, p, EPI_PAGED));
+        }
       }
       if (fork) {
         cudaEventRecord(h->ev_join, h->side);
@@ -743,14 +807,24 @@ static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int
     TcGemm to{};
     to.A = (const bf16*)attn; to.lda = L.dq; to.W = (const bf16*)(P + L.wo); to.ldw = L.dq; to.M = T; to.N = A.d; to.K = L.dq;
     to.epi = TC_RESID; to.X = x; to.ldx = A.d;
-    if (!try_tc(h, ctx, to, KVP_CLASS_AUX_GEMM, &tc_err)) KVP_TIMED(KVP_CLASS_AUX_GEMM, launch_gemm_simt(ctx, o, EPI_RESID));
-    KVP_TIMED(KVP_CLASS_OTHER, launch_rmsnorm(ctx, x, (const float*)(P + L.ffn_norm), A.eps, T, A.d, hbuf, h->opt.dtype));
+    if (gu_fused) {      // the O projection completes x: it also writes the gate/up projection's operand
+      to.H = (bf16*)hbuf; to.ldh = A.d; to.gain_next = (const float*)(P + L.ffn_norm);
+      to.ss_out = norm_ss + (size_t)(2 * j + 1) * T;
+    }
+    if (!try_tc(h, ctx, to, KVP_CLASS_AUX_GEMM, &tc_err)) {
+      if (gu_fused) return fail(h, KVP_ERR_CUDA, "internal: fused norm planned for a projection the tensor-core kernel refuses");
+      KVP_TIMED(KVP_CLASS_AUX_GEMM, launch_gemm_simt(ctx, o, EPI_RESID));
+    }
+    if (!gu_fused)
+      KVP_TIMED(KVP_CLASS_OTHER, launch_rmsnorm(ctx, x, (const float*)(P + L.ffn_norm), A.eps, T, A.d, hbuf, h->opt.dtype));
     GemmArgs f{};
     f.A = hbuf; f.lda = A.d; f.W = P + L.wgu; f.ldw = A.d; f.M = T; f.N = 2 * L.ffn; f.K = A.d; f.C = gu; f.ldc = 2 * L.ffn;
     TcGemm tf{};
     tf.A = (const bf16*)hbuf; tf.lda = A.d; tf.W = (const bf16*)(P + L.wgu); tf.ldw = A.d; tf.M = T; tf.N = 2 * L.ffn; tf.K = A.d;
     tf.epi = TC_SWIGLU; tf.C = (bf16*)act; tf.ldc = L.ffn; tf.ffn = L.G == 64 ? L.ffn : 1;
+    if (gu_fused) { tf.ss_in = norm_ss + (size_t)(2 * j + 1) * T; tf.rms_eps = A.eps; }
     if (!try_tc(h, ctx, tf, KVP_CLASS_AUX_GEMM, &tc_err)) {
+      if (gu_fused) return fail(h, KVP_ERR_CUDA, "internal: fused norm planned for a projection the tensor-core kernel refuses");
       KVP_TIMED(KVP_CLASS_AUX_GEMM, launch_gemm_simt(ctx, f, EPI_STORE));
       KVP_TIMED(KVP_CLASS_OTHER, launch_swiglu(ctx, gu, T, L.ffn, L.G, act));
     }
@@ -759,7 +833,14 @@ static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int
     TcGemm td{};
     td.A = (const bf16*)act; td.lda = L.ffn; td.W = (const bf16*)(P + L.wd); td.ldw = L.ffn; td.M = T; td.N = A.d; td.K = L.ffn;
     td.epi = TC_RESID; td.X = x; td.ldx = A.d;
-    if (!try_tc(h, ctx, td, KVP_CLASS_AUX_GEMM, &tc_err)) KVP_TIMED(KVP_CLASS_AUX_GEMM, launch_gemm_simt(ctx, d, EPI_RESID));
+    if (next_fused) {    // the down projection completes x: it also writes the next layer's QKV operand (hi + lo parts)
+      td.H = (bf16*)hbuf; td.H_lo = (bf16*)h_lo; td.ldh = A.d; td.gain_next = (const float*)(P + A.L[j + 1].attn_norm);
+      td.ss_out = norm_ss + (size_t)(2 * (j + 1)) * T;
+    }
+    if (!try_tc(h, ctx, td, KVP_CLASS_AUX_GEMM, &tc_err)) {
+      if (next_fused) return fail(h, KVP_ERR_CUDA, "internal: fused norm planned for a projection the tensor-core kernel refuses");
+      KVP_TIMED(KVP_CLASS_AUX_GEMM, launch_gemm_simt(ctx, d, EPI_RESID));
+    }
   }
   if (pending_join) cudaStreamWaitEvent(s, h->ev_join, 0);     // the base step reads what the predictor wrote
   h->gemm_sms = h->step_grid_sms = h->n_sm;

@@ -35,6 +35,7 @@ struct PredGroup {
   int col0[MAX_PRED_SEG + 1];
   int din;
   size_t fk, fv, bk, bv;
+  bool half_path;     // FK / FV stored as IEEE halves; K_A / V_A reach the predictor as halves in one pass
 };
 
 struct PackSlot {
@@ -46,7 +47,7 @@ struct PackSlot {
 
 struct WsLayout {
   size_t status, cu, last_idx, tok_pos, tok_slot, rope_tab, x, h, h_lo, qkv, qkv32, kv_lo, attn, gu, act;
-  size_t xb, hb, qkvb, ab, actb, part, tok_stage, first_stage, xbt, gub, attn_sched, attn_done, total;
+  size_t xb, hb, qkvb, ab, actb, part, tok_stage, first_stage, xbt, gub, attn_sched, attn_done, norm_ss, total;
 };
 
 struct kvp_handle {

@@ -64,10 +64,10 @@ class ArgmaxTally:
                          for m in self.mismatches)
 
 
-def make_session(pair, W, prompts, extra_len=0):
+def make_session(pair, W, prompts, extra_len=0, flags=0):
     import paper_2410_08391_b200 as kvp
     return kvp.Session(pair, W, max_batch=prompts.batch, max_total_tokens=prompts.total,
-                       max_len=int(prompts.lengths.max()), extra_len=extra_len)
+                       max_len=int(prompts.lengths.max()), extra_len=extra_len, flags=flags)
 
 
 def run_prefill(sess, prompts):

@@ -56,6 +56,8 @@ CASES = [
     ("t_hd128_qkn", [40, 9, 130, 17, 64, 65, 3, 90, 128], "fanin"),
     ("t_small_qkn", [4200, 70], "fanin"),
     ("t_small_qkn", [1, 2, 3, 5, 8, 13, 21, 34, 55, 89] * 13, "fanin"),
+    # many tokens: several waves of tiles per SM in every kernel of the prefill
+    ("t_small", [1900] * 9 + [1901], "fanin"),
     # other group sizes of the step attention over the bf16 cache (1, 2 and 8 query heads per kv head), with more
     # than 4 sequences and with a small batch over a long cache
     ("t_mha", [40, 9, 130, 17, 64, 65], "fanin"),
@@ -86,6 +88,26 @@ def test_prefill_predict_matches_oracle(name, lens, regime):
             assert len(tally.mismatches) <= max(1, tally.compared // 50), tally.report()
         else:
             assert not tally.mismatches, tally.report()
+    finally:
+        s.close()
+
+
+@pytest.mark.parametrize("flags", [1, 2, 3])
+@pytest.mark.parametrize("name,lens,regime", [("t_small", [1900] * 9 + [1901], "fanin"), ("t_hd128", [1300] * 9 + [1207], "n002"),
+                                              ("t_small_qkn", [1900] * 10, "fanin"), ("t_bias", [1900] * 10, "fanin"),
+                                              ("t_scaled", [1500] * 13, "fanin")],
+                         ids=lambda v: str(v).replace(" ", "")[:40])
+def test_kernel_variants_match_oracle(name, lens, regime, flags):
+    """The optional kernel variants (kvp_options.flags: K/V projection + predictor as one kernel; RMSNorm folded into
+    the GEMMs around it) on calls large enough for them to be taken: same results within the same tolerances."""
+    pair = wl.pair(name)
+    W = wl.make_weights(pair, seed=1, regime=regime)
+    pr = wl.custom_prompts(pair.base.vocab, lens, seed=1)
+    s = make_session(pair, W, pr, flags=flags)
+    try:
+        ek, ev, el, tally = compare_prefill(s, pair, W, pr, seqs=[0, len(lens) - 1])
+        print(f"{name} flags {flags}: K {ek:.2e} V {ev:.2e} logits {el:.2e}")
+        assert not tally.mismatches, tally.report()
     finally:
         s.close()
 
