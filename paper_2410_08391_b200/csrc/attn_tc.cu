@@ -5,8 +5,12 @@
 // [T, q|k|v] projection buffer; both query tiles use them.  Warp 1 issues S = Q K^T and
 // O += P V with tcgen05.mma; S and O of both query tiles live in tensor memory.  Two groups of
 // four warps, one per query tile, own one query row per thread: a thread reads its row of S
-// into registers in one go (which frees S for the next key tile at once), keeps the running
-// max / sum in fp32 and writes P as bf16 into shared memory in the swizzled operand layout.
+// into registers in one go, keeps the running max / sum in fp32 and writes P as packed bf16
+// back into tensor memory, from where the P V product takes it as its A operand (P never
+// touches shared memory).  head_dim 64: P has columns of its own, so S of the next key tile is
+// computed while the softmax of this one runs; head_dim 128: tensor memory is full (2 x S, 2 x O),
+// P overwrites the first half of its S, and the two query tiles take turns: one tile's softmax
+// runs while the tensor core works on the other tile's P V and next S.
 // O is accumulated by the tensor core itself and only touched when a row's maximum has grown
 // by more than 2^8 since the exponent offset was last fixed; then the group rescales its O in
 // tensor memory (tcgen05.ld / st).  While one group computes exponentials the tensor core works
@@ -22,15 +26,19 @@ using namespace tcp;
 
 constexpr int BQ = 128;                 // queries per tile; a CTA has two tiles
 constexpr int N_THREADS = 320;          // warps: 0 TMA, 1 MMA, 2-5 tile 0, 6-9 tile 1
-constexpr int STAGES = 3;
+constexpr int MAX_STAGES = 4;
 constexpr float RESCALE_LOG2 = 8.f;     // tolerated growth of a row maximum before O is rescaled
 
 template <int HD> struct Cfg {
-  static constexpr int BKV = HD == 64 ? 128 : 64;       // keys per tile
+  static constexpr int BKV = 128;                       // keys per tile
+  static constexpr int STAGES = HD == 64 ? 4 : 2;       // K/V tile pairs in flight (32 / 64 KiB each)
   static constexpr int Q_BYTES = BQ * HD * 2;
   static constexpr int KV_BYTES = BKV * HD * 2;         // a K or a V tile
-  static constexpr int P_BYTES = BQ * BKV * 2;
-  static constexpr int SMEM = 2 * Q_BYTES + 2 * P_BYTES + STAGES * 2 * KV_BYTES + 1024 + 256;
+  static constexpr int SMEM = 2 * Q_BYTES + STAGES * 2 * KV_BYTES + 1024 + 256;
+  // tensor-memory columns: S of tile g, O of tile g, P of tile g (packed bf16: 64 columns for 128 keys)
+  static constexpr int S_COL = 0, O_COL = 256;
+  static constexpr bool P_ALIASES_S = HD == 128;
+  static constexpr int P_COL = P_ALIASES_S ? 0 : 384, P_STRIDE = P_ALIASES_S ? 128 : 64;
 };
 
 __device__ __forceinline__ float fast_exp2(float x) {
@@ -38,12 +46,27 @@ __device__ __forceinline__ float fast_exp2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
 // MN-major operand tile: 64 contiguous MN elements per 128-byte row, rows = K index, 8-row groups
 // 1024 B apart (stride offset), next 64 MN elements `lbo` bytes away (leading offset)
 __device__ __forceinline__ uint64_t desc_mnmajor(uint32_t addr, uint32_t lbo) {
   uint64_t lo = ((addr & 0x3FFFFu) >> 4) | ((uint64_t)((lbo >> 4) & 0x3FFFu) << 16);
   uint64_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);
   return lo | (hi << 32);
+}
+
+// D += A B with A taken from tensor memory (row i of A in lane i, two 16-bit elements per 32-bit column)
+__device__ __forceinline__ void tc_mma_bf16_ta(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
 }
 
 struct Params {
@@ -59,14 +82,14 @@ template <int HD>
 __global__ void __launch_bounds__(N_THREADS, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kv, const Params p) {
   using C = Cfg<HD>;
-  constexpr int BKV = C::BKV, QB = C::Q_BYTES, KB = C::KV_BYTES, PB = C::P_BYTES, NBOX = HD / 64;
+  constexpr int BKV = C::BKV, QB = C::Q_BYTES, KB = C::KV_BYTES, NBOX = HD / 64, STAGES = C::STAGES;
   constexpr int KV_BOX = BKV * 128;     // bytes of one 64-column box of a K or V tile
   extern __shared__ uint8_t smem_raw[];
   pdl_trigger();
   if (threadIdx.x == 32) { prefetch_tensormap(&map_q); prefetch_tensormap(&map_kv); }
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  const uint32_t sQ = smem_u32(smem), sP = sQ + 2 * QB, sKV = sP + 2 * PB;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 2 * QB + 2 * PB + STAGES * 2 * KB);
+  const uint32_t sQ = smem_u32(smem), sKV = sQ + 2 * QB;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 2 * QB + STAGES * 2 * KB);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 9);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const uint32_t bar_base = smem_u32(bars);
@@ -86,7 +109,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  // tensor memory: S of tile g at column 128 g, O of tile g at column 256 + 128 g
+  // tensor memory: S of tile g at column 128 g, O of tile g at column 256 + HD g, P: see Cfg
   if (warp == 1) tmem_alloc(smem_u32(tmem_slot), 512);
   tc_fence_before();
   __syncthreads();
@@ -161,15 +184,18 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             tc_fence_after();
             const uint32_t sv = sKV + (jp[g] % STAGES) * 2 * KB + KB;
 #pragma unroll
-            for (int kk = 0; kk < BKV / 16; ++kk)
-              tc_mma_bf16(tmem_base + 256 + g * 128, desc_kmajor(sP + g * PB + (kk >> 2) * 16384 + (kk & 3) * 32),
-                          desc_mnmajor(sv + kk * 2048, KV_BOX), idesc_pv, (jp[g] > 0 || kk > 0) ? 1u : 0u);
+            for (int kk = 0; kk < BKV / 16; ++kk)      // 16 keys = 8 packed columns of P per step
+              tc_mma_bf16_ta(tmem_base + C::O_COL + g * HD, tmem_base + C::P_COL + g * C::P_STRIDE + kk * 8,
+                             desc_mnmajor(sv + kk * 2048, KV_BOX), idesc_pv, (jp[g] > 0 || kk > 0) ? 1u : 0u);
             tc_commit(pv_done(g));
             ++jp[g];
             progress = true;
           }
-          // S of the next key tile: its K tile has landed and the group holds the previous S in registers
-          if (js[g] < n_kv[g] && mbar_poll(s_free(g), (js[g] - 1) & 1) && mbar_poll(kv_full(js[g] % STAGES), (js[g] / STAGES) & 1)) {
+          // S of the next key tile: its K tile has landed, and the columns are free: with P in columns of its own once
+          // the group holds the previous S in registers; where P overwrites S, once the P V product that reads it has
+          // been issued (the tensor core executes in issue order)
+          if (js[g] < n_kv[g] && (C::P_ALIASES_S ? jp[g] >= js[g] : mbar_poll(s_free(g), (js[g] - 1) & 1)) &&
+              mbar_poll(kv_full(js[g] % STAGES), (js[g] / STAGES) & 1)) {
             tc_fence_after();
             issue_s(g, js[g] % STAGES);
             ++js[g];
@@ -200,8 +226,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     const int r = quarter * 32 + lane;          // row of the query tile owned by this thread
     const int qs = q0 + g * BQ, q_pos = qs + r;
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
-    const uint32_t tS = tmem_base + lane_off + g * 128, tO = tmem_base + lane_off + 256 + g * 128;
-    const uint32_t sPg = sP + g * PB;
+    const uint32_t tS = tmem_base + lane_off + C::S_COL + g * 128, tO = tmem_base + lane_off + C::O_COL + g * HD;
+    const uint32_t tP = tmem_base + lane_off + C::P_COL + g * C::P_STRIDE;
     const float c = p.scale_log2e;
     const int n = n_kv[g];
     float m_ref = -INFINITY, l = 0.f;
@@ -224,10 +250,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 #pragma unroll
         for (int i = 0; i < BKV; ++i) if (kbase + i > q_pos) s[i] = -INFINITY;
       }
-      float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};    // four chains instead of one of length BKV
+      float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};    // four chains of three-input maxima
 #pragma unroll
-      for (int i = 0; i < BKV; i += 4) {
-        mx[0] = fmaxf(mx[0], s[i]); mx[1] = fmaxf(mx[1], s[i + 1]); mx[2] = fmaxf(mx[2], s[i + 2]); mx[3] = fmaxf(mx[3], s[i + 3]);
+      for (int i = 0; i < BKV; i += 8) {
+        mx[0] = fmax3(mx[0], s[i], s[i + 1]); mx[1] = fmax3(mx[1], s[i + 2], s[i + 3]);
+        mx[2] = fmax3(mx[2], s[i + 4], s[i + 5]); mx[3] = fmax3(mx[3], s[i + 6], s[i + 7]);
       }
       const float mt = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
       if (j > 0) {     // the previous P V product has read P and finished writing O
@@ -255,22 +282,29 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         if (need) m_ref = mt;
       }
       const float mc = (m_ref == -INFINITY) ? 0.f : m_ref * c;
-      float rs[4] = {0.f, 0.f, 0.f, 0.f};
+      float2 rs2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+      const float2 c2 = make_float2(c, c), nmc2 = make_float2(-mc, -mc);
 #pragma unroll
-      for (int g8 = 0; g8 < BKV / 8; ++g8) {
-        float e[8];
+      for (int hf = 0; hf < BKV / 64; ++hf) {        // 64 keys = 32 packed columns of P per tensor-memory store
+        uint32_t pk[32];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) { e[i] = fast_exp2(s[g8 * 8 + i] * c - mc); rs[i & 3] += e[i]; }   // exp2(-inf) = 0
-        const int k0 = g8 * 8;
-        const uint32_t addr = sPg + (k0 >> 6) * 16384 + r * 128 + ((((k0 & 63) >> 3) ^ (r & 7)) << 4);
-        __nv_bfloat162 a0 = __floats2bfloat162_rn(e[0], e[1]), a1 = __floats2bfloat162_rn(e[2], e[3]);
-        __nv_bfloat162 a2 = __floats2bfloat162_rn(e[4], e[5]), a3 = __floats2bfloat162_rn(e[6], e[7]);
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(*reinterpret_cast<uint32_t*>(&a0)),
-                     "r"(*reinterpret_cast<uint32_t*>(&a1)), "r"(*reinterpret_cast<uint32_t*>(&a2)),
-                     "r"(*reinterpret_cast<uint32_t*>(&a3)) : "memory");
+        for (int g8 = 0; g8 < 8; ++g8) {
+          const int k0 = hf * 64 + g8 * 8;
+          float2 x[4];
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            x[q] = __ffma2_rn(make_float2(s[k0 + 2 * q], s[k0 + 2 * q + 1]), c2, nmc2);     // two scaled scores per instruction
+            x[q].x = fast_exp2(x[q].x); x[q].y = fast_exp2(x[q].y);                      // exp2(-inf) = 0
+            const __nv_bfloat162 h2 = __floats2bfloat162_rn(x[q].x, x[q].y);              // key 2i in the low half of column i
+            pk[g8 * 4 + q] = *reinterpret_cast<const uint32_t*>(&h2);
+          }
+          rs2[0] = __fadd2_rn(rs2[0], x[0]); rs2[1] = __fadd2_rn(rs2[1], x[1]);
+          rs2[0] = __fadd2_rn(rs2[0], x[2]); rs2[1] = __fadd2_rn(rs2[1], x[3]);
+        }
+        tmem_st32(tP + hf * 32, reinterpret_cast<const float*>(pk));
       }
-      l += (rs[0] + rs[1]) + (rs[2] + rs[3]);
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P visible to the tensor core's reads
+      tmem_st_wait();
+      l += (rs2[0].x + rs2[0].y) + (rs2[1].x + rs2[1].y);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(p_ready(g));
@@ -370,7 +404,7 @@ void launch_attn_schedule(const int* cu_dev, int batch, int tiles, int2* sched, 
 cudaError_t launch_attn_tc(const bf16* qkv, int ld, int total, int nq, int nkv, int hd, const int* cu_dev, const int2* sched,
                            int n_items, int tiles, bf16* out, int ldo, int* status, cudaStream_t st, int64_t* n_launch) {
   CUtensorMap mq, mkv;
-  const int bkv = hd == 64 ? 128 : 64;
+  const int bkv = 128;
   if (!tc_make_map_bf16(&mq, qkv, total, (long long)(nq + 2 * nkv) * hd, ld, BQ)) return cudaErrorInvalidValue;
   if (!tc_make_map_bf16(&mkv, qkv, total, (long long)(nq + 2 * nkv) * hd, ld, bkv)) return cudaErrorInvalidValue;
   Params p{cu_dev, sched, nq, nkv, out, ldo, (1.f / sqrtf((float)hd)) * 1.4426950408889634f, status, tiles};
