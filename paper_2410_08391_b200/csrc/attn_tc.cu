@@ -76,9 +76,11 @@ struct Params {
   float scale_log2e;
   int* status;
   int tiles;                            // query tiles per CTA: 2, or 1 when pairs would leave SMs idle
+  bf16* out_lo;                         // bf16 remainder of the output (same layout as out), or null
 };
 
-template <int HD>
+// F16: q, k, v hold IEEE halves instead of bf16 (and P is packed as halves): same kernel, other operand format bits
+template <int HD, bool F16>
 __global__ void __launch_bounds__(N_THREADS, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kv, const Params p) {
   using C = Cfg<HD>;
@@ -154,9 +156,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   } else if (warp == 1) {
     if (lane == 0) {
       // S = Q K^T: M = 128 queries, N = BKV keys, both operands K-major over head_dim
-      const uint32_t idesc_s = idesc_bf16(BQ, BKV);
+      const uint32_t fmt_mask = F16 ? ~((7u << 7) | (7u << 10)) : ~0u;       // operand format fields: 0 = IEEE half
+      const uint32_t idesc_s = idesc_bf16(BQ, BKV) & fmt_mask;
       // O += P V: A = P (K-major over keys), B = V as stored [key][dim] = MN-major, N = head_dim
-      const uint32_t idesc_pv = idesc_bf16(BQ, HD) | (1u << 16);
+      const uint32_t idesc_pv = (idesc_bf16(BQ, HD) & fmt_mask) | (1u << 16);
       auto issue_s = [&](int g, int stage) {
         const uint32_t sk = sKV + stage * 2 * KB;
 #pragma unroll
@@ -295,8 +298,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           for (int q = 0; q < 4; ++q) {
             x[q] = __ffma2_rn(make_float2(s[k0 + 2 * q], s[k0 + 2 * q + 1]), c2, nmc2);     // two scaled scores per instruction
             x[q].x = fast_exp2(x[q].x); x[q].y = fast_exp2(x[q].y);                      // exp2(-inf) = 0
-            const __nv_bfloat162 h2 = __floats2bfloat162_rn(x[q].x, x[q].y);              // key 2i in the low half of column i
-            pk[g8 * 4 + q] = *reinterpret_cast<const uint32_t*>(&h2);
+            if (F16) {                                                                    // key 2i in the low half of column i
+              const __half2 h2 = __floats2half2_rn(x[q].x, x[q].y);
+              pk[g8 * 4 + q] = *reinterpret_cast<const uint32_t*>(&h2);
+            } else {
+              const __nv_bfloat162 h2 = __floats2bfloat162_rn(x[q].x, x[q].y);
+              pk[g8 * 4 + q] = *reinterpret_cast<const uint32_t*>(&h2);
+            }
           }
           rs2[0] = __fadd2_rn(rs2[0], x[0]); rs2[1] = __fadd2_rn(rs2[1], x[1]);
           rs2[0] = __fadd2_rn(rs2[0], x[2]); rs2[1] = __fadd2_rn(rs2[1], x[3]);
@@ -333,6 +341,17 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             u.x = *reinterpret_cast<uint32_t*>(&a0); u.y = *reinterpret_cast<uint32_t*>(&a1);
             u.z = *reinterpret_cast<uint32_t*>(&a2); u.w = *reinterpret_cast<uint32_t*>(&a3);
             *reinterpret_cast<uint4*>(dst + cc + g8 * 8) = u;
+            if (p.out_lo) {
+              float rem[8];
+#pragma unroll
+              for (int i = 0; i < 8; ++i) { const float f = v[g8 * 8 + i] * inv; rem[i] = f - __bfloat162float(__float2bfloat16_rn(f)); }
+              __nv_bfloat162 b0 = __floats2bfloat162_rn(rem[0], rem[1]), b1 = __floats2bfloat162_rn(rem[2], rem[3]);
+              __nv_bfloat162 b2 = __floats2bfloat162_rn(rem[4], rem[5]), b3 = __floats2bfloat162_rn(rem[6], rem[7]);
+              uint4 w;
+              w.x = *reinterpret_cast<uint32_t*>(&b0); w.y = *reinterpret_cast<uint32_t*>(&b1);
+              w.z = *reinterpret_cast<uint32_t*>(&b2); w.w = *reinterpret_cast<uint32_t*>(&b3);
+              *reinterpret_cast<uint4*>(p.out_lo + (size_t)(base + q_pos) * p.ldo + (size_t)head * HD + cc + g8 * 8) = w;
+            }
           }
         }
       }
@@ -377,12 +396,12 @@ __global__ void __launch_bounds__(256) attn_schedule_kernel(const int* __restric
   }
 }
 
-template <int HD>
+template <int HD, bool F16>
 cudaError_t go(const CUtensorMap& mq, const CUtensorMap& mkv, const Params& p, dim3 grid, cudaStream_t st) {
   static bool raised[TC_MAX_DEVICES] = {};
-  cudaError_t e = tc_raise_smem_limit(attn_tc_kernel<HD>, Cfg<HD>::SMEM, raised);
+  cudaError_t e = tc_raise_smem_limit(attn_tc_kernel<HD, F16>, Cfg<HD>::SMEM, raised);
   if (e != cudaSuccess) return e;
-  return launch_overlapped(attn_tc_kernel<HD>, grid, dim3(N_THREADS), Cfg<HD>::SMEM, st, mq, mkv, p);
+  return launch_overlapped(attn_tc_kernel<HD, F16>, grid, dim3(N_THREADS), Cfg<HD>::SMEM, st, mq, mkv, p);
 }
 }  // namespace
 
@@ -402,13 +421,15 @@ void launch_attn_schedule(const int* cu_dev, int batch, int tiles, int2* sched, 
 }
 
 cudaError_t launch_attn_tc(const bf16* qkv, int ld, int total, int nq, int nkv, int hd, const int* cu_dev, const int2* sched,
-                           int n_items, int tiles, bf16* out, int ldo, int* status, cudaStream_t st, int64_t* n_launch) {
+                           int n_items, int tiles, bf16* out, int ldo, int* status, cudaStream_t st, int64_t* n_launch,
+                           bool half_operands, bf16* out_lo) {
   CUtensorMap mq, mkv;
   const int bkv = 128;
   if (!tc_make_map_bf16(&mq, qkv, total, (long long)(nq + 2 * nkv) * hd, ld, BQ)) return cudaErrorInvalidValue;
   if (!tc_make_map_bf16(&mkv, qkv, total, (long long)(nq + 2 * nkv) * hd, ld, bkv)) return cudaErrorInvalidValue;
-  Params p{cu_dev, sched, nq, nkv, out, ldo, (1.f / sqrtf((float)hd)) * 1.4426950408889634f, status, tiles};
+  Params p{cu_dev, sched, nq, nkv, out, ldo, (1.f / sqrtf((float)hd)) * 1.4426950408889634f, status, tiles, out_lo};
   dim3 grid(nq, n_items);
   ++*n_launch;
-  return hd == 64 ? go<64>(mq, mkv, p, grid, st) : go<128>(mq, mkv, p, grid, st);
+  if (half_operands) return hd == 64 ? go<64, true>(mq, mkv, p, grid, st) : go<128, true>(mq, mkv, p, grid, st);
+  return hd == 64 ? go<64, false>(mq, mkv, p, grid, st) : go<128, false>(mq, mkv, p, grid, st);
 }

@@ -165,9 +165,10 @@ void launch_attn_prefill_simt(const LaunchCtx&, const void* qkv, int ld, int nq,
 // qkv: one layer's projection buffer [T, ld], own keys at column k_col, values at k_col + nkv * hd; kv_lo (bf16 mode,
 // may be null): lo parts [T, ld_lo] of keys then values.  sum_k / sum_v (device) += mean |predicted - own|.
 void launch_kv_l1(const LaunchCtx&, const void* qkv, int ld, int k_col, const void* kv_lo, int ld_lo, int T_tokens, int nkv,
-                  int hd, const int* tok_slot, const void* kpool, const void* vpool, float* sum_k, float* sum_v);
+                  int hd, const int* tok_slot, const void* kpool, const void* vpool, float* sum_k, float* sum_v,
+                  bool qkv_is_half = false /* bf16 mode: keys and values of qkv are IEEE halves, no lo parts */);
 void launch_kv_take(const LaunchCtx&, void* qkv, int ld, int k_col, int T_tokens, int nkv, int hd, const int* tok_slot,
-                    const void* kpool, const void* vpool);
+                    const void* kpool, const void* vpool, bool qkv_is_half = false);
 
 // base single-token step
 enum StepGemvMode : int { GEMV_STORE = 0, GEMV_RESID = 1, GEMV_SWIGLU = 2 };

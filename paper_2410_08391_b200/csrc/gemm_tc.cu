@@ -101,6 +101,7 @@ struct Params {
   float* X; int ldx;
   bf16* C_lo; int ld_lo; int lo_col_begin;
   int lo_is_half;        // C_lo receives the whole value as an IEEE half instead of the bf16 remainder
+  int c_is_half;         // TC_QKV: C itself is written as IEEE halves (attention with half operands)
   int f16_operands;      // A and W hold IEEE halves (both operands of one MMA have the same type)
   int rot_cols; int hd;
   const float2* rope_tab; const int* tok_pos;
@@ -240,6 +241,12 @@ __device__ __forceinline__ void epilogue_tile(const Params& p, uint32_t tmem_acc
 #pragma unroll
       for (int i = 0; i < 32; ++i) { const float gi = g[i] * rinv; g[i] = __fdividef(gi, 1.f + __expf(-gi)) * (u[i] * rinv); }
       store32_bf16(p.C + (size_t)m * p.ldc + n, g, n_valid);
+      if (p.C_lo) {        // bf16 remainder of the activation, for a down projection that takes both parts
+        bf16* lo = p.C_lo + (size_t)m * p.ld_lo + n;
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          if (q * 8 < n_valid) *reinterpret_cast<uint4*>(lo + q * 8) = pack8_lo(g + q * 8);
+      }
     }
   } else {  // TC_QKV: RoPE on columns < rot_cols, hi part to C, lo part of columns >= lo_col_begin to C_lo
     int half = p.hd >> 1;
@@ -290,8 +297,16 @@ __device__ __forceinline__ void epilogue_tile(const Params& p, uint32_t tmem_acc
           }
         }
         bf16* dst = p.C + (size_t)m * p.ldc + n;
-        store32_bf16(dst, a, 32);
-        store32_bf16(dst + half, b, 32);
+        if (p.c_is_half) {
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            *reinterpret_cast<uint4*>(dst + g * 8) = pack8_half(a + g * 8);
+            *reinterpret_cast<uint4*>(dst + half + g * 8) = pack8_half(b + g * 8);
+          }
+        } else {
+          store32_bf16(dst, a, 32);
+          store32_bf16(dst + half, b, 32);
+        }
         if (p.C_lo && n >= p.lo_col_begin) {
           bf16* lo = p.C_lo + (size_t)m * p.ld_lo + (n - p.lo_col_begin);
           if (p.lo_is_half) {
@@ -588,7 +603,8 @@ bool tc_gemm_supported(const TcGemm& g) {
       if (g.H && (g.N % 8 || g.ldh % 8 || !al16(g.H) || (g.H_lo && !al16(g.H_lo)) || !g.gain_next || !g.ss_out || g.A2 ||
                   !tc_gemm_resid_can_fuse(g.M, g.N, g.n_sm))) return false;
       return g.N % 4 == 0 && g.ldx % 4 == 0 && al16(g.X);
-    case TC_SWIGLU: return g.ffn % 64 == 0 && g.N == 2 * g.ffn && g.ldc % 8 == 0 && al16(g.C);
+    case TC_SWIGLU:
+      return g.ffn % 64 == 0 && g.N == 2 * g.ffn && g.ldc % 8 == 0 && al16(g.C) && (!g.C_lo || (g.ld_lo % 8 == 0 && al16(g.C_lo)));
     case TC_QKV:
       return (g.hd == 64 || g.hd == 128) && g.N % g.hd == 0 && g.rot_cols % g.hd == 0 && g.lo_col_begin % g.hd == 0 &&
              g.ldc % 8 == 0 && al16(g.C) && (!g.C_lo || (g.ld_lo % 8 == 0 && al16(g.C_lo))) && g.rope_tab && g.tok_pos;
@@ -624,7 +640,7 @@ cudaError_t launch_gemm_tc(const TcGemm& g, int* status, cudaStream_t st, int64_
   p.rot_cols = g.rot_cols; p.hd = g.hd; p.rope_tab = g.rope_tab; p.tok_pos = g.tok_pos; p.ffn = g.ffn; p.paged = g.paged;
   p.H = g.H; p.H_lo = g.H_lo; p.ldh = g.ldh; p.gain_next = g.gain_next; p.ss_out = g.ss_out;
   p.ss_in = g.ss_in; p.rms_eps = g.rms_eps;
-  p.lo_is_half = g.lo_is_half; p.f16_operands = g.f16_operands;
+  p.lo_is_half = g.lo_is_half; p.f16_operands = g.f16_operands; p.c_is_half = g.c_is_half;
   const int tiles = ((g.M + BM - 1) / BM) * ((g.N + bn - 1) / bn);
   const long long kblocks = (long long)tiles * ((g.K + BK - 1) / BK);
   int grid = stream_k ? (int)(kblocks < g.n_sm ? kblocks : g.n_sm) : (tiles < g.n_sm ? tiles : g.n_sm);

@@ -5,7 +5,7 @@
 enum TcEpi : int {
   TC_STORE = 0,   // C[m, n] = bf16(acc)
   TC_RESID = 1,   // X[m, n] += acc (fp32 residual stream)
-  TC_SWIGLU = 2,  // W rows interleaved (64 gate rows, 64 up rows); C[m, c] = bf16(silu(gate_c) * up_c)
+  TC_SWIGLU = 2,  // W rows interleaved (64 gate rows, 64 up rows); C[m, c] = bf16(silu(gate_c) * up_c) (+ remainder to C_lo)
   TC_QKV = 3,     // RoPE on columns < rot_cols, bf16 hi to C, bf16 lo of columns >= lo_col_begin to C_lo
   TC_PAGED = 4    // predictor: columns scattered into cache pages
 };
@@ -36,6 +36,7 @@ struct TcGemm {
   bf16* H; bf16* H_lo; int ldh; const float* gain_next; float* ss_out;
   const float* ss_in; float rms_eps;
   int lo_is_half;                  // TC_QKV: C_lo receives the whole value as an IEEE half (not the bf16 remainder)
+  int c_is_half;                   // TC_QKV: C is written as IEEE halves (for an attention that takes half operands)
   int f16_operands;                // A and W hold IEEE halves instead of bf16 (same 2 bytes; both operands alike)
   int n_sm;
   int bn;                          // tile width: 128, 256, or 0 = chosen by the launcher

@@ -1032,7 +1032,7 @@ kvp_status kvp_poll_status(kvp_handle* h, void* workspace, void* stream) {
 // ---- training-time forward (Sec. 4.1 "Training", Sec. 4.3) ------------------------------------------------
 namespace {
 struct TrainWs {
-  size_t status, cu, last_idx, tok_pos, tok_slot, rope_tab, x, h, h_lo, qkv, qkv32, kv_lo, attn, gu, act, attn_sched, total;
+  size_t status, cu, last_idx, tok_pos, tok_slot, rope_tab, x, h, h_lo, qkv, qkv32, kv_lo, attn, attn_lo, gu, act, act_lo, attn_sched, total;
 };
 TrainWs train_ws_layout(const kvp_handle* h, int64_t Bm, int64_t Tm) {
   TrainWs w;
@@ -1053,8 +1053,10 @@ TrainWs train_ws_layout(const kvp_handle* h, int64_t Bm, int64_t Tm) {
   w.qkv32 = take(Tm * B.max_nqkv * 4);
   w.kv_lo = take(Tm * 2 * (size_t)B.max_dkv * es);
   w.attn = take(Tm * B.max_dq * es);
+  w.attn_lo = take(Tm * B.max_dq * es);
   w.gu = take(Tm * 2 * (size_t)B.max_ffn * es);
   w.act = take(Tm * (size_t)B.max_ffn * es);
+  w.act_lo = take(Tm * (size_t)B.max_ffn * es);
   w.attn_sched = take((size_t)(Tm / 128 + Bm + 1) * 8);
   w.total = off;
   return w;
@@ -1103,6 +1105,14 @@ extern "C" kvp_status kvp_train_forward(kvp_handle* h, const int32_t* tokens, co
   char* act = ws + w.act;
   int2* attn_sched = (int2*)(ws + w.attn_sched);
   cudaError_t tc_err = cudaSuccess;
+  // This forward feeds activations to four projections per layer at EVERY position and its attention reads the whole
+  // predicted cache, so bf16's 8 significant bits at those points would dominate the logits error.  Where the tensor-core
+  // kernels take the shapes, every projection operand travels as a bf16 value plus its bf16 remainder (two MMA passes),
+  // q / k / v reach the attention as IEEE halves (the cache's own format: predicted entries are copied, not re-rounded).
+  bool hp = split && (B.L[0].hd == 64 || B.L[0].hd == 128) && B.d % 8 == 0 && B.vocab % 4 == 0;
+  for (int i = 0; i < B.n_layers && hp; ++i) hp = B.L[i].ffn % 64 == 0 && B.L[i].G == 64;
+  char* attn_lo = hp ? ws + w.attn_lo : nullptr;
+  char* act_lo = hp ? ws + w.act_lo : nullptr;
   // token -> (sequence position, cache slot); seq_lens is rewritten with the same lengths the cache already holds
   launch_build_index(ctx, cs.cu.data(), batch, T, cu_dev, tok_pos, tok_slot, (int*)(ws + w.last_idx), cache->block_table,
                      cache->max_pages_per_seq, cache->n_pages, cache->seq_lens);
@@ -1128,13 +1138,15 @@ extern "C" kvp_status kvp_train_forward(kvp_handle* h, const int32_t* tokens, co
       const float* qn = B.qk_norm ? (const float*)(P + L.q_norm) : nullptr;
       const float* kn = B.qk_norm ? (const float*)(P + L.k_norm) : nullptr;
       TcGemm tq{};
-      tq.A = (const bf16*)hbuf; tq.lda = B.d; tq.A2 = (const bf16*)h_lo; tq.lda2 = B.d; tq.split_begin = L.dq - col_begin;
+      tq.A = (const bf16*)hbuf; tq.lda = B.d; tq.A2 = (const bf16*)h_lo; tq.lda2 = B.d; tq.split_begin = hp ? 0 : L.dq - col_begin;
       tq.W = (const bf16*)(P + L.wqkv + (size_t)col_begin * B.d * es); tq.ldw = B.d; tq.M = T; tq.N = n_out; tq.K = B.d;
       tq.epi = TC_QKV; tq.C = (bf16*)(qkv + (size_t)col_begin * es); tq.ldc = L.nqkv;
       tq.C_lo = (bf16*)kv_lo; tq.ld_lo = 2 * L.dkv; tq.lo_col_begin = q_heads * L.hd;
       tq.rot_cols = (q_heads + L.nkv) * L.hd; tq.hd = L.hd; tq.rope_tab = rope_tab; tq.tok_pos = tok_pos;
       tq.q_gain = qn; tq.k_gain = kn; tq.q_cols = q_heads * L.hd; tq.eps = B.eps;
+      if (hp) { tq.c_is_half = 1; tq.C_lo = nullptr; }
       if (!try_tc(h, ctx, tq, KVP_CLASS_OTHER, &tc_err)) {
+        if (hp) return fail(h, KVP_ERR_CUDA, "internal: the tensor-core kernel refused a projection of the training-time forward");
         GemmArgs g{};
         g.A = hbuf; g.lda = B.d; g.M = T; g.K = B.d; g.A2 = h_lo; g.lda2 = B.d; g.split_begin = L.dq - col_begin;
         g.W = P + L.wqkv + (size_t)col_begin * B.d * es; g.ldw = B.d; g.N = n_out; g.C = qkv32; g.ldc = g.N;
@@ -1144,31 +1156,36 @@ extern "C" kvp_status kvp_train_forward(kvp_handle* h, const int32_t* tokens, co
       }
       if (pass == 0) {
         launch_kv_l1(ctx, qkv, L.nqkv, L.dq, kv_lo, 2 * L.dkv, T, L.nkv, L.hd, tok_slot, cache->k_pools[i], cache->v_pools[i],
-                     l1_k + i, l1_v + i);
+                     l1_k + i, l1_v + i, hp);
         if (last) break;
       } else {
-        launch_kv_take(ctx, qkv, L.nqkv, L.dq, T, L.nkv, L.hd, tok_slot, cache->k_pools[i], cache->v_pools[i]);
+        launch_kv_take(ctx, qkv, L.nqkv, L.dq, T, L.nkv, L.hd, tok_slot, cache->k_pools[i], cache->v_pools[i], hp);
       }
       if (split && attn_items <= 65535 && attn_tc_supported(L.hd, L.nqkv, qkv, L.dq, attn)) {
         cudaError_t e = launch_attn_tc((const bf16*)qkv, L.nqkv, T, L.nq, L.nkv, L.hd, cu_dev, attn_sched, attn_items, attn_tiles,
-                                       (bf16*)attn, L.dq, ctx.status, ctx.st, ctx.n_launch);
+                                       (bf16*)attn, L.dq, ctx.status, ctx.st, ctx.n_launch, hp, (bf16*)attn_lo);
         if (e != cudaSuccess && tc_err == cudaSuccess) tc_err = e;
       } else {
+        if (hp) return fail(h, KVP_ERR_CUDA, "internal: the tensor-core attention refused the training-time forward");
         launch_attn_prefill_simt(ctx, qkv, L.nqkv, L.nq, L.nkv, L.hd, cu_dev, batch, T, attn, L.dq);
       }
       TcGemm to{};
       to.A = (const bf16*)attn; to.lda = L.dq; to.W = (const bf16*)(P + L.wo); to.ldw = L.dq; to.M = T; to.N = B.d; to.K = L.dq;
       to.epi = TC_RESID; to.X = x; to.ldx = B.d;
+      if (hp) { to.A2 = (const bf16*)attn_lo; to.lda2 = L.dq; to.split_begin = 0; }
       if (!try_tc(h, ctx, to, KVP_CLASS_OTHER, &tc_err)) {
+        if (hp) return fail(h, KVP_ERR_CUDA, "internal: the tensor-core kernel refused a projection of the training-time forward");
         GemmArgs o{};
         o.A = attn; o.lda = L.dq; o.W = P + L.wo; o.ldw = L.dq; o.M = T; o.N = B.d; o.K = L.dq; o.X = x; o.ldx = B.d;
         launch_gemm_simt(ctx, o, EPI_RESID);
       }
-      launch_rmsnorm(ctx, x, (const float*)(P + L.ffn_norm), B.eps, T, B.d, hbuf, h->opt.dtype);
+      launch_rmsnorm(ctx, x, (const float*)(P + L.ffn_norm), B.eps, T, B.d, hbuf, h->opt.dtype, hp ? h_lo : nullptr);
       TcGemm tf{};
       tf.A = (const bf16*)hbuf; tf.lda = B.d; tf.W = (const bf16*)(P + L.wgu); tf.ldw = B.d; tf.M = T; tf.N = 2 * L.ffn; tf.K = B.d;
       tf.epi = TC_SWIGLU; tf.C = (bf16*)act; tf.ldc = L.ffn; tf.ffn = L.G == 64 ? L.ffn : 1;
+      if (hp) { tf.A2 = (const bf16*)h_lo; tf.lda2 = B.d; tf.split_begin = 0; tf.C_lo = (bf16*)act_lo; tf.ld_lo = L.ffn; }
       if (!try_tc(h, ctx, tf, KVP_CLASS_OTHER, &tc_err)) {
+        if (hp) return fail(h, KVP_ERR_CUDA, "internal: the tensor-core kernel refused a projection of the training-time forward");
         GemmArgs f{};
         f.A = hbuf; f.lda = B.d; f.W = P + L.wgu; f.ldw = B.d; f.M = T; f.N = 2 * L.ffn; f.K = B.d; f.C = gu; f.ldc = 2 * L.ffn;
         launch_gemm_simt(ctx, f, EPI_STORE);
@@ -1177,7 +1194,9 @@ extern "C" kvp_status kvp_train_forward(kvp_handle* h, const int32_t* tokens, co
       TcGemm td{};
       td.A = (const bf16*)act; td.lda = L.ffn; td.W = (const bf16*)(P + L.wd); td.ldw = L.ffn; td.M = T; td.N = B.d; td.K = L.ffn;
       td.epi = TC_RESID; td.X = x; td.ldx = B.d;
+      if (hp) { td.A2 = (const bf16*)act_lo; td.lda2 = L.ffn; td.split_begin = 0; }
       if (!try_tc(h, ctx, td, KVP_CLASS_OTHER, &tc_err)) {
+        if (hp) return fail(h, KVP_ERR_CUDA, "internal: the tensor-core kernel refused a projection of the training-time forward");
         GemmArgs d{};
         d.A = act; d.lda = L.ffn; d.W = P + L.wd; d.ldw = L.ffn; d.M = T; d.N = B.d; d.K = L.ffn; d.X = x; d.ldx = B.d;
         launch_gemm_simt(ctx, d, EPI_RESID);
@@ -1185,11 +1204,12 @@ extern "C" kvp_status kvp_train_forward(kvp_handle* h, const int32_t* tokens, co
     }
   }
   if (logits_out) {      // logits of every position: final norm, LM head (accumulated onto zeros by the residual epilogue)
-    launch_rmsnorm(ctx, x, (const float*)(P + B.final_norm), B.eps, T, B.d, hbuf, h->opt.dtype);
+    launch_rmsnorm(ctx, x, (const float*)(P + B.final_norm), B.eps, T, B.d, hbuf, h->opt.dtype, hp ? h_lo : nullptr);
     cudaMemsetAsync(logits_out, 0, (size_t)T * B.vocab * 4, s);
     TcGemm tl{};
     tl.A = (const bf16*)hbuf; tl.lda = B.d; tl.W = (const bf16*)(P + B.lm_head); tl.ldw = B.d; tl.M = T; tl.N = B.vocab; tl.K = B.d;
     tl.epi = TC_RESID; tl.X = logits_out; tl.ldx = B.vocab;
+    if (hp) { tl.A2 = (const bf16*)h_lo; tl.lda2 = B.d; tl.split_begin = 0; }
     if (!try_tc(h, ctx, tl, KVP_CLASS_OTHER, &tc_err)) {
       GemmArgs g{};
       g.A = hbuf; g.lda = B.d; g.W = P + B.lm_head; g.ldw = B.d; g.M = T; g.N = B.vocab; g.K = B.d; g.X = logits_out; g.ldx = B.vocab;

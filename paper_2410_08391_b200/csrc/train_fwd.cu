@@ -15,8 +15,8 @@ __device__ __forceinline__ size_t cache_off(int slot, int c, int nkv, int hd) {
 
 // sums[0] += inv_n * sum |K_hat - K_B|, sums[1] += inv_n * sum |V_hat - V_B| over all tokens and columns.
 // The layer's own keys and values are read as hi (+ lo, bf16 mode) parts.
-template <class T>
-__global__ void __launch_bounds__(256) kv_l1_kernel(const T* __restrict__ qkv, int ld, int k_col, const bf16* __restrict__ kv_lo,
+template <class T, class QT>
+__global__ void __launch_bounds__(256) kv_l1_kernel(const QT* __restrict__ qkv, int ld, int k_col, const bf16* __restrict__ kv_lo,
                                                     int ld_lo, int T_tokens, int nkv, int hd, const int* __restrict__ tok_slot,
                                                     const typename KvOf<T>::type* __restrict__ kpool,
                                                     const typename KvOf<T>::type* __restrict__ vpool, float inv_n,
@@ -47,8 +47,8 @@ __global__ void __launch_bounds__(256) kv_l1_kernel(const T* __restrict__ qkv, i
 }
 
 // The layer's key and value columns of the projection buffer take the predicted cache's entries.
-template <class T>
-__global__ void __launch_bounds__(256) kv_take_kernel(T* __restrict__ qkv, int ld, int k_col, int T_tokens, int nkv, int hd,
+template <class T, class QT>
+__global__ void __launch_bounds__(256) kv_take_kernel(QT* __restrict__ qkv, int ld, int k_col, int T_tokens, int nkv, int hd,
                                                       const int* __restrict__ tok_slot,
                                                       const typename KvOf<T>::type* __restrict__ kpool,
                                                       const typename KvOf<T>::type* __restrict__ vpool) {
@@ -59,8 +59,8 @@ __global__ void __launch_bounds__(256) kv_take_kernel(T* __restrict__ qkv, int l
     const int slot = tok_slot[t];
     if (slot < 0) continue;
     const size_t off = cache_off(slot, c, nkv, hd);
-    qkv[(size_t)t * ld + k_col + c] = from_f<T>(to_f(kpool[off]));
-    qkv[(size_t)t * ld + k_col + dkv + c] = from_f<T>(to_f(vpool[off]));
+    qkv[(size_t)t * ld + k_col + c] = from_f<QT>(to_f(kpool[off]));          // exact when QT is the cache's own type
+    qkv[(size_t)t * ld + k_col + dkv + c] = from_f<QT>(to_f(vpool[off]));
   }
 }
 
@@ -69,28 +69,34 @@ int grid_of(size_t n) { size_t g = (n + 255) / 256; return (int)(g < 1 ? 1 : (g 
 }  // namespace
 
 void launch_kv_l1(const LaunchCtx& ctx, const void* qkv, int ld, int k_col, const void* kv_lo, int ld_lo, int T_tokens, int nkv,
-                  int hd, const int* tok_slot, const void* kpool, const void* vpool, float* sum_k, float* sum_v) {
+                  int hd, const int* tok_slot, const void* kpool, const void* vpool, float* sum_k, float* sum_v, bool qkv_is_half) {
   const size_t n = (size_t)T_tokens * nkv * hd;
   if (n == 0) return;
   const float inv_n = 1.f / (float)n;
   ++*ctx.n_launch;
   if (ctx.dtype == 0)
-    kv_l1_kernel<float><<<grid_of(n), 256, 0, ctx.st>>>((const float*)qkv, ld, k_col, nullptr, 0, T_tokens, nkv, hd, tok_slot,
+    kv_l1_kernel<float, float><<<grid_of(n), 256, 0, ctx.st>>>((const float*)qkv, ld, k_col, nullptr, 0, T_tokens, nkv, hd, tok_slot,
                                                        (const float*)kpool, (const float*)vpool, inv_n, sum_k, sum_v);
+  else if (qkv_is_half)
+    kv_l1_kernel<bf16, kv16><<<grid_of(n), 256, 0, ctx.st>>>((const kv16*)qkv, ld, k_col, nullptr, 0, T_tokens, nkv, hd,
+                                                            tok_slot, (const kv16*)kpool, (const kv16*)vpool, inv_n, sum_k, sum_v);
   else
-    kv_l1_kernel<bf16><<<grid_of(n), 256, 0, ctx.st>>>((const bf16*)qkv, ld, k_col, (const bf16*)kv_lo, ld_lo, T_tokens, nkv, hd,
-                                                      tok_slot, (const kv16*)kpool, (const kv16*)vpool, inv_n, sum_k, sum_v);
+    kv_l1_kernel<bf16, bf16><<<grid_of(n), 256, 0, ctx.st>>>((const bf16*)qkv, ld, k_col, (const bf16*)kv_lo, ld_lo, T_tokens, nkv, hd,
+                                                            tok_slot, (const kv16*)kpool, (const kv16*)vpool, inv_n, sum_k, sum_v);
 }
 
 void launch_kv_take(const LaunchCtx& ctx, void* qkv, int ld, int k_col, int T_tokens, int nkv, int hd, const int* tok_slot,
-                    const void* kpool, const void* vpool) {
+                    const void* kpool, const void* vpool, bool qkv_is_half) {
   const size_t n = (size_t)T_tokens * nkv * hd;
   if (n == 0) return;
   ++*ctx.n_launch;
   if (ctx.dtype == 0)
-    kv_take_kernel<float><<<grid_of(n), 256, 0, ctx.st>>>((float*)qkv, ld, k_col, T_tokens, nkv, hd, tok_slot, (const float*)kpool,
+    kv_take_kernel<float, float><<<grid_of(n), 256, 0, ctx.st>>>((float*)qkv, ld, k_col, T_tokens, nkv, hd, tok_slot, (const float*)kpool,
                                                          (const float*)vpool);
+  else if (qkv_is_half)
+    kv_take_kernel<bf16, kv16><<<grid_of(n), 256, 0, ctx.st>>>((kv16*)qkv, ld, k_col, T_tokens, nkv, hd, tok_slot, (const kv16*)kpool,
+                                                              (const kv16*)vpool);
   else
-    kv_take_kernel<bf16><<<grid_of(n), 256, 0, ctx.st>>>((bf16*)qkv, ld, k_col, T_tokens, nkv, hd, tok_slot, (const kv16*)kpool,
-                                                        (const kv16*)vpool);
+    kv_take_kernel<bf16, bf16><<<grid_of(n), 256, 0, ctx.st>>>((bf16*)qkv, ld, k_col, T_tokens, nkv, hd, tok_slot, (const kv16*)kpool,
+                                                              (const kv16*)vpool);
 }

@@ -236,7 +236,7 @@ def test_train_forward_matches_oracle(name, lens, regime):
             assert rel_fro(got, ref_logits) <= tol, f"seq {b}: logits {rel_fro(got, ref_logits):.3e}"
             # the last row is the inference path's first step (also checked there); every row must hold on its own
             worst = max(rel_fro(got[t], ref_logits[t]) for t in range(lens[b]))
-            assert worst <= 2 * tol, f"seq {b}: worst row {worst:.3e}"
+            assert worst <= tol, f"seq {b}: worst row {worst:.3e}"
             t0 += lens[b]
         # the predicted cache is rounded to the run dtype before it is compared: one bf16 rounding of O(1) entries
         slack = 4e-3 if pair.dtype == "bf16" else 1e-5
@@ -459,12 +459,12 @@ def test_train_forward_config_2_sampled_rows_match_oracle():
         n = 192
         ref_logits, _, _, _ = orc.train_forward(pair, W, pr.seq(0)[:n])
         got = logits[:n].cpu().numpy()
-        # Unlike the inference path's single step (fp32 activations), this forward feeds bf16 activations to four
-        # projections in each of 28 layers at every position: rounding the stored tensors alone moves the oracle's
-        # own logits by 1.85e-2 here (worst row 2.3e-2; oracle/train_forward_rounding_floor.py c2 192).  The bound
-        # is that floor plus the 1e-2 allowed everywhere else.
-        assert rel_fro(got, ref_logits) <= 1.85e-2 + TOL[pair.dtype]
-        assert max(rel_fro(got[t], ref_logits[t]) for t in range(n)) <= 2.3e-2 + 2 * TOL[pair.dtype]
+        # every projection operand of this forward travels as a bf16 value plus its bf16 remainder and the attention takes
+        # IEEE halves, so the ordinary tolerance holds for the whole block of rows and for every row on its own
+        e_all = rel_fro(got, ref_logits)
+        e_row = max(rel_fro(got[t], ref_logits[t]) for t in range(n))
+        print(f"c2 training-time forward, first {n} rows: logits err {e_all:.2e}, worst row {e_row:.2e}")
+        assert e_all <= TOL[pair.dtype] and e_row <= TOL[pair.dtype]
         assert bool((l1_k > 0).all()) and bool((l1_v > 0).all())
     finally:
         s.close()
