@@ -95,15 +95,16 @@ typedef struct {
   int32_t flags;          /* 0, or a sum of KVP_OPT_* (kernel variants; results are the same within rounding) */
 } kvp_options;
 
-/* Kernel variants that are built and tested but are not the default schedule because they measured slower on the
- * benchmark configurations (numbers in the design notes):
+/* Schedule variants (results are the same within rounding; the design notes give the measurements):
  *   KVP_OPT_FUSED_KV_PRED  the K/V projection of an auxiliary layer and the KV predictor as ONE kernel (the predictor
  *                          is the projection's epilogue; K_A / V_A reach it through shared memory), used for calls
- *                          with at least one 128-token block per SM;
- *   KVP_OPT_FUSED_NORM     RMSNorm folded into the GEMMs around it (the residual GEMM that completes x also writes
- *                          bf16(x * gain) and the rows' sums of squares, the next GEMM scales its rows by 1 / rms),
- *                          used where every output tile of the residual GEMMs belongs to one CTA. */
-enum { KVP_OPT_FUSED_KV_PRED = 1, KVP_OPT_FUSED_NORM = 2 };
+ *                          with at least one 128-token block per SM.  Off by default: it measured slower than the
+ *                          projection GEMM followed by a predictor GEMM.
+ *   KVP_OPT_SEPARATE_NORM  RMSNorm as a kernel of its own in front of every projection.  By default, wherever every
+ *                          output tile of the residual GEMMs belongs to one CTA (calls of some thousand tokens and
+ *                          more), RMSNorm is folded into the GEMMs around it: the residual GEMM that completes x also
+ *                          writes bf16(x * gain) and the rows' sums of squares, the next GEMM scales its rows by 1 / rms. */
+enum { KVP_OPT_FUSED_KV_PRED = 1, KVP_OPT_SEPARATE_NORM = 2 };
 
 /* A named tensor handed to kvp_load_weights().  Names:
  *   "aux.embed" [vocab, d_A]

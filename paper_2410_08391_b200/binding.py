@@ -132,7 +132,7 @@ def kvp_layer_map_uniform(n_base: int, n_aux: int) -> List[int]:
     return list(out)[:n_base]
 
 
-KVP_OPT_FUSED_KV_PRED, KVP_OPT_FUSED_NORM = 1, 2
+KVP_OPT_FUSED_KV_PRED, KVP_OPT_SEPARATE_NORM = 1, 2
 
 
 def kvp_create(aux, base, layer_map: Sequence[int], dtype: str = "bf16", predictor_bias: bool = False,

@@ -186,6 +186,13 @@ void launch_step_append(const LaunchCtx&, const float* qkv, int nq, int nkv, int
 void launch_argmax(const LaunchCtx&, const float* logits, int batch, int vocab, int* out);
 void launch_add_int(const LaunchCtx&, int* v, int n, int delta);
 int step_attn_splits(int batch, int nkv, int max_keys);
+// warp-level tensor-core variant for the half-precision cache (pages fetched through a swizzling tensor map)
+int step_attn_mma_splits(int batch, int nkv, int max_keys, int upper);
+bool step_attn_mma_supported(int dtype, int nq, int nkv, int hd, const void* kpool, const void* vpool, int n_pages);
+cudaError_t launch_step_attn_mma(const LaunchCtx&, const float* q, int ldq, int nq, int nkv, int hd, float theta, const void* kpool,
+                                 const void* vpool, const int* block_table, int max_pages_per_seq, int n_pages, const int* seq_lens,
+                                 int extra, int batch, int n_split, int max_keys, float* part, float* out, const float* q_gain,
+                                 float eps, int* split_done);
 // bandwidth-bound variant for the bf16 cache (pages fetched with bulk asynchronous copies)
 int step_attn_ring_splits(int nq, int nkv, int hd, int batch, int max_keys, int upper);
 bool step_attn_ring_supported(int dtype, int nq, int nkv, int hd, const void* kpool, const void* vpool);

@@ -30,18 +30,23 @@ using namespace tcp;
 constexpr int BM = 128, BK = 64;
 constexpr int GROUP_M = 16;                                // row blocks per rasterisation group
 constexpr int N_THREADS = 224;                             // warps: 0 A loads, 1 MMA, 2 W loads, 3-6 epilogue
-template <int BN> struct Tile {
-  static constexpr int STAGES = BN == 256 ? 4 : 6;
+constexpr int N_THREADS_NORM = 352;                        // fused-norm residual kernel: 8 epilogue warps (3-10), two per lane quarter
+constexpr int TC_RESID_NORM = 100;                         // internal: TC_RESID with the folded RMSNorm producer (own shared-memory plan)
+template <int BN, int EPI = TC_STORE> struct Tile {
+  // the fused-norm residual epilogue needs a deeper prefetch ring for the old values of X: one operand stage less
+  static constexpr int STAGES = (BN == 256 ? 4 : 6) - (EPI == TC_RESID_NORM ? 1 : 0);
+  static constexpr int XS = 2;                              // 4 KiB slots per epilogue warp
+  static constexpr int EPI_WARPS = EPI == TC_RESID_NORM ? 8 : 4;
+  static constexpr int THREADS = EPI == TC_RESID_NORM ? N_THREADS_NORM : N_THREADS;
+  static constexpr int XRING = (EPI == TC_RESID || EPI == TC_RESID_NORM) ? EPI_WARPS * XS * 4096 : 0;
   static constexpr int A_BYTES = BM * BK * 2, W_BYTES = BN * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + W_BYTES;    // 48 KiB / 32 KiB
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + XRING + 1024 /*align*/ + 512 /*barriers*/;
 };
 // Fused-norm residual epilogue: each epilogue warp prefetches the residual stream's old values of its 32 rows,
 // 32 columns at a time, into a private ring of XS slots (TMA, 128-byte swizzle) while the main loop of the next
 // tile runs, so the read-modify-write of X never waits on memory.
-constexpr int XS = 2;
 constexpr int X_SLOT_BYTES = 32 * 32 * 4;
-constexpr int XRING_BYTES = 4 * XS * X_SLOT_BYTES;       // 32 KiB
 __device__ __forceinline__ uint4 pack8(const float* v) {
   __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
   __nv_bfloat162 c = __floats2bfloat162_rn(v[4], v[5]), d = __floats2bfloat162_rn(v[6], v[7]);
@@ -163,26 +168,6 @@ struct Sched {
 
 __device__ __forceinline__ void red_add4(float* dst, float a, float b, float c, float d) {
   asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
-}
-
-// Fused-norm producer, 32 final values of X (row m, columns n ..): operand of the next GEMM and sum of squares.
-__device__ __forceinline__ float norm_out32(const Params& p, int m, int n, int n_valid, float* v) {
-  float ss = 0.f;
-#pragma unroll
-  for (int i = 0; i < 32; ++i) {
-    const bool in = i < n_valid;
-    ss = fmaf(in ? v[i] : 0.f, v[i], ss);
-    v[i] = in ? v[i] * p.gain_next[n + i] : 0.f;
-  }
-  bf16* h = p.H + (size_t)m * p.ldh + n;
-  store32_bf16(h, v, n_valid);
-  if (p.H_lo) {
-    bf16* lo = p.H_lo + (size_t)m * p.ldh + n;
-#pragma unroll
-    for (int g = 0; g < 4; ++g)
-      if (g * 8 < n_valid) *reinterpret_cast<uint4*>(lo + g * 8) = pack8_lo(v + g * 8);
-  }
-  return ss;
 }
 
 // ---- epilogues: one thread owns one output row of the tile ---------------------------------
@@ -329,17 +314,18 @@ __device__ __forceinline__ void epilogue_tile(const Params& p, uint32_t tmem_acc
 }
 
 template <int EPI, int BN>
-__global__ void __launch_bounds__(N_THREADS, 1)
+__global__ void __launch_bounds__((Tile<BN, EPI>::THREADS), 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_a2,
                const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, const Params p) {
-  using T = Tile<BN>;
-  constexpr int STAGES = T::STAGES, STAGE_BYTES = T::STAGE_BYTES;
+  using T = Tile<BN, EPI>;
+  constexpr int STAGES = T::STAGES, STAGE_BYTES = T::STAGE_BYTES, XS = T::XS;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  constexpr int XR = EPI == TC_RESID ? XRING_BYTES : 0;
+  constexpr int XR = T::XRING;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES + XR);
-  // bars: full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], x_full[4][XS]; then tmem base, abort flag
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4 + 4 * XS);
+  // bars: full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], x_full[epilogue warps][XS]; then tmem base, abort flag
+  constexpr int EW = T::EPI_WARPS;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4 + EW * XS);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const uint32_t smem_base = smem_u32(smem);
   const uint32_t bar_base = smem_u32(bars);
@@ -359,8 +345,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 2); mbar_init(empty_bar(s), 1); }   // two loaders per stage
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
-    for (int q = 0; q < 4; ++q) for (int x = 0; x < XS; ++x) mbar_init(xfull_bar(q, x), 1);
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), EW); }
+    for (int q = 0; q < EW; ++q) for (int x = 0; x < XS; ++x) mbar_init(xfull_bar(q, x), 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -435,28 +421,33 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
   } else {
     // ---------------- epilogue: 4 warps, each owns the 32 tensor-memory lanes of its quarter ----------------
-    const int quarter = warp & 3;
+    const int quarter = warp & 3;                 // tensor-memory lanes this warp may read
+    const int ew = warp - 3;                      // epilogue warp index
+    constexpr int NH = EW / 4;                    // warps per lane quarter: each takes every NH-th block of 32 columns
+    const int half = ew >> 2;
     Sched<BN> sched(p);
     Work w;
     int acc = 0; uint32_t acc_phase = 0;
     bool ok = true;
     // fused norm (TC_RESID with H, every tile owned by one CTA): the old values of X arrive through this warp's ring
-    const bool fused = EPI == TC_RESID && p.H != nullptr;
-    const uint32_t xring = smem_base + STAGES * STAGE_BYTES + quarter * (XS * X_SLOT_BYTES);
+    constexpr bool fused = EPI == TC_RESID_NORM;
+    const uint32_t xring = smem_base + STAGES * STAGE_BYTES + ew * (XS * X_SLOT_BYTES);
     Sched<BN> pre(p);
     Work pw;
     bool pre_ok = fused && pre.next(pw);
-    int pre_c = 0;
+    int pre_c = half;
+    while (pre_ok && pw.n0 + pre_c * 32 >= p.N) { pre_ok = pre.next(pw); pre_c = half; }     // (a tile without a block for this warp)
     uint32_t x_issued = 0, x_used = 0;
-    auto prefetch_x = [&]() {      // next 32 x 32 block of X in (tile, column) order into the slot just freed
+    auto prefetch_x = [&]() {      // this warp's next 32 x 32 block of X in (tile, column) order into the slot just freed
       if (!pre_ok) return;
       const int slot = x_issued % XS;
       if (lane == 0) {
-        mbar_expect_tx(xfull_bar(quarter, slot), X_SLOT_BYTES);
-        tma_load_2d(xring + slot * X_SLOT_BYTES, &map_x, pw.n0 + pre_c * 32, pw.m0 + quarter * 32, xfull_bar(quarter, slot));
+        mbar_expect_tx(xfull_bar(ew, slot), X_SLOT_BYTES);
+        tma_load_2d(xring + slot * X_SLOT_BYTES, &map_x, pw.n0 + pre_c * 32, pw.m0 + quarter * 32, xfull_bar(ew, slot));
       }
       ++x_issued;
-      if (pw.n0 + (++pre_c) * 32 >= p.N || pre_c * 32 >= BN) { pre_ok = pre.next(pw); pre_c = 0; }
+      pre_c += NH;
+      while (pre_ok && (pw.n0 + pre_c * 32 >= p.N || pre_c * 32 >= BN)) { pre_ok = pre.next(pw); pre_c = half; }
     };
     if (fused) for (int i = 0; i < XS; ++i) prefetch_x();
     while (sched.next(w)) {
@@ -469,11 +460,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       if (fused) {
         float row_ss = 0.f;
 #pragma unroll 1
-        for (int c = 0; c < BN && ok; c += 32) {
+        for (int c = half * 32; c < BN && ok; c += 32 * NH) {
           const int n = w.n0 + c, n_valid = p.N - n;
           if (n_valid <= 0) break;
           const int slot = x_used % XS;
-          ok = mbar_wait(xfull_bar(quarter, slot), (x_used / XS) & 1u, abort_flag, p.status);
+          ok = mbar_wait(xfull_bar(ew, slot), (x_used / XS) & 1u, abort_flag, p.status);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           float v[32];
@@ -487,20 +478,77 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             if (g == 0) tmem_ld_wait();
             v[4 * g] += o.x; v[4 * g + 1] += o.y; v[4 * g + 2] += o.z; v[4 * g + 3] += o.w;
           }
+          // The new values leave through the slot: every thread owns a ROW here, and 16-byte stores of 32 different rows
+          // cost eight times the memory transactions of whole 128-byte lines.  Each thread puts its row back into the slot,
+          // then the warp reads the slot line by line and stores it coalesced; the operand rows (bf16 value, remainder) follow
+          // through the same 4 KiB.
+          const uint32_t sl = xring + slot * X_SLOT_BYTES;
+          const int row_base = w.m0 + quarter * 32;
           __syncwarp();
+#pragma unroll
+          for (int g = 0; g < 8; ++g)
+            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(xrow + ((g ^ (lane & 7)) << 4)), "f"(v[4 * g]), "f"(v[4 * g + 1]),
+                         "f"(v[4 * g + 2]), "f"(v[4 * g + 3]) : "memory");
+          __syncwarp();
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {            // 4 rows x 128 bytes per instruction
+            const int r = 4 * i + (lane >> 3), j = lane & 7;
+            float4 o;
+            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(o.x), "=f"(o.y), "=f"(o.z), "=f"(o.w)
+                         : "r"(sl + r * 128 + ((j ^ (r & 7)) << 4)));
+            if (row_base + r < p.M && n + 4 * j < p.N) *reinterpret_cast<float4*>(p.X + (size_t)(row_base + r) * p.ldx + n + 4 * j) = o;
+          }
+          // operand of the next GEMM and the row's sum of squares
+          float ssq = 0.f;
+          if (n_valid >= 32) {
+#pragma unroll
+            for (int g = 0; g < 8; ++g) {
+              const float4 gn = __ldg(reinterpret_cast<const float4*>(p.gain_next + n) + g);
+              ssq = fmaf(v[4 * g], v[4 * g], ssq); ssq = fmaf(v[4 * g + 1], v[4 * g + 1], ssq);
+              ssq = fmaf(v[4 * g + 2], v[4 * g + 2], ssq); ssq = fmaf(v[4 * g + 3], v[4 * g + 3], ssq);
+              v[4 * g] *= gn.x; v[4 * g + 1] *= gn.y; v[4 * g + 2] *= gn.z; v[4 * g + 3] *= gn.w;
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const bool in = i < n_valid;
+              ssq = fmaf(in ? v[i] : 0.f, v[i], ssq);
+              v[i] = in ? v[i] * p.gain_next[n + i] : 0.f;
+            }
+          }
+          row_ss += ssq;
+          __syncwarp();                            // the slot has been read back by every lane
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            const uint4 hi = pack8(v + g * 8);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sl + lane * 64 + g * 16), "r"(hi.x), "r"(hi.y), "r"(hi.z), "r"(hi.w) : "memory");
+            if (p.H_lo) {
+              const uint4 lo = pack8_lo(v + g * 8);
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sl + 2048 + lane * 64 + g * 16), "r"(lo.x), "r"(lo.y), "r"(lo.z), "r"(lo.w) : "memory");
+            }
+          }
+          __syncwarp();
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {            // 8 rows x 64 bytes per instruction
+            const int r = 8 * i + (lane >> 2), c = lane & 3;
+            if (row_base + r < p.M && n + 8 * c < p.N) {
+              uint4 u;
+              asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(u.x), "=r"(u.y), "=r"(u.z), "=r"(u.w) : "r"(sl + r * 64 + c * 16));
+              *reinterpret_cast<uint4*>(p.H + (size_t)(row_base + r) * p.ldh + n + 8 * c) = u;
+              if (p.H_lo) {
+                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(u.x), "=r"(u.y), "=r"(u.z), "=r"(u.w) : "r"(sl + 2048 + r * 64 + c * 16));
+                *reinterpret_cast<uint4*>(p.H_lo + (size_t)(row_base + r) * p.ldh + n + 8 * c) = u;
+              }
+            }
+          }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // this warp's own writes to the slot come before the copy engine's
+          __syncwarp();                            // the slot is free: the next block of X may land in it
           ++x_used;
           prefetch_x();
-          if (m < p.M) {
-            float* x = p.X + (size_t)m * p.ldx + n;
-#pragma unroll
-            for (int g = 0; g < 8; ++g)
-              if (g * 4 < n_valid) *reinterpret_cast<float4*>(x + 4 * g) = make_float4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
-            row_ss += norm_out32(p, m, n, n_valid, v);
-          }
         }
         if (!ok) break;
         if (m < p.M) atomicAdd(p.ss_out + m, row_ss);
-      } else if (EPI == TC_RESID) {
+      } else if (EPI == TC_RESID || EPI == TC_RESID_NORM) {
         // X += acc through the copy engine: a 32 x 32 block of the accumulator goes into one of this warp's slots
         // (swizzled like a tensor tile) and leaves as ONE reduce-add of whole 128-byte rows, instead of 256 separate
         // 16-byte atomics.  Rows and columns beyond the matrix are clipped by the tensor map.
@@ -538,7 +586,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       if (lane == 0) mbar_arrive(tempty_bar(acc));
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
-    if (EPI == TC_RESID && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");    // this warp's reduces have completed
+    if ((EPI == TC_RESID || EPI == TC_RESID_NORM) && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");    // this warp's reduces have completed
   }
   tc_fence_before();
   __syncthreads();
@@ -556,18 +604,18 @@ bool make_map(CUtensorMap* m, const void* base, int rows, int cols, int ld, int 
 
 template <int EPI, int BN>
 cudaError_t go(const CUtensorMap& a, const CUtensorMap& a2, const CUtensorMap& w, const CUtensorMap& x, const Params& p, int grid, cudaStream_t st) {
-  constexpr int SMEM = Tile<BN>::SMEM_BYTES + (EPI == TC_RESID ? XRING_BYTES : 0);
+  constexpr int SMEM = Tile<BN, EPI>::SMEM_BYTES;
   static bool raised[TC_MAX_DEVICES] = {};
   cudaError_t e = tc_raise_smem_limit(gemm_tc_kernel<EPI, BN>, SMEM, raised);
   if (e != cudaSuccess) return e;
-  return launch_overlapped(gemm_tc_kernel<EPI, BN>, dim3(grid), dim3(N_THREADS), SMEM, st, a, a2, w, x, p);
+  return launch_overlapped(gemm_tc_kernel<EPI, BN>, dim3(grid), dim3(Tile<BN, EPI>::THREADS), SMEM, st, a, a2, w, x, p);
 }
 
 template <int BN>
 cudaError_t go_epi(int epi, const CUtensorMap& a, const CUtensorMap& a2, const CUtensorMap& w, const CUtensorMap& x, const Params& p, int grid, cudaStream_t st) {
   switch (epi) {
     case TC_STORE: return go<TC_STORE, BN>(a, a2, w, x, p, grid, st);
-    case TC_RESID: return go<TC_RESID, BN>(a, a2, w, x, p, grid, st);
+    case TC_RESID: return p.H ? go<TC_RESID_NORM, BN>(a, a2, w, x, p, grid, st) : go<TC_RESID, BN>(a, a2, w, x, p, grid, st);
     case TC_SWIGLU: return go<TC_SWIGLU, BN>(a, a2, w, x, p, grid, st);
     case TC_QKV: return go<TC_QKV, BN>(a, a2, w, x, p, grid, st);
     default: return go<TC_PAGED, BN>(a, a2, w, x, p, grid, st);

@@ -392,7 +392,7 @@ kvp_status kvp_create(const kvp_model_cfg* aux, const kvp_model_cfg* base, const
   if (!aux || !base || !layer_map || !opt) return KVP_ERR_INVALID_ARG;
   if (validate_model(aux) || validate_model(base)) return KVP_ERR_SHAPE;
   if (opt->dtype != KVP_F32 && opt->dtype != KVP_BF16) return KVP_ERR_INVALID_ARG;
-  if (opt->page_tokens != PAGE_TOKENS || (opt->flags & ~(KVP_OPT_FUSED_KV_PRED | KVP_OPT_FUSED_NORM)) != 0) return KVP_ERR_INVALID_ARG;
+  if (opt->page_tokens != PAGE_TOKENS || (opt->flags & ~(KVP_OPT_FUSED_KV_PRED | KVP_OPT_SEPARATE_NORM)) != 0) return KVP_ERR_INVALID_ARG;
   if (opt->predictor_bias != 0 && opt->predictor_bias != 1) return KVP_ERR_INVALID_ARG;
   if (aux->vocab != base->vocab) return KVP_ERR_SHAPE;   // one token stream feeds both models
   if (unsupported_model(aux) || unsupported_model(base)) return KVP_ERR_UNSUPPORTED;
@@ -607,7 +607,7 @@ static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int
   float* norm_ss = (float*)(ws + w.norm_ss);
   // (the producer needs every output tile to belong to one CTA: enough tiles for the SMs the GEMMs of this call get)
   const int sms_for_gemms = (h->side != nullptr && !h->timing && T <= 4096 && h->step_sms > 0) ? h->n_sm - h->step_sms : h->n_sm;
-  const bool can_fuse = (h->opt.flags & KVP_OPT_FUSED_NORM) != 0 && tc_gemm_resid_can_fuse(T, A.d, h->n_sm) &&
+  const bool can_fuse = (h->opt.flags & KVP_OPT_SEPARATE_NORM) == 0 && tc_gemm_resid_can_fuse(T, A.d, h->n_sm) &&
                         tc_gemm_resid_can_fuse(T, A.d, sms_for_gemms);
   if (can_fuse) cudaMemsetAsync(norm_ss, 0, (size_t)2 * A.n_layers * T * 4, s);
   auto shape_ok = [&](int K, int N) { return can_fuse && h->opt.dtype == KVP_BF16 && K % 8 == 0 && N % 8 == 0 && A.d % 8 == 0; };

@@ -606,6 +606,15 @@ void launch_step_attn(const LaunchCtx& ctx, const float* q, int ldq, int nq, int
   fill_inv_freq(&inv, hd, theta);
   int n_split = step_attn_splits(batch, nkv, max_keys);
   dim3 grid(n_split, nkv, batch);
+  if (split_done && step_attn_mma_supported(ctx.dtype, nq, nkv, hd, kpool, vpool, n_pages)) {
+    // half-precision cache, head_dim 64 / 128: warp-level tensor-core kernel (pages through a swizzling tensor map)
+    const int ns = step_attn_mma_splits(batch, nkv, max_keys, n_split);
+    if (ns > 1) cudaMemsetAsync(split_done, 0, (size_t)batch * nkv * sizeof(int), ctx.st);
+    if (launch_step_attn_mma(ctx, q, ldq, nq, nkv, hd, theta, kpool, vpool, block_table, mpps, n_pages, seq_lens, extra, batch, ns, max_keys, part, out,
+                             q_gain, eps, split_done) == cudaSuccess)
+      return;
+    cudaGetLastError();      // (a tensor map could not be made: the kernels below take plain pointers)
+  }
   if (step_attn_ring_supported(ctx.dtype, nq, nkv, hd, kpool, vpool)) {
     n_split = step_attn_ring_splits(nq, nkv, hd, batch, max_keys, n_split);
     // up to 4 heads per kv head: the CTA that finishes a group's last split merges it (counters cleared here)

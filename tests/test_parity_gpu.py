@@ -89,8 +89,9 @@ def test_prefill_predict_matches_oracle(name, lens, regime):
                                               ("t_scaled", [1500] * 13, "fanin")],
                          ids=lambda v: str(v).replace(" ", "")[:40])
 def test_kernel_variants_match_oracle(name, lens, regime, flags):
-    """The optional kernel variants (kvp_options.flags: K/V projection + predictor as one kernel; RMSNorm folded into
-    the GEMMs around it) on calls large enough for them to be taken: same results within the same tolerances."""
+    """The schedule variants (kvp_options.flags: K/V projection + predictor as one kernel; RMSNorm as its own kernel
+    instead of folded into the GEMMs around it) on calls large enough for the choice to matter (flags = 0, the default, is
+    what every other many-token case runs): same results within the same tolerances."""
     pair = wl.pair(name)
     W = wl.make_weights(pair, seed=1, regime=regime)
     pr = wl.custom_prompts(pair.base.vocab, lens, seed=1)
