@@ -35,10 +35,11 @@ constexpr int TC_RESID_NORM = 100;                         // internal: TC_RESID
 template <int BN, int EPI = TC_STORE> struct Tile {
   // the fused-norm residual epilogue needs a deeper prefetch ring for the old values of X: one operand stage less
   static constexpr int STAGES = (BN == 256 ? 4 : 6) - (EPI == TC_RESID_NORM ? 1 : 0);
-  static constexpr int XS = 2;                              // 4 KiB slots per epilogue warp
-  static constexpr int EPI_WARPS = EPI == TC_RESID_NORM ? 8 : 4;
-  static constexpr int THREADS = EPI == TC_RESID_NORM ? N_THREADS_NORM : N_THREADS;
-  static constexpr int XRING = (EPI == TC_RESID || EPI == TC_RESID_NORM) ? EPI_WARPS * XS * 4096 : 0;
+  static constexpr int XS = EPI == TC_PAGED ? 1 : 2;        // 4 KiB slots per epilogue warp
+  // epilogues that move every element through shared memory get eight warps (two per tensor-memory lane quarter)
+  static constexpr int EPI_WARPS = (EPI == TC_RESID_NORM || EPI == TC_PAGED) ? 8 : 4;
+  static constexpr int THREADS = EPI_WARPS == 8 ? N_THREADS_NORM : N_THREADS;
+  static constexpr int XRING = (EPI == TC_RESID || EPI == TC_RESID_NORM || EPI == TC_PAGED) ? EPI_WARPS * XS * 4096 : 0;
   static constexpr int A_BYTES = BM * BK * 2, W_BYTES = BN * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + W_BYTES;    // 48 KiB / 32 KiB
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + XRING + 1024 /*align*/ + 512 /*barriers*/;
@@ -577,6 +578,54 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             asm volatile("cp.async.bulk.commit_group;" ::: "memory");
           }
           ++x_used;
+        }
+      } else if (EPI == TC_PAGED) {
+        // Predicted columns into cache pages.  A thread owns a token ROW of the accumulator, but 16-byte stores of 32
+        // different rows cost four times the memory transactions of 64-byte row pieces: the 32 x 32 block goes through
+        // this warp's shared-memory slot as halves and leaves as 8 rows x 64 bytes per store instruction.
+        const PagedOut& q = p.paged;
+        const uint32_t sl = xring;
+        const int row_base = w.m0 + quarter * 32;
+        int slot4[4];              // cache slots of the four rows this lane writes in the read-back pattern
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int mr = row_base + 8 * i + (lane >> 2);
+          slot4[i] = mr < p.M ? q.tok_slot[mr] : -1;
+        }
+#pragma unroll 1
+        for (int c = half * 32; c < BN; c += 32 * NH) {
+          const int n = w.n0 + c;
+          if (n >= p.N) break;
+          float v[32];
+          tmem_ld32(tmem_acc + c, v);
+          tmem_ld_wait();
+          if (q.bias) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] += q.bias[n + i];
+          }
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            const uint4 u = pack8_half(v + g * 8);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sl + lane * 64 + g * 16), "r"(u.x), "r"(u.y), "r"(u.z), "r"(u.w) : "memory");
+          }
+          __syncwarp();
+          int sg = 0;
+          while (sg + 1 < q.n_seg && n >= q.col0[sg + 1]) ++sg;
+          const int in_seg = n - q.col0[sg];
+          const int head = in_seg / q.head_dim, dim = in_seg - head * q.head_dim;
+          kv16* pool = (kv16*)q.pool[sg];
+          const int nkv_s = q.n_kv[sg];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int r = 8 * i + (lane >> 2), cq = lane & 3;
+            if (slot4[i] >= 0) {
+              uint4 u;
+              asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(u.x), "=r"(u.y), "=r"(u.z), "=r"(u.w) : "r"(sl + r * 64 + cq * 16));
+              const int page = slot4[i] / PAGE_TOKENS, prow = slot4[i] - page * PAGE_TOKENS;
+              *reinterpret_cast<uint4*>(pool + (((size_t)page * nkv_s + head) * PAGE_TOKENS + prow) * q.head_dim + dim + 8 * cq) = u;
+            }
+          }
+          __syncwarp();
         }
       } else {
         epilogue_tile<EPI, BN>(p, tmem_acc, m, w.n0, m < p.M);
