@@ -159,15 +159,21 @@ def run_reference(args):
     full = wl.prompts(name, seed=0)
     n = min(REF_SAMPLE_TOKENS, int(full.lengths[0]))
     sample = wl.Prompts(full.seq(0)[:n].copy(), np.array([n], np.int32))
-    for _ in range(args.warmup):
+    # One oracle step on the 3B-shaped pair takes tens of seconds whatever the sample (its base step converts every
+    # weight to fp64), so the number of steps is bounded to keep the whole run within a few minutes; the line says so.
+    big = pair.base.d_model > 2048
+    warmup, steps = (min(args.warmup, 1), min(args.steps, 3)) if big else (args.warmup, args.steps)
+    for _ in range(warmup):
         time_oracle(pair, W, sample)
-    ts = [time_oracle(pair, W, sample) for _ in range(args.steps)]
+    ts = [time_oracle(pair, W, sample) for _ in range(max(steps, 1))]
     t = sum(ts) / len(ts)
     val = n / t
     desc = f"first {n} tokens of sequence 0 of workload {args.workload}, whole path, fp64 numpy"
+    if (warmup, steps) != (args.warmup, args.steps):
+        desc += f"; {steps} timed steps after {warmup} warm-up (asked for {args.steps} / {args.warmup}: bounded to a few minutes)"
     print(json.dumps({
-        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": warmup, "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64", "data": "synthetic", "config": {"workload": args.workload, "sample": desc},
         "cpu_baseline": {"value": val, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": desc},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -384,7 +390,7 @@ class Bench:
                        "kernels alone and their sum exceeds ms_per_step where the timed schedule overlaps them"),
             "per_class": {c: frac_of(c) for c in alg if per_step[c][0] > 0},
         }
-        t12 = (per_step["aux_gemm"][0] + per_step["aux_attn"][0] + per_step["predictor"][0]) * 1e-3
+        t12 = (per_step["aux_gemm"][0] + per_step["aux_attn"][0] + per_step["predictor"][0] + per_step.get("kv_pred", (0.0, 0))[0]) * 1e-3
         f12 = work["tensor_flops"] / max(t12, 1e-12) / 1e12
         out["tensor_frac_stage12"] = {"achieved_tflops": f12, "frac": f12 / (tpeak / scale), "peak_kind": which,
                                       "frac_of_burst": f12 / (peaks["bf16_tflops"] / scale),
@@ -407,6 +413,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--train-forward", action="store_true",
                     help="also time the training-time forward (base model over the whole prompt on the predicted cache)")
+    ap.add_argument("--prompt-lengths", default="",
+                    help="comma-separated prompt lengths replacing the headline workload's batch (same pair, same token recipe): "
+                         "cut-down shapes for profiler captures")
     ap.add_argument("--opt-flags", type=int, default=0, help="kvp_options.flags: optional kernel variants (see include/kvp.h)")
     ap.add_argument("--decode-steps", type=int, default=16, help="generation steps timed after the TTFT measurement (0 = none)")
     args = ap.parse_args()
@@ -426,6 +435,9 @@ def main():
         head_prompts = wl.sweep_prompts(wl.SWEEP8_LENGTHS[-1], seed=0)
     else:
         head_prompts = wl.prompts(args.workload, seed=0)
+    if args.prompt_lengths:
+        lens = [int(x) for x in args.prompt_lengths.split(",")]
+        head_prompts = wl.custom_prompts(head_pair.base.vocab, lens, seed=0, zipf=args.workload != "c5")
     head = B.measure(args.workload, head_pair, head_prompts, args.steps, args.warmup, full=True)
 
     cpu_baseline = None

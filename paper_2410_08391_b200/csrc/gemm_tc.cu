@@ -37,7 +37,7 @@ template <int BN, int EPI = TC_STORE> struct Tile {
   static constexpr int STAGES = (BN == 256 ? 4 : 6) - (EPI == TC_RESID_NORM ? 1 : 0);
   static constexpr int XS = EPI == TC_PAGED ? 1 : 2;        // 4 KiB slots per epilogue warp
   // epilogues that move every element through shared memory get eight warps (two per tensor-memory lane quarter)
-  static constexpr int EPI_WARPS = (EPI == TC_RESID_NORM || EPI == TC_PAGED) ? 8 : 4;
+  static constexpr int EPI_WARPS = (EPI == TC_RESID_NORM || EPI == TC_PAGED || EPI == TC_QKV || EPI == TC_SWIGLU) ? 8 : 4;
   static constexpr int THREADS = EPI_WARPS == 8 ? N_THREADS_NORM : N_THREADS;
   static constexpr int XRING = (EPI == TC_RESID || EPI == TC_RESID_NORM || EPI == TC_PAGED) ? EPI_WARPS * XS * 4096 : 0;
   static constexpr int A_BYTES = BM * BK * 2, W_BYTES = BN * BK * 2;
@@ -73,22 +73,6 @@ __device__ __forceinline__ uint4 pack8_lo(const float* v) {
 #pragma unroll
   for (int i = 0; i < 8; ++i) r[i] = v[i] - __bfloat162float(__float2bfloat16_rn(v[i]));
   return pack8(r);
-}
-// 32 values as cache elements (halves, saturating)
-__device__ __forceinline__ void store32_kv(kv16* dst, const float* v, int n_valid) {
-#pragma unroll
-  for (int g = 0; g < 4; ++g)
-    if (g * 8 < n_valid) {
-      uint4 u;
-      uint32_t* w = &u.x;
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const __half2 h = __floats2half2_rn(fminf(fmaxf(v[g * 8 + 2 * i], -65504.f), 65504.f),
-                                            fminf(fmaxf(v[g * 8 + 2 * i + 1], -65504.f), 65504.f));
-        w[i] = *reinterpret_cast<const uint32_t*>(&h);
-      }
-      *reinterpret_cast<uint4*>(dst + g * 8) = u;
-    }
 }
 __device__ __forceinline__ void store32_bf16(bf16* dst, const float* v, int n_valid) {
 #pragma unroll
@@ -167,54 +151,27 @@ struct Sched {
   }
 };
 
-__device__ __forceinline__ void red_add4(float* dst, float a, float b, float c, float d) {
-  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
-}
-
 // ---- epilogues: one thread owns one output row of the tile ---------------------------------
+// `part` of `n_parts`: the warps that share a lane quarter take turns over the blocks of 32 columns (TC_QKV: over the heads)
 template <int EPI, int BN>
-__device__ __forceinline__ void epilogue_tile(const Params& p, uint32_t tmem_acc, int m, int n0, bool row_ok) {
+__device__ __forceinline__ void epilogue_tile(const Params& p, uint32_t tmem_acc, int m, int n0, bool row_ok, int part, int n_parts) {
   // tmem_acc already carries this warp's lane quarter in its upper half
-  if (EPI == TC_STORE || EPI == TC_RESID || EPI == TC_PAGED) {
-    int slot = -1;
-    if (EPI == TC_PAGED && row_ok) slot = p.paged.tok_slot[m];
+  if (EPI == TC_STORE) {
 #pragma unroll 1
-    for (int c = 0; c < BN; c += 32) {
+    for (int c = part * 32; c < BN; c += 32 * n_parts) {
       int n = n0 + c;
       int n_valid = p.N - n;
       if (n_valid <= 0) break;           // uniform over the warp
       float v[32];
       tmem_ld32(tmem_acc + c, v);
       tmem_ld_wait();
-      if (!row_ok) continue;
-      if (EPI == TC_STORE) {
-        store32_bf16(p.C + (size_t)m * p.ldc + n, v, n_valid);
-      } else if (EPI == TC_RESID) {
-        float* x = p.X + (size_t)m * p.ldx + n;
-#pragma unroll
-        for (int g = 0; g < 8; ++g)
-          if (g * 4 < n_valid) red_add4(x + 4 * g, v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
-      } else {
-        if (slot < 0) continue;
-        const PagedOut& q = p.paged;
-        int s = 0;
-        while (s + 1 < q.n_seg && n >= q.col0[s + 1]) ++s;
-        int cc = n - q.col0[s];
-        int head = cc / q.head_dim, dim = cc - head * q.head_dim;
-        if (q.bias) {
-#pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] += q.bias[n + i];
-        }
-        int page = slot / PAGE_TOKENS, row = slot - page * PAGE_TOKENS;
-        kv16* dst = (kv16*)q.pool[s] + (((size_t)page * q.n_kv[s] + head) * PAGE_TOKENS + row) * q.head_dim + dim;
-        store32_kv(dst, v, n_valid);
-      }
+      if (row_ok) store32_bf16(p.C + (size_t)m * p.ldc + n, v, n_valid);
     }
   } else if (EPI == TC_SWIGLU) {
     // every 128 columns of the tile: [0, 64) gate rows, [64, 128) the matching up rows
     const float rinv = (p.ss_in && row_ok) ? rsqrtf(p.ss_in[m] / (float)p.K + p.rms_eps) : 1.f;
 #pragma unroll 1
-    for (int c = 0; c < BN / 2; c += 32) {
+    for (int c = part * 32; c < BN / 2; c += 32 * n_parts) {
       int grp = c >> 6, cc = c & 63;
       int n = ((n0 + grp * 128) >> 1) + cc;
       int n_valid = p.ffn - n;
@@ -239,7 +196,7 @@ __device__ __forceinline__ void epilogue_tile(const Params& p, uint32_t tmem_acc
     const float2* tab = row_ok ? p.rope_tab + (size_t)p.tok_pos[m] * half : nullptr;
     const float rinv = (p.ss_in && row_ok) ? rsqrtf(p.ss_in[m] / (float)p.K + p.rms_eps) : 1.f;
 #pragma unroll 1
-    for (int h0 = 0; h0 < BN; h0 += p.hd) {
+    for (int h0 = part * p.hd; h0 < BN; h0 += p.hd * n_parts) {
       if (n0 + h0 >= p.N) break;
       // query / key norm: this thread's row of the head is scaled by 1 / rms and the head's gain before RoPE
       const float* gain = (n0 + h0 < p.rot_cols) ? (n0 + h0 < p.q_cols ? p.q_gain : p.k_gain) : nullptr;
@@ -628,7 +585,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           __syncwarp();
         }
       } else {
-        epilogue_tile<EPI, BN>(p, tmem_acc, m, w.n0, m < p.M);
+        epilogue_tile<EPI, BN>(p, tmem_acc, m, w.n0, m < p.M, half, NH);
       }
       tc_fence_before();
       __syncwarp();
