@@ -1,21 +1,25 @@
 // Causal grouped-query attention over a ragged batch on the sm_100a tensor cores.
 //
 // One CTA = 256 consecutive queries of one sequence (two tiles of 128) and one query head.
-// Warp 0 streams K and V tiles of the matching kv head with TMA straight out of the packed
-// [T, q|k|v] projection buffer; both query tiles use them.  Warp 1 issues S = Q K^T and
-// O += P V with tcgen05.mma; S and O of both query tiles live in tensor memory.  Two groups of
-// four warps, one per query tile, own one query row per thread: a thread reads its row of S
-// into registers in one go, keeps the running max / sum in fp32 and writes P as packed bf16
-// back into tensor memory, from where the P V product takes it as its A operand (P never
-// touches shared memory).  head_dim 64: P has columns of its own, so S of the next key tile is
-// computed while the softmax of this one runs; head_dim 128: tensor memory is full (2 x S, 2 x O),
-// P overwrites the first half of its S, and the two query tiles take turns: one tile's softmax
-// runs while the tensor core works on the other tile's P V and next S.
+// Warp 0 streams K and V tiles (128 keys) of the matching kv head with TMA straight out of the
+// packed [T, q|k|v] projection buffer, K and V through rings of their own (the K tile of the next
+// S product is wanted long before the V tile of this P V product); both query tiles use them.
+// S = Q K^T and O += P V run on tcgen05.mma with S, P and O in tensor memory.  Two groups of four
+// warps, one per query tile, own one query row per thread: a thread copies its row of S into
+// registers in one go (which frees the S columns at once), keeps the running max / sum in fp32
+// and writes P as packed 16-bit values into tensor-memory columns of its own, from where the P V
+// product takes it as its A operand (P never touches shared memory).  So S of the next key tile
+// is computed while the softmax of this one runs, and a group never waits for its own products.
+//   head_dim 64: every tile has its S, P and O columns (2 x (128 + 64 + 64) = 512); one warp
+//     issues the products of both tiles.
+//   head_dim 128: the two O take half of tensor memory, so both tiles share ONE S buffer, used in
+//     turns (S0(0), S1(0), S0(1), ...), and each has an issuing warp of its own.
+// The issuing warps are event loops: whichever product has its inputs is issued, all 32 lanes
+// running the loop so that its state stays warp-uniform and one elected lane issuing.
 // O is accumulated by the tensor core itself and only touched when a row's maximum has grown
 // by more than 2^8 since the exponent offset was last fixed; then the group rescales its O in
-// tensor memory (tcgen05.ld / st).  While one group computes exponentials the tensor core works
-// for the other.  Key tiles above the diagonal are skipped; tiles touching it are masked.
-// Work is ordered so that, over the whole batch, CTAs with the most key tiles start first.
+// tensor memory (tcgen05.ld / st).  Key tiles above the diagonal are skipped; tiles touching it
+// are masked.  Work is ordered so that, over the whole batch, CTAs with the most key tiles start first.
 #include <math.h>
 
 #include "attn_tc.h"
@@ -25,20 +29,24 @@ namespace {
 using namespace tcp;
 
 constexpr int BQ = 128;                 // queries per tile; a CTA has two tiles
-constexpr int N_THREADS = 320;          // warps: 0 TMA, 1 MMA, 2-5 tile 0, 6-9 tile 1
-constexpr int MAX_STAGES = 4;
+constexpr int N_THREADS = 384;          // warps: 0 TMA, 1 / 2 issuers of tile 0 / 1, 3 idle, 4-7 softmax of tile 0, 8-11 of tile 1
 constexpr float RESCALE_LOG2 = 8.f;     // tolerated growth of a row maximum before O is rescaled
 
 template <int HD> struct Cfg {
   static constexpr int BKV = 128;                       // keys per tile
-  static constexpr int STAGES = HD == 64 ? 4 : 2;       // K/V tile pairs in flight (32 / 64 KiB each)
+  static constexpr int K_STAGES = HD == 64 ? 4 : 3;     // K tiles in flight (16 / 32 KiB each)
+  static constexpr int V_STAGES = HD == 64 ? 4 : 2;     // V tiles in flight
   static constexpr int Q_BYTES = BQ * HD * 2;
   static constexpr int KV_BYTES = BKV * HD * 2;         // a K or a V tile
-  static constexpr int SMEM = 2 * Q_BYTES + STAGES * 2 * KV_BYTES + 1024 + 256;
-  // tensor-memory columns: S of tile g, O of tile g, P of tile g (packed bf16: 64 columns for 128 keys)
-  static constexpr int S_COL = 0, O_COL = 256;
-  static constexpr bool P_ALIASES_S = HD == 128;
-  static constexpr int P_COL = P_ALIASES_S ? 0 : 384, P_STRIDE = P_ALIASES_S ? 128 : 64;
+  static constexpr int SMEM = 2 * Q_BYTES + (K_STAGES + V_STAGES) * KV_BYTES + 1024 + 256;
+  // Tensor-memory columns.  head_dim 64: S of tile g, O of tile g, P of tile g (packed 16-bit: 64 columns for 128 keys).
+  // head_dim 128: the two O take half of the 512 columns, so both query tiles share ONE S buffer (a group copies its S
+  // into registers at once, then the buffer is free for the other group) and each has P columns of its own.
+  static constexpr bool S_SHARED = HD == 128;
+  static constexpr bool TWO_ISSUERS = HD == 128;      // one issuing warp per query tile, or one for both
+  static constexpr int S_COL0 = 0, S_STRIDE = S_SHARED ? 0 : 128;
+  static constexpr int P_COL0 = S_SHARED ? 128 : 384, P_STRIDE = 64;
+  static constexpr int O_COL0 = 256, O_STRIDE = HD;
 };
 
 __device__ __forceinline__ float fast_exp2(float x) {
@@ -59,13 +67,33 @@ __device__ __forceinline__ uint64_t desc_mnmajor(uint32_t addr, uint32_t lbo) {
   return lo | (hi << 32);
 }
 
-// D += A B with A taken from tensor memory (row i of A in lane i, two 16-bit elements per 32-bit column)
-__device__ __forceinline__ void tc_mma_bf16_ta(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+// one lane of a converged warp
+__device__ __forceinline__ bool elect_one() {
+  uint32_t is_leader;
+  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(is_leader));
+  return is_leader != 0;
+}
+// D (+)= A B.  The matrix descriptors of one tile differ only in the start-address field (low word), so they are passed
+// as two words and the issuing loop only adds to the low one.  mma_ts: A from tensor memory (row i of A in lane i, two
+// 16-bit elements per 32-bit column).
+template <bool ACC>
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi, uint32_t idesc) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "mov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\t"
+      "setp.ne.b32 p, %6, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "n"(ACC ? 1 : 0)
+      : "memory");
+}
+template <bool ACC>
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "n"(ACC ? 1 : 0)
       : "memory");
 }
 
@@ -84,34 +112,39 @@ template <int HD, bool F16>
 __global__ void __launch_bounds__(N_THREADS, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kv, const Params p) {
   using C = Cfg<HD>;
-  constexpr int BKV = C::BKV, QB = C::Q_BYTES, KB = C::KV_BYTES, NBOX = HD / 64, STAGES = C::STAGES;
+  constexpr int BKV = C::BKV, QB = C::Q_BYTES, KB = C::KV_BYTES, NBOX = HD / 64, KS = C::K_STAGES, VS = C::V_STAGES;
   constexpr int KV_BOX = BKV * 128;     // bytes of one 64-column box of a K or V tile
   extern __shared__ uint8_t smem_raw[];
   pdl_trigger();
   if (threadIdx.x == 32) { prefetch_tensormap(&map_q); prefetch_tensormap(&map_kv); }
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  const uint32_t sQ = smem_u32(smem), sKV = sQ + 2 * QB;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 2 * QB + STAGES * 2 * KB);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 9);
+  const uint32_t sQ = smem_u32(smem), sK = sQ + 2 * QB, sV = sK + KS * KB;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 2 * QB + (KS + VS) * KB);
+  constexpr int N_BARS = 2 * KS + 2 * VS + 9;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + N_BARS);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const uint32_t bar_base = smem_u32(bars);
-  auto kv_full = [&](int s) { return bar_base + 8u * s; };
-  auto kv_empty = [&](int s) { return bar_base + 8u * (STAGES + s); };
-  auto s_full = [&](int g) { return bar_base + 8u * (2 * STAGES + g); };
-  auto s_free = [&](int g) { return bar_base + 8u * (2 * STAGES + 2 + g); };
-  auto p_ready = [&](int g) { return bar_base + 8u * (2 * STAGES + 4 + g); };
-  auto pv_done = [&](int g) { return bar_base + 8u * (2 * STAGES + 6 + g); };
-  const uint32_t q_full = bar_base + 8u * (2 * STAGES + 8);
+  auto k_full = [&](int s) { return bar_base + 8u * s; };
+  auto k_empty = [&](int s) { return bar_base + 8u * (KS + s); };
+  auto v_full = [&](int s) { return bar_base + 8u * (2 * KS + s); };
+  auto v_empty = [&](int s) { return bar_base + 8u * (2 * KS + VS + s); };
+  constexpr int B0 = 2 * KS + 2 * VS;
+  auto s_full = [&](int g) { return bar_base + 8u * (B0 + g); };
+  auto s_free = [&](int g) { return bar_base + 8u * (B0 + 2 + g); };
+  auto p_ready = [&](int g) { return bar_base + 8u * (B0 + 4 + g); };
+  auto pv_done = [&](int g) { return bar_base + 8u * (B0 + 6 + g); };
+  const uint32_t q_full = bar_base + 8u * (B0 + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(kv_full(s), 1); mbar_init(kv_empty(s), 1); }
+    // a K (V) stage goes back to the loader when BOTH query tiles are through with it: one arrival per issuer warp
+    for (int s = 0; s < KS; ++s) { mbar_init(k_full(s), 1); mbar_init(k_empty(s), C::TWO_ISSUERS ? 2 : 1); }
+    for (int s = 0; s < VS; ++s) { mbar_init(v_full(s), 1); mbar_init(v_empty(s), C::TWO_ISSUERS ? 2 : 1); }
     for (int g = 0; g < 2; ++g) { mbar_init(s_full(g), 1); mbar_init(s_free(g), 4); mbar_init(p_ready(g), 4); mbar_init(pv_done(g), 1); }
     mbar_init(q_full, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  // tensor memory: S of tile g at column 128 g, O of tile g at column 256 + HD g, P: see Cfg
   if (warp == 1) tmem_alloc(smem_u32(tmem_slot), 512);
   tc_fence_before();
   __syncthreads();
@@ -128,7 +161,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   n_kv[1] = (p.tiles == 2 && q0 + BQ < L) ? (min(L, q0 + 2 * BQ) + BKV - 1) / BKV : 0;
   const int n_max = max(n_kv[0], n_kv[1]);
 
-
   if (warp == 0) {
     if (lane == 0) {
       bool ok = true;
@@ -138,99 +170,140 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 #pragma unroll
         for (int x = 0; x < NBOX; ++x) tma_load_2d(sQ + g * QB + x * 16384, &map_q, head * HD + x * 64, base + q0 + g * BQ, q_full);
       const int kcol = (p.nq + kvh) * HD, vcol = (p.nq + p.nkv + kvh) * HD;
-      int stage = 0; uint32_t phase = 0;
-      for (int j = 0; j < n_max && ok; ++j) {
-        ok = mbar_wait(kv_empty(stage), phase ^ 1u, abort_flag, p.status);
-        if (!ok) break;
-        const uint32_t sk = sKV + stage * 2 * KB, sv = sk + KB;
-        mbar_expect_tx(kv_full(stage), 2 * KB);
+      // An issuer per tile: K tile j + 1 is wanted (for the next S) before V tile j (for this P V), and loads go out in
+      // that order; one issuer: K and V of a tile together (their stages also come back together).
+      auto load_k = [&](int j) {
+        const int st = j % KS;
+        if (!mbar_wait(k_empty(st), ((j / KS) & 1u) ^ 1u, abort_flag, p.status)) return false;
+        mbar_expect_tx(k_full(st), KB);
 #pragma unroll
-        for (int x = 0; x < NBOX; ++x) {
-          tma_load_2d(sk + x * KV_BOX, &map_kv, kcol + x * 64, base + j * BKV, kv_full(stage));
-          tma_load_2d(sv + x * KV_BOX, &map_kv, vcol + x * 64, base + j * BKV, kv_full(stage));
-        }
-        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        for (int x = 0; x < NBOX; ++x) tma_load_2d(sK + st * KB + x * KV_BOX, &map_kv, kcol + x * 64, base + j * BKV, k_full(st));
+        return true;
+      };
+      if (C::TWO_ISSUERS) ok = load_k(0);
+      for (int j = 0; j < n_max && ok; ++j) {
+        if (!C::TWO_ISSUERS) ok = load_k(j);
+        else if (j + 1 < n_max) ok = load_k(j + 1);
+        if (!ok) break;
+        const int st = j % VS;
+        ok = mbar_wait(v_empty(st), ((j / VS) & 1u) ^ 1u, abort_flag, p.status);
+        if (!ok) break;
+        mbar_expect_tx(v_full(st), KB);
+#pragma unroll
+        for (int x = 0; x < NBOX; ++x) tma_load_2d(sV + st * KB + x * KV_BOX, &map_kv, vcol + x * 64, base + j * BKV, v_full(st));
       }
       if (!ok) drain_after_abort();
     }
-  } else if (warp == 1) {
-    if (lane == 0) {
-      // S = Q K^T: M = 128 queries, N = BKV keys, both operands K-major over head_dim
-      const uint32_t fmt_mask = F16 ? ~((7u << 7) | (7u << 10)) : ~0u;       // operand format fields: 0 = IEEE half
-      const uint32_t idesc_s = idesc_bf16(BQ, BKV) & fmt_mask;
-      // O += P V: A = P (K-major over keys), B = V as stored [key][dim] = MN-major, N = head_dim
-      const uint32_t idesc_pv = (idesc_bf16(BQ, HD) & fmt_mask) | (1u << 16);
-      auto issue_s = [&](int g, int stage) {
-        const uint32_t sk = sKV + stage * 2 * KB;
+  } else if (warp == 1 || (warp == 2 && C::TWO_ISSUERS)) {
+    // Issuer of the tensor-core instructions: one warp per query tile (head_dim 128) or one warp for both (head_dim 64).
+    // All 32 lanes run this loop, so that addresses, descriptors and loop state stay warp-uniform; one elected lane issues
+    // each instruction.
+    const int g_lo = C::TWO_ISSUERS ? warp - 1 : 0, g_hi = C::TWO_ISSUERS ? warp - 1 : 1;
+    // S = Q K^T: M = 128 queries, N = BKV keys, both operands K-major over head_dim
+    const uint32_t fmt_mask = F16 ? ~((7u << 7) | (7u << 10)) : ~0u;       // operand format fields: 0 = IEEE half
+    const uint32_t idesc_s = idesc_bf16(BQ, BKV) & fmt_mask;
+    // O += P V: A = P (K-major over keys), B = V as stored [key][dim] = MN-major, N = head_dim
+    const uint32_t idesc_pv = (idesc_bf16(BQ, HD) & fmt_mask) | (1u << 16);
+    const uint64_t dq0 = desc_kmajor(sQ), dk0 = desc_kmajor(sK), dv0 = desc_mnmajor(sV, KV_BOX);
+    const uint32_t dq_lo = (uint32_t)dq0, dk_lo = (uint32_t)dk0, dv_lo = (uint32_t)dv0;
+    const uint32_t dk_hi = (uint32_t)(dk0 >> 32), dv_hi = (uint32_t)(dv0 >> 32);      // Q and K share the high word
+    auto poll = [&](uint32_t bar, uint32_t parity) { return __all_sync(0xffffffffu, mbar_poll(bar, parity)); };
+    bool ok = __all_sync(0xffffffffu, mbar_wait(q_full, 0, abort_flag, p.status));
+    // Event loop: S of the next key tile and P V of the oldest tile not yet multiplied are issued as soon as their own
+    // inputs are there, in whichever order that happens.  ts / tp = next S / P V tile of a query tile; tk / tv = next key
+    // tile it does NOT use, whose stage still has to be handed back on its behalf.
+    int ts[2] = {0, 0}, tp[2] = {0, 0}, tk[2] = {n_kv[0], n_kv[1]}, tv[2] = {n_kv[0], n_kv[1]};
+    int released = 0;                   // one issuer for both tiles: key tiles whose stages have been handed back
+    uint32_t idle = 0;
+    auto pending = [&](int g) { return tp[g] < n_kv[g] || (C::TWO_ISSUERS && (tk[g] < n_max || tv[g] < n_max)); };
+    while (ok && (pending(g_lo) || pending(g_hi))) {
+      bool progress = false;
 #pragma unroll
-        for (int kk = 0; kk < HD / 16; ++kk)
-          tc_mma_bf16(tmem_base + g * 128, desc_kmajor(sQ + g * QB + (kk >> 2) * 16384 + (kk & 3) * 32),
-                      desc_kmajor(sk + (kk >> 2) * KV_BOX + (kk & 3) * 32), idesc_s, kk > 0 ? 1u : 0u);
-        tc_commit(s_full(g));
-      };
-      bool ok = mbar_wait(q_full, 0, abort_flag, p.status);
-      if (ok) ok = mbar_wait(kv_full(0), 0, abort_flag, p.status);
-      if (ok) {
-        tc_fence_after();
-        for (int g = 0; g < 2; ++g) if (n_kv[g] > 0) issue_s(g, 0);
-      }
-      // Event loop: whichever of the two groups has something ready gets it issued, so a group never
-      // waits behind the other one's softmax.  js = next S tile, jp = next P V product of a group.
-      int js[2] = {1, 1}, jp[2] = {0, 0};
-      int released = 0;                 // key tiles whose stage has been handed back to the loader
-      uint32_t idle = 0;
-      while (ok && (jp[0] < n_kv[0] || jp[1] < n_kv[1])) {
-        bool progress = false;
+      for (int g = 0; g < 2; ++g) {
+        if (g < g_lo || g > g_hi) continue;
+        const int n = n_kv[g], n_other = n_kv[g ^ 1];
+        const uint32_t tS = tmem_base + C::S_COL0 + g * C::S_STRIDE, tP = tmem_base + C::P_COL0 + g * C::P_STRIDE;
+        const uint32_t tO = tmem_base + C::O_COL0 + g * C::O_STRIDE;
+        auto issue_s = [&]() {
+          if (ts[g] < n) {
+            const int t = ts[g];
+            // the S columns are free once their last user has copied them into registers
+            bool ready = t == 0 || poll(s_free(g), (t - 1) & 1u);
+            if (C::S_SHARED && ready) {       // uses of the shared buffer alternate: S0(0), S1(0), S0(1), S1(1), ...
+              if (g == 1) { if (t < n_other) ready = poll(s_free(0), t & 1u); }
+              else if (t > 0 && t - 1 < n_other) ready = poll(s_free(1), (t - 1) & 1u);
+            }
+            const int ks = t % KS;
+            if (ready && poll(k_full(ks), (t / KS) & 1u)) {
+              tc_fence_after();
+              const uint32_t aq = dq_lo + g * (QB >> 4), bq = dk_lo + ks * (KB >> 4);
+              if (elect_one()) mma_ss<false>(tS, aq, dk_hi, bq, dk_hi, idesc_s);
 #pragma unroll
-        for (int g = 0; g < 2; ++g) {
-          if (jp[g] < n_kv[g] && mbar_poll(p_ready(g), jp[g] & 1)) {
-            tc_fence_after();
-            const uint32_t sv = sKV + (jp[g] % STAGES) * 2 * KB + KB;
-#pragma unroll
-            for (int kk = 0; kk < BKV / 16; ++kk)      // 16 keys = 8 packed columns of P per step
-              tc_mma_bf16_ta(tmem_base + C::O_COL + g * HD, tmem_base + C::P_COL + g * C::P_STRIDE + kk * 8,
-                             desc_mnmajor(sv + kk * 2048, KV_BOX), idesc_pv, (jp[g] > 0 || kk > 0) ? 1u : 0u);
-            tc_commit(pv_done(g));
-            ++jp[g];
-            progress = true;
+              for (int kk = 1; kk < HD / 16; ++kk)
+                if (elect_one()) mma_ss<true>(tS, aq + (kk >> 2) * (16384 >> 4) + (kk & 3) * 2, dk_hi, bq + (kk >> 2) * (KV_BOX >> 4) + (kk & 3) * 2, dk_hi, idesc_s);
+              if (elect_one()) { tc_commit(s_full(g)); if (C::TWO_ISSUERS) tc_commit(k_empty(ks)); }
+              ++ts[g];
+              progress = true;
+            }
           }
-          // S of the next key tile: its K tile has landed, and the columns are free: with P in columns of its own once
-          // the group holds the previous S in registers; where P overwrites S, once the P V product that reads it has
-          // been issued (the tensor core executes in issue order)
-          if (js[g] < n_kv[g] && (C::P_ALIASES_S ? jp[g] >= js[g] : mbar_poll(s_free(g), (js[g] - 1) & 1)) &&
-              mbar_poll(kv_full(js[g] % STAGES), (js[g] / STAGES) & 1)) {
-            tc_fence_after();
-            issue_s(g, js[g] % STAGES);
-            ++js[g];
-            progress = true;
+        };
+        auto issue_pv = [&]() {
+          if (tp[g] < ts[g]) {
+            const int t = tp[g], vs = t % VS;
+            if (poll(p_ready(g), t & 1u) && poll(v_full(vs), (t / VS) & 1u)) {
+              tc_fence_after();
+              const uint32_t bv = dv_lo + vs * (KB >> 4);
+              if (t > 0) { if (elect_one()) mma_ts<true>(tO, tP, bv, dv_hi, idesc_pv); }
+              else { if (elect_one()) mma_ts<false>(tO, tP, bv, dv_hi, idesc_pv); }
+#pragma unroll
+              for (int kk = 1; kk < BKV / 16; ++kk)      // 16 keys = 8 packed columns of P per step
+                if (elect_one()) mma_ts<true>(tO, tP + kk * 8, bv + kk * (2048 >> 4), dv_hi, idesc_pv);
+              if (elect_one()) { tc_commit(pv_done(g)); if (C::TWO_ISSUERS) tc_commit(v_empty(vs)); }
+              ++tp[g];
+              progress = true;
+            }
           }
-        }
-        // a stage goes back to the loader once every group that uses its tile has issued S and P V on it
-        while (released < n_max && (n_kv[0] <= released || jp[0] > released) && (n_kv[1] <= released || jp[1] > released)) {
-          tc_commit(kv_empty(released % STAGES));
-          ++released;
+        };
+        // one issuer for both tiles: P V first (it is what the tile's next softmax waits for); an issuer per tile: S first
+        if (C::TWO_ISSUERS) { issue_s(); issue_pv(); } else { issue_pv(); issue_s(); }
+        // (a stage's barrier is only asked about the tile that follows the last one seen on it: parity waits are ambiguous beyond that)
+        if (C::TWO_ISSUERS && ts[g] >= n && tk[g] < n_max && poll(k_full(tk[g] % KS), (tk[g] / KS) & 1u)) {
+          if (lane == 0) mbar_arrive(k_empty(tk[g] % KS));
+          ++tk[g];
           progress = true;
         }
-        if (progress) {
-          idle = 0;
-        } else if (++idle > SPIN_LIMIT) {
-          *abort_flag = 1;
-          dev_flag(p.status, DEV_TIMEOUT);
-          ok = false;
-        } else if ((idle & 63u) == 63u) {
-          if (*abort_flag) ok = false;
+        if (C::TWO_ISSUERS && tp[g] >= n && tv[g] < n_max && poll(v_full(tv[g] % VS), (tv[g] / VS) & 1u)) {
+          if (lane == 0) mbar_arrive(v_empty(tv[g] % VS));
+          ++tv[g];
+          progress = true;
         }
       }
-      if (!ok) drain_after_abort();
+      if (!C::TWO_ISSUERS) {
+        // a K / V stage pair goes back to the loader once every query tile that uses its key tile has issued P V on it
+        while (released < n_max && (n_kv[0] <= released || tp[0] > released) && (n_kv[1] <= released || tp[1] > released)) {
+          if (elect_one()) { tc_commit(k_empty(released % KS)); tc_commit(v_empty(released % VS)); }
+          ++released;
+        }
+      }
+      if (progress) {
+        idle = 0;
+      } else if (++idle > SPIN_LIMIT) {
+        if (lane == 0) { *abort_flag = 1; dev_flag(p.status, DEV_TIMEOUT); }
+        ok = false;
+      } else if ((idle & 63u) == 63u) {
+        if (__any_sync(0xffffffffu, *abort_flag != 0)) ok = false;
+      }
     }
-  } else {
-    const int g = (warp - 2) >> 2;              // query tile of this warp's group
+    if (!ok && lane == 0) drain_after_abort();
+    __syncwarp();
+  } else if (warp >= 4) {
+    const int g = (warp - 4) >> 2;              // query tile of this warp's group
     const int quarter = warp & 3;               // tensor-memory lane quarter this warp may access
     const int r = quarter * 32 + lane;          // row of the query tile owned by this thread
     const int qs = q0 + g * BQ, q_pos = qs + r;
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
-    const uint32_t tS = tmem_base + lane_off + C::S_COL + g * 128, tO = tmem_base + lane_off + C::O_COL + g * HD;
-    const uint32_t tP = tmem_base + lane_off + C::P_COL + g * C::P_STRIDE;
+    const uint32_t tS = tmem_base + lane_off + C::S_COL0 + g * C::S_STRIDE, tO = tmem_base + lane_off + C::O_COL0 + g * C::O_STRIDE;
+    const uint32_t tP = tmem_base + lane_off + C::P_COL0 + g * C::P_STRIDE;
     const float c = p.scale_log2e;
     const int n = n_kv[g];
     float m_ref = -INFINITY, l = 0.f;
