@@ -97,6 +97,14 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_
       : "memory");
 }
 
+// 32 lanes x 128 columns of fp32 in one instruction: thread i of the warp gets lane (row) i, register j = column j.
+__device__ __forceinline__ void tmem_ld128(uint32_t taddr, float* v) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x128.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63, %64, %65, %66, %67, %68, %69, %70, %71, %72, %73, %74, %75, %76, %77, %78, %79, %80, %81, %82, %83, %84, %85, %86, %87, %88, %89, %90, %91, %92, %93, %94, %95, %96, %97, %98, %99, %100, %101, %102, %103, %104, %105, %106, %107, %108, %109, %110, %111, %112, %113, %114, %115, %116, %117, %118, %119, %120, %121, %122, %123, %124, %125, %126, %127}, [%128];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63]), "=r"(r[64]), "=r"(r[65]), "=r"(r[66]), "=r"(r[67]), "=r"(r[68]), "=r"(r[69]), "=r"(r[70]), "=r"(r[71]), "=r"(r[72]), "=r"(r[73]), "=r"(r[74]), "=r"(r[75]), "=r"(r[76]), "=r"(r[77]), "=r"(r[78]), "=r"(r[79]), "=r"(r[80]), "=r"(r[81]), "=r"(r[82]), "=r"(r[83]), "=r"(r[84]), "=r"(r[85]), "=r"(r[86]), "=r"(r[87]), "=r"(r[88]), "=r"(r[89]), "=r"(r[90]), "=r"(r[91]), "=r"(r[92]), "=r"(r[93]), "=r"(r[94]), "=r"(r[95]), "=r"(r[96]), "=r"(r[97]), "=r"(r[98]), "=r"(r[99]), "=r"(r[100]), "=r"(r[101]), "=r"(r[102]), "=r"(r[103]), "=r"(r[104]), "=r"(r[105]), "=r"(r[106]), "=r"(r[107]), "=r"(r[108]), "=r"(r[109]), "=r"(r[110]), "=r"(r[111]), "=r"(r[112]), "=r"(r[113]), "=r"(r[114]), "=r"(r[115]), "=r"(r[116]), "=r"(r[117]), "=r"(r[118]), "=r"(r[119]), "=r"(r[120]), "=r"(r[121]), "=r"(r[122]), "=r"(r[123]), "=r"(r[124]), "=r"(r[125]), "=r"(r[126]), "=r"(r[127])
+               : "r"(taddr) : "memory");
+}
+
 struct Params {
   const int* cu; const int2* sched;     // sched[i] = (sequence, first query of the pair of tiles)
   int nq, nkv;
@@ -314,8 +322,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       if (!ok) break;
       tc_fence_after();
       float s[BKV];
-#pragma unroll
-      for (int cc = 0; cc < BKV; cc += 32) tmem_ld32(tS + cc, s + cc);
+      tmem_ld128(tS, s);
       tmem_ld_wait();
       tc_fence_before();
       __syncwarp();
@@ -333,14 +340,18 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         mx[2] = fmax3(mx[2], s[i + 4], s[i + 5]); mx[3] = fmax3(mx[3], s[i + 6], s[i + 7]);
       }
       const float mt = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-      if (j > 0) {     // the previous P V product has read P and finished writing O
-        ok = mbar_wait(pv_done(g), (j - 1) & 1, abort_flag, p.status);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        tc_fence_after();
-      }
+      // The previous P V product must have read P and finished writing O before P is overwritten or O rescaled.  The
+      // exponentials do not depend on it: the wait sits in front of the first P store (and of the rare rescale).
+      bool pv_seen = j == 0;
       const bool need = mt > m_ref && (m_ref == -INFINITY || (mt - m_ref) * c > RESCALE_LOG2);
       if (__any_sync(0xffffffffu, need)) {
+        if (!pv_seen) {
+          ok = mbar_wait(pv_done(g), (j - 1) & 1, abort_flag, p.status);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          tc_fence_after();
+          pv_seen = true;
+        }
         const float alpha = (need && m_ref != -INFINITY) ? fast_exp2((m_ref - mt) * c) : 1.f;
         if (j > 0) {
 #pragma unroll 1
@@ -382,8 +393,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           rs2[0] = __fadd2_rn(rs2[0], x[0]); rs2[1] = __fadd2_rn(rs2[1], x[1]);
           rs2[0] = __fadd2_rn(rs2[0], x[2]); rs2[1] = __fadd2_rn(rs2[1], x[3]);
         }
-        tmem_st32(tP + hf * 32, reinterpret_cast<const float*>(pk));
+        if (hf == 0 && !pv_seen) {
+          ok = mbar_wait(pv_done(g), (j - 1) & 1, abort_flag, p.status);
+          ok = __all_sync(0xffffffffu, ok);
+          tc_fence_after();
+        }
+        if (ok) tmem_st32(tP + hf * 32, reinterpret_cast<const float*>(pk));
       }
+      if (!ok) break;
       tmem_st_wait();
       l += (rs2[0].x + rs2[0].y) + (rs2[1].x + rs2[1].y);
       tc_fence_before();
