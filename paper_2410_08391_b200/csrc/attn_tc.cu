@@ -44,6 +44,9 @@ template <int HD> struct Cfg {
   // into registers at once, then the buffer is free for the other group) and each has P columns of its own.
   static constexpr bool S_SHARED = HD == 128;
   static constexpr bool TWO_ISSUERS = HD == 128;      // one issuing warp per query tile, or one for both
+  // head_dim 64 is bound by the exp unit (one exponential per 2 x 64 MACs): one pair of exponentials in eight is computed on the
+  // FMA pipe instead (+5 %; larger shares, and any share at head_dim 128, cost more issue slots than they save)
+  static constexpr bool FMA_EXP2 = HD == 64;
   static constexpr int S_COL0 = 0, S_STRIDE = S_SHARED ? 0 : 128;
   static constexpr int P_COL0 = S_SHARED ? 128 : 384, P_STRIDE = 64;
   static constexpr int O_COL0 = 256, O_STRIDE = HD;
@@ -53,6 +56,21 @@ __device__ __forceinline__ float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+// 2^x for a pair on the FMA pipe: x = n + f with n = round(x), |f| <= 1/2; a cubic for 2^f (relative error 7.5e-5),
+// n added into the exponent field.  x <= 127; anything below -126 (masked scores included) gives 2^-126.
+__device__ __forceinline__ float2 exp2_fma(float2 x) {
+  x.x = fmaxf(x.x, -126.f); x.y = fmaxf(x.y, -126.f);
+  const float2 magic = make_float2(12582912.f, 12582912.f);          // 1.5 * 2^23: the sum's low mantissa bits hold round(x)
+  const float2 r = __fadd2_rn(x, magic);
+  const float2 n = __fadd2_rn(r, make_float2(-12582912.f, -12582912.f));
+  const float2 f = __ffma2_rn(n, make_float2(-1.f, -1.f), x);
+  float2 p = __ffma2_rn(f, make_float2(0.0551714076f, 0.0551714076f), make_float2(0.2426107455f, 0.2426107455f));
+  p = __ffma2_rn(p, f, make_float2(0.6932609900f, 0.6932609900f));
+  p = __ffma2_rn(p, f, make_float2(0.9999280967f, 0.9999280967f));
+  p.x = __int_as_float(__float_as_int(p.x) + (__float_as_int(r.x) << 23));
+  p.y = __int_as_float(__float_as_int(p.y) + (__float_as_int(r.y) << 23));
+  return p;
 }
 __device__ __forceinline__ float fmax3(float a, float b, float c) {
   float d;
@@ -381,7 +399,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
             x[q] = __ffma2_rn(make_float2(s[k0 + 2 * q], s[k0 + 2 * q + 1]), c2, nmc2);     // two scaled scores per instruction
-            x[q].x = fast_exp2(x[q].x); x[q].y = fast_exp2(x[q].y);                      // exp2(-inf) = 0
+            if (C::FMA_EXP2 && ((g8 * 4 + q) & 7) == 7) x[q] = exp2_fma(x[q]);
+            else { x[q].x = fast_exp2(x[q].x); x[q].y = fast_exp2(x[q].y); }             // exp2(-inf) = 0
             if (F16) {                                                                    // key 2i in the low half of column i
               const __half2 h2 = __floats2half2_rn(x[q].x, x[q].y);
               pk[g8 * 4 + q] = *reinterpret_cast<const uint32_t*>(&h2);
