@@ -147,7 +147,7 @@ void launch_build_index(const LaunchCtx&, const int* cu_host /*[B+1]*/, int batc
 void launch_embed(const LaunchCtx&, const int* tokens, const int* gather_idx, int n_rows,
                   const void* table, int vocab, int d, float* x);
 void launch_rmsnorm(const LaunchCtx&, const float* x, const float* gain, float eps, int rows, int d,
-                    void* out, int out_dtype, void* out_lo = nullptr);
+                    void* out, int out_dtype, void* out_lo = nullptr, bool out_half = false);
 // fp32 projection output [rows, n_heads*hd] -> RoPE on the first n_heads_rot heads -> run dtype
 // `out` (row stride ld_out) and, for heads >= lo_head_begin, the bf16 lo part in `out_lo`.
 // With q_gain / k_gain (fp32 [head_dim], or null): heads < n_q_heads are RMS-normalised with q_gain and the

@@ -91,6 +91,7 @@ struct Params {
   float* X; int ldx;
   bf16* C_lo; int ld_lo; int lo_col_begin;
   int lo_is_half;        // C_lo receives the whole value as an IEEE half instead of the bf16 remainder
+  int h_is_half;         // H is written as IEEE halves
   int c_is_half;         // TC_QKV: C itself is written as IEEE halves (attention with half operands)
   int f16_operands;      // A and W hold IEEE halves (both operands of one MMA have the same type)
   int rot_cols; int hd;
@@ -478,7 +479,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           __syncwarp();                            // the slot has been read back by every lane
 #pragma unroll
           for (int g = 0; g < 4; ++g) {
-            const uint4 hi = pack8(v + g * 8);
+            const uint4 hi = p.h_is_half ? pack8_half(v + g * 8) : pack8(v + g * 8);
             asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sl + lane * 64 + g * 16), "r"(hi.x), "r"(hi.y), "r"(hi.z), "r"(hi.w) : "memory");
             if (p.H_lo) {
               const uint4 lo = pack8_lo(v + g * 8);
@@ -694,7 +695,7 @@ cudaError_t launch_gemm_tc(const TcGemm& g, int* status, cudaStream_t st, int64_
   p.rot_cols = g.rot_cols; p.hd = g.hd; p.rope_tab = g.rope_tab; p.tok_pos = g.tok_pos; p.ffn = g.ffn; p.paged = g.paged;
   p.H = g.H; p.H_lo = g.H_lo; p.ldh = g.ldh; p.gain_next = g.gain_next; p.ss_out = g.ss_out;
   p.ss_in = g.ss_in; p.rms_eps = g.rms_eps;
-  p.lo_is_half = g.lo_is_half; p.f16_operands = g.f16_operands; p.c_is_half = g.c_is_half;
+  p.lo_is_half = g.lo_is_half; p.f16_operands = g.f16_operands; p.c_is_half = g.c_is_half; p.h_is_half = g.h_is_half;
   const int tiles = ((g.M + BM - 1) / BM) * ((g.N + bn - 1) / bn);
   const long long kblocks = (long long)tiles * ((g.K + BK - 1) / BK);
   int grid = stream_k ? (int)(kblocks < g.n_sm ? kblocks : g.n_sm) : (tiles < g.n_sm ? tiles : g.n_sm);

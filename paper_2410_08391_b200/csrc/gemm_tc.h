@@ -35,7 +35,8 @@ struct TcGemm {
   // TC_QKV / TC_SWIGLU with ss_in: the accumulator rows are scaled by rsqrt(ss_in[m] / K + rms_eps).
   bf16* H; bf16* H_lo; int ldh; const float* gain_next; float* ss_out;
   const float* ss_in; float rms_eps;
-  int lo_is_half;                  // TC_QKV: C_lo receives the whole value as an IEEE half (not the bf16 remainder)
+  int lo_is_half;                             // TC_QKV: C_lo receives the whole value as an IEEE half (not the bf16 remainder)
+  int h_is_half;                              // TC_RESID with H: H is written as IEEE halves (then without H_lo)
   int c_is_half;                   // TC_QKV: C is written as IEEE halves (for an attention that takes half operands)
   int f16_operands;                // A and W hold IEEE halves instead of bf16 (same 2 bytes; both operands alike)
   int n_sm;

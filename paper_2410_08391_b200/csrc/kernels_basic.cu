@@ -135,12 +135,14 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restr
   }
 }
 
+// out_half: the 16-bit output is written as IEEE halves (and no remainder)
 void launch_rmsnorm(const LaunchCtx& ctx, const float* x, const float* gain, float eps, int rows, int d, void* out,
-                    int out_dtype, void* out_lo) {
+                    int out_dtype, void* out_lo, bool out_half) {
   if (rows == 0) return;
   LAUNCH_COUNT(ctx);
   int grid = (rows + 7) / 8;
-  if (out_dtype == 0) launch_overlapped(rmsnorm_kernel<float>, dim3(grid), dim3(256), 0, ctx.st, x, gain, eps, rows, d, (float*)out, (float*)nullptr);
+  if (out_dtype != 0 && out_half) launch_overlapped(rmsnorm_kernel<kv16>, dim3(grid), dim3(256), 0, ctx.st, x, gain, eps, rows, d, (kv16*)out, (kv16*)nullptr);
+  else if (out_dtype == 0) launch_overlapped(rmsnorm_kernel<float>, dim3(grid), dim3(256), 0, ctx.st, x, gain, eps, rows, d, (float*)out, (float*)nullptr);
   else launch_overlapped(rmsnorm_kernel<bf16>, dim3(grid), dim3(256), 0, ctx.st, x, gain, eps, rows, d, (bf16*)out, (bf16*)out_lo);
 }
 

@@ -87,7 +87,7 @@ void plan_model(ModelPlan& p, const kvp_model_cfg* m, int es, bool bf16_mode, si
   }
 }
 
-void add_model_slots(kvp_handle* h, const char* prefix, const ModelPlan& p, int n_live_layers, bool with_head) {
+void add_model_slots(kvp_handle* h, const char* prefix, const ModelPlan& p, int n_live_layers, bool with_head, const std::vector<uint8_t>* qkv_half = nullptr) {
   int dt = h->opt.dtype;
   auto name = [&](int l, const char* leaf) { char b[96]; snprintf(b, sizeof b, "%s.L%d.%s", prefix, l, leaf); return std::string(b); };
   h->slots[std::string(prefix) + ".embed"] = PackSlot{p.embed, p.vocab, p.d, dt, RowMap{0, 0, 0, 0}};
@@ -99,9 +99,10 @@ void add_model_slots(kvp_handle* h, const char* prefix, const ModelPlan& p, int 
       h->slots[name(l, "q_norm")] = PackSlot{L.q_norm, 1, L.hd, 0, RowMap{0, 0, 0, 0}};
       h->slots[name(l, "k_norm")] = PackSlot{L.k_norm, 1, L.hd, 0, RowMap{0, 0, 0, 0}};
     }
-    h->slots[name(l, "wq")] = PackSlot{L.wqkv, L.dq, p.d, dt, RowMap{0, 0, 0, 0}};
-    h->slots[name(l, "wk")] = PackSlot{L.wqkv, L.dkv, p.d, dt, RowMap{L.dq, 0, 0, 0}};
-    h->slots[name(l, "wv")] = PackSlot{L.wqkv, L.dkv, p.d, dt, RowMap{L.dq + L.dkv, 0, 0, 0}};
+    const int dq3 = (qkv_half && (*qkv_half)[l]) ? 2 : dt;     // stored as IEEE halves where the projection runs on f16 operands
+    h->slots[name(l, "wq")] = PackSlot{L.wqkv, L.dq, p.d, dq3, RowMap{0, 0, 0, 0}};
+    h->slots[name(l, "wk")] = PackSlot{L.wqkv, L.dkv, p.d, dq3, RowMap{L.dq, 0, 0, 0}};
+    h->slots[name(l, "wv")] = PackSlot{L.wqkv, L.dkv, p.d, dq3, RowMap{L.dq + L.dkv, 0, 0, 0}};
     h->slots[name(l, "wo")] = PackSlot{L.wo, p.d, L.dq, dt, RowMap{0, 0, 0, 0}};
     h->slots[name(l, "w_gate")] = PackSlot{L.wgu, L.ffn, p.d, dt, RowMap{0, L.G, 0, L.ffn}};
     h->slots[name(l, "w_up")] = PackSlot{L.wgu, L.ffn, p.d, dt, RowMap{L.G == 0 ? L.ffn : 0, L.G, 1, L.ffn}};
@@ -460,7 +461,12 @@ kvp_status kvp_create(const kvp_model_cfg* aux, const kvp_model_cfg* base, const
     if (opt->predictor_bias) { g.bk = take((size_t)dout * 4); g.bv = take((size_t)dout * 4); }
   }
   h->packed_bytes = off;
-  add_model_slots(h, "aux", h->aux, j_max + 1, false);
+  // The QKV projection of an auxiliary layer takes f16 operands wherever the tensor-core kernel is sure to run it (the
+  // kernel that does K/V projection and predictor in one reads bf16 weights, so not with that option).
+  h->qkv_half.assign(j_max + 1, 0);
+  for (int j = 0; j <= j_max; ++j)
+    h->qkv_half[j] = bf && (h->aux.L[j].hd == 64 || h->aux.L[j].hd == 128) && h->aux.d % 8 == 0 && !(opt->flags & KVP_OPT_FUSED_KV_PRED);
+  add_model_slots(h, "aux", h->aux, j_max + 1, false, &h->qkv_half);
   add_model_slots(h, "base", h->base, base->n_layers, true);
   for (int j = 0; j <= j_max; ++j) {
     const PredGroup& g = h->groups[j];
@@ -673,8 +679,9 @@ static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int
     const bool last = (j == h->j_max);   // only K and V of the last mapped layer are needed
     const bool qkv_fused = fused_in[2 * j] != 0, gu_fused = fused_in[2 * j + 1] != 0;
     const bool next_fused = !last && fused_in[2 * (j + 1)] != 0;
+    const bool qkv_half = h->qkv_half[j] != 0;
     if (!qkv_fused)
-      KVP_TIMED(KVP_CLASS_OTHER, launch_rmsnorm(ctx, x, (const float*)(P + L.attn_norm), A.eps, T, A.d, hbuf, h->opt.dtype, h_lo));
+      KVP_TIMED(KVP_CLASS_OTHER, launch_rmsnorm(ctx, x, (const float*)(P + L.attn_norm), A.eps, T, A.d, hbuf, h->opt.dtype, qkv_half ? nullptr : h_lo, qkv_half));
     // predictor of this layer: K_hat_i = K_A,j FK_i^T, V_hat_i = V_A,j FV_i^T for every base layer i with j_i = j
     const PredGroup& pg = h->groups[j];
     const bool half_path = pg.half_path;
@@ -715,6 +722,7 @@ static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int
     tq.C_lo = (bf16*)kv_lo; tq.ld_lo = 2 * L.dkv; tq.lo_col_begin = q_heads * L.hd;
     tq.rot_cols = (q_heads + L.nkv) * L.hd; tq.hd = L.hd; tq.rope_tab = rope_tab; tq.tok_pos = tok_pos;
     if (fused_kv) { tq.C_lo = nullptr; tq.rot_cols = q_heads * L.hd; tq.A2 = nullptr; }
+    if (qkv_half) { tq.A2 = nullptr; tq.f16_operands = 1; }      // h and W_qkv are halves: one pass over every column
     const float* qn = A.qk_norm ? (const float*)(P + L.q_norm) : nullptr;
     const float* kn = A.qk_norm ? (const float*)(P + L.k_norm) : nullptr;
     tq.q_gain = qn; tq.k_gain = kn; tq.q_cols = q_heads * L.hd; tq.eps = A.eps;
@@ -730,6 +738,7 @@ static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int
     } else if (!try_tc(h, ctx, tq, KVP_CLASS_AUX_GEMM, &tc_err)) {
       if (half_path && h->groups[j].n_seg > 0) return fail(h, KVP_ERR_CUDA, "internal: half-precision predictor input planned for a projection the tensor-core kernel refuses");
       if (qkv_fused) return fail(h, KVP_ERR_CUDA, "internal: fused norm planned for a projection the tensor-core kernel refuses");
+      if (qkv_half) return fail(h, KVP_ERR_CUDA, "internal: half-precision operands planned for a projection the tensor-core kernel refuses");
       GemmArgs g{};
       g.A = hbuf; g.lda = A.d; g.M = T; g.K = A.d;
       g.A2 = h_lo; g.lda2 = A.d;
@@ -834,7 +843,9 @@ static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int
     td.A = (const bf16*)act; td.lda = L.ffn; td.W = (const bf16*)(P + L.wd); td.ldw = L.ffn; td.M = T; td.N = A.d; td.K = L.ffn;
     td.epi = TC_RESID; td.X = x; td.ldx = A.d;
     if (next_fused) {    // the down projection completes x: it also writes the next layer's QKV operand (hi + lo parts)
-      td.H = (bf16*)hbuf; td.H_lo = (bf16*)h_lo; td.ldh = A.d; td.gain_next = (const float*)(P + A.L[j + 1].attn_norm);
+      const bool next_half = h->qkv_half[j + 1] != 0;     // ... or as halves, where that projection takes f16 operands
+      td.H = (bf16*)hbuf; td.H_lo = next_half ? nullptr : (bf16*)h_lo; td.h_is_half = next_half ? 1 : 0;
+      td.ldh = A.d; td.gain_next = (const float*)(P + A.L[j + 1].attn_norm);
       td.ss_out = norm_ss + (size_t)(2 * (j + 1)) * T;
     }
     if (!try_tc(h, ctx, td, KVP_CLASS_AUX_GEMM, &tc_err)) {

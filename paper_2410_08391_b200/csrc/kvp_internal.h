@@ -41,7 +41,7 @@ struct PredGroup {
 struct PackSlot {
   size_t off;      // destination byte offset of row 0 / element 0
   int rows, cols;  // expected source shape (rows = 1 for vectors)
-  int dst_dtype;   // 0 f32, 1 bf16
+  int dst_dtype;   // 0 f32, 1 bf16, 2 IEEE half
   RowMap map;
 };
 
@@ -57,6 +57,10 @@ struct kvp_handle {
   kvp_options opt;
   int es;                               // element size of the run dtype
   std::vector<PredGroup> groups;        // one per auxiliary layer 0..j_max
+  // Auxiliary layers whose QKV projection takes its operands as IEEE halves: the normalised input is written once as
+  // halves (11 significant bits) instead of a bf16 value plus remainder, W_q / W_k / W_v are stored as halves, and the
+  // K / V columns need no second pass.
+  std::vector<uint8_t> qkv_half;
   std::unordered_map<std::string, PackSlot> slots;
   std::vector<std::string> req_prefill, req_decode_extra;
   std::unordered_set<std::string> loaded;
