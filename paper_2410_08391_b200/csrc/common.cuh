@@ -24,6 +24,12 @@ template <class T> __device__ __forceinline__ T from_f(float v);
 template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
 template <> __device__ __forceinline__ bf16 from_f<bf16>(float v) { return __float2bfloat16_rn(v); }
 template <> __device__ __forceinline__ kv16 from_f<kv16>(float v) { return __float2half_rn(fminf(fmaxf(v, -65504.f), 65504.f)); }
+// two values as packed IEEE halves (lo in the low 16 bits), saturating at the largest finite half: one instruction
+__device__ __forceinline__ uint32_t half2_sat(float lo, float hi) {
+  uint32_t d;
+  asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
 // the two cache elements held by a 32-bit word (element 2i in the low half)
 __device__ __forceinline__ float kv_lo(uint32_t u) { return __low2float(*reinterpret_cast<const __half2*>(&u)); }
 __device__ __forceinline__ float kv_hi(uint32_t u) { return __high2float(*reinterpret_cast<const __half2*>(&u)); }

@@ -61,10 +61,7 @@ __device__ __forceinline__ uint4 pack8_half(const float* v) {
   uint4 u;
   uint32_t* w = &u.x;
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const __half2 h = __floats2half2_rn(fminf(fmaxf(v[2 * i], -65504.f), 65504.f), fminf(fmaxf(v[2 * i + 1], -65504.f), 65504.f));
-    w[i] = *reinterpret_cast<const uint32_t*>(&h);
-  }
+  for (int i = 0; i < 4; ++i) w[i] = half2_sat(v[2 * i], v[2 * i + 1]);
   return u;
 }
 // bf16 rounding remainders of 8 values
