@@ -96,6 +96,7 @@ struct Params {
   int ffn;               // SwiGLU: output width
   const float* q_gain; const float* k_gain; int q_cols; float eps;   // TC_QKV: query / key norm (null = off)
   PagedOut paged;
+  int paged_wide;        // TC_PAGED: head_dim and every segment boundary are multiples of 64 (128-byte row pieces)
   // RMSNorm folded into its neighbours.  Producer (TC_RESID with H; every tile owned by one CTA): the epilogue
   // reads the old X (prefetched by TMA), stores X + acc, and also writes the next GEMM's operand
   // H = bf16(X * gain_next) (+ its bf16 remainder H_lo) and adds the row's share of sum X^2 to ss_out[m].  Consumer (TC_QKV / TC_SWIGLU with ss_in): every row of the accumulator is scaled by
@@ -541,46 +542,94 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const PagedOut& q = p.paged;
         const uint32_t sl = xring;
         const int row_base = w.m0 + quarter * 32;
-        int slot4[4];              // cache slots of the four rows this lane writes in the read-back pattern
+        if (p.paged_wide) {
+          // head_dim and every segment boundary are multiples of 64: 64 columns at a time (half a head_dim-128 row or a
+          // whole head_dim-64 row of a token), staged as 32 rows x 128 bytes (16-byte pieces swizzled by the row) and
+          // stored as 4 rows x 128 bytes per instruction.
+          int slot8[8];            // cache slots of the eight rows this lane writes in the read-back pattern
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const int mr = row_base + 8 * i + (lane >> 2);
-          slot4[i] = mr < p.M ? q.tok_slot[mr] : -1;
-        }
+          for (int i = 0; i < 8; ++i) {
+            const int mr = row_base + 4 * i + (lane >> 3);
+            slot8[i] = mr < p.M ? q.tok_slot[mr] : -1;
+          }
 #pragma unroll 1
-        for (int c = half * 32; c < BN; c += 32 * NH) {
-          const int n = w.n0 + c;
-          if (n >= p.N) break;
-          float v[32];
-          tmem_ld32(tmem_acc + c, v);
-          tmem_ld_wait();
-          if (q.bias) {
+          for (int c = half * 64; c < BN; c += 64 * NH) {
+            const int n = w.n0 + c;
+            if (n >= p.N) break;
+            float v[64];
+            tmem_ld32(tmem_acc + c, v);
+            tmem_ld32(tmem_acc + c + 32, v + 32);
+            tmem_ld_wait();
+            if (q.bias) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) v[i] += q.bias[n + i];
-          }
+              for (int i = 0; i < 64; ++i) v[i] += q.bias[n + i];
+            }
 #pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            const uint4 u = pack8_half(v + g * 8);
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sl + lane * 64 + g * 16), "r"(u.x), "r"(u.y), "r"(u.z), "r"(u.w) : "memory");
+            for (int g = 0; g < 8; ++g) {
+              const uint4 u = pack8_half(v + g * 8);
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sl + lane * 128 + ((g ^ (lane & 7)) << 4)), "r"(u.x), "r"(u.y), "r"(u.z), "r"(u.w) : "memory");
+            }
+            __syncwarp();
+            int sg = 0;
+            while (sg + 1 < q.n_seg && n >= q.col0[sg + 1]) ++sg;
+            const int in_seg = n - q.col0[sg];
+            const int head = in_seg / q.head_dim, dim = in_seg - head * q.head_dim;
+            kv16* pool = (kv16*)q.pool[sg];
+            const int nkv_s = q.n_kv[sg];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const int r = 4 * i + (lane >> 3), cq = lane & 7;
+              if (slot8[i] >= 0) {
+                uint4 u;
+                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(u.x), "=r"(u.y), "=r"(u.z), "=r"(u.w) : "r"(sl + r * 128 + ((cq ^ (r & 7)) << 4)));
+                const int page = slot8[i] / PAGE_TOKENS, prow = slot8[i] - page * PAGE_TOKENS;
+                *reinterpret_cast<uint4*>(pool + (((size_t)page * nkv_s + head) * PAGE_TOKENS + prow) * q.head_dim + dim + 8 * cq) = u;
+              }
+            }
+            __syncwarp();
           }
-          __syncwarp();
-          int sg = 0;
-          while (sg + 1 < q.n_seg && n >= q.col0[sg + 1]) ++sg;
-          const int in_seg = n - q.col0[sg];
-          const int head = in_seg / q.head_dim, dim = in_seg - head * q.head_dim;
-          kv16* pool = (kv16*)q.pool[sg];
-          const int nkv_s = q.n_kv[sg];
+        } else {
+          int slot4[4];              // cache slots of the four rows this lane writes in the read-back pattern
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
-            const int r = 8 * i + (lane >> 2), cq = lane & 3;
-            if (slot4[i] >= 0) {
-              uint4 u;
-              asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(u.x), "=r"(u.y), "=r"(u.z), "=r"(u.w) : "r"(sl + r * 64 + cq * 16));
-              const int page = slot4[i] / PAGE_TOKENS, prow = slot4[i] - page * PAGE_TOKENS;
-              *reinterpret_cast<uint4*>(pool + (((size_t)page * nkv_s + head) * PAGE_TOKENS + prow) * q.head_dim + dim + 8 * cq) = u;
-            }
+            const int mr = row_base + 8 * i + (lane >> 2);
+            slot4[i] = mr < p.M ? q.tok_slot[mr] : -1;
           }
-          __syncwarp();
+#pragma unroll 1
+          for (int c = half * 32; c < BN; c += 32 * NH) {
+            const int n = w.n0 + c;
+            if (n >= p.N) break;
+            float v[32];
+            tmem_ld32(tmem_acc + c, v);
+            tmem_ld_wait();
+            if (q.bias) {
+#pragma unroll
+              for (int i = 0; i < 32; ++i) v[i] += q.bias[n + i];
+            }
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+              const uint4 u = pack8_half(v + g * 8);
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sl + lane * 64 + g * 16), "r"(u.x), "r"(u.y), "r"(u.z), "r"(u.w) : "memory");
+            }
+            __syncwarp();
+            int sg = 0;
+            while (sg + 1 < q.n_seg && n >= q.col0[sg + 1]) ++sg;
+            const int in_seg = n - q.col0[sg];
+            const int head = in_seg / q.head_dim, dim = in_seg - head * q.head_dim;
+            kv16* pool = (kv16*)q.pool[sg];
+            const int nkv_s = q.n_kv[sg];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const int r = 8 * i + (lane >> 2), cq = lane & 3;
+              if (slot4[i] >= 0) {
+                uint4 u;
+                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(u.x), "=r"(u.y), "=r"(u.z), "=r"(u.w) : "r"(sl + r * 64 + cq * 16));
+                const int page = slot4[i] / PAGE_TOKENS, prow = slot4[i] - page * PAGE_TOKENS;
+                *reinterpret_cast<uint4*>(pool + (((size_t)page * nkv_s + head) * PAGE_TOKENS + prow) * q.head_dim + dim + 8 * cq) = u;
+              }
+            }
+            __syncwarp();
+          }
         }
       } else {
         epilogue_tile<EPI, BN>(p, tmem_acc, m, w.n0, m < p.M, half, NH);
@@ -692,6 +741,11 @@ cudaError_t launch_gemm_tc(const TcGemm& g, int* status, cudaStream_t st, int64_
   p.rot_cols = g.rot_cols; p.hd = g.hd; p.rope_tab = g.rope_tab; p.tok_pos = g.tok_pos; p.ffn = g.ffn; p.paged = g.paged;
   p.H = g.H; p.H_lo = g.H_lo; p.ldh = g.ldh; p.gain_next = g.gain_next; p.ss_out = g.ss_out;
   p.ss_in = g.ss_in; p.rms_eps = g.rms_eps;
+  p.paged_wide = 0;
+  if (g.epi == TC_PAGED) {
+    p.paged_wide = g.paged.head_dim % 64 == 0 && g.N % 64 == 0;
+    for (int sg = 0; sg <= g.paged.n_seg; ++sg) if (g.paged.col0[sg] % 64) p.paged_wide = 0;
+  }
   p.lo_is_half = g.lo_is_half; p.f16_operands = g.f16_operands; p.c_is_half = g.c_is_half; p.h_is_half = g.h_is_half;
   const int tiles = ((g.M + BM - 1) / BM) * ((g.N + bn - 1) / bn);
   const long long kblocks = (long long)tiles * ((g.K + BK - 1) / BK);
