@@ -35,11 +35,11 @@ constexpr int TC_RESID_NORM = 100;                         // internal: TC_RESID
 template <int BN, int EPI = TC_STORE> struct Tile {
   // the fused-norm residual epilogue needs a deeper prefetch ring for the old values of X: one operand stage less
   static constexpr int STAGES = (BN == 256 ? 4 : 6) - (EPI == TC_RESID_NORM ? 1 : 0);
-  static constexpr int XS = EPI == TC_PAGED ? 1 : 2;        // 4 KiB slots per epilogue warp
+  static constexpr int XS = (EPI == TC_PAGED || EPI == TC_QKV) ? 1 : 2;        // 4 KiB slots per epilogue warp
   // epilogues that move every element through shared memory get eight warps (two per tensor-memory lane quarter)
   static constexpr int EPI_WARPS = (EPI == TC_RESID_NORM || EPI == TC_PAGED || EPI == TC_QKV || EPI == TC_SWIGLU) ? 8 : 4;
   static constexpr int THREADS = EPI_WARPS == 8 ? N_THREADS_NORM : N_THREADS;
-  static constexpr int XRING = (EPI == TC_RESID || EPI == TC_RESID_NORM || EPI == TC_PAGED) ? EPI_WARPS * XS * 4096 : 0;
+  static constexpr int XRING = (EPI == TC_RESID || EPI == TC_RESID_NORM || EPI == TC_PAGED || EPI == TC_QKV) ? EPI_WARPS * XS * 4096 : 0;
   static constexpr int A_BYTES = BM * BK * 2, W_BYTES = BN * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + W_BYTES;    // 48 KiB / 32 KiB
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + XRING + 1024 /*align*/ + 512 /*barriers*/;
@@ -153,7 +153,7 @@ struct Sched {
 // ---- epilogues: one thread owns one output row of the tile ---------------------------------
 // `part` of `n_parts`: the warps that share a lane quarter take turns over the blocks of 32 columns (TC_QKV: over the heads)
 template <int EPI, int BN>
-__device__ __forceinline__ void epilogue_tile(const Params& p, uint32_t tmem_acc, int m, int n0, bool row_ok, int part, int n_parts) {
+__device__ __forceinline__ void epilogue_tile(const Params& p, uint32_t tmem_acc, int m, int n0, bool row_ok, int part, int n_parts, uint32_t slot, int row_base) {
   // tmem_acc already carries this warp's lane quarter in its upper half
   if (EPI == TC_STORE) {
 #pragma unroll 1
@@ -192,6 +192,7 @@ __device__ __forceinline__ void epilogue_tile(const Params& p, uint32_t tmem_acc
     }
   } else {  // TC_QKV: RoPE on columns < rot_cols, hi part to C, lo part of columns >= lo_col_begin to C_lo
     int half = p.hd >> 1;
+    const int lane = threadIdx.x & 31;
     const float2* tab = row_ok ? p.rope_tab + (size_t)p.tok_pos[m] * half : nullptr;
     const float rinv = (p.ss_in && row_ok) ? rsqrtf(p.ss_in[m] / (float)p.K + p.rms_eps) : 1.f;
 #pragma unroll 1
@@ -219,52 +220,56 @@ __device__ __forceinline__ void epilogue_tile(const Params& p, uint32_t tmem_acc
         tmem_ld32(tmem_acc + h0 + half + j, b);
         tmem_ld_wait();
         int n = n0 + h0 + j;
-        if (!row_ok) continue;
-        if (p.ss_in) {
+        if (row_ok) {
+          if (p.ss_in) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) { a[i] *= rinv; b[i] *= rinv; }
-        }
-        if (gain) {
+            for (int i = 0; i < 32; ++i) { a[i] *= rinv; b[i] *= rinv; }
+          }
+          if (gain) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) { a[i] *= rn * gain[j + i]; b[i] *= rn * gain[half + j + i]; }
-        }
-        if (n < p.rot_cols) {
+            for (int i = 0; i < 32; ++i) { a[i] *= rn * gain[j + i]; b[i] *= rn * gain[half + j + i]; }
+          }
+          if (n < p.rot_cols) {
 #pragma unroll
-          for (int i = 0; i < 32; i += 2) {
-            float4 cs = *reinterpret_cast<const float4*>(tab + j + i);   // (cos, sin) of two frequencies
-            float x1 = a[i], x2 = b[i];
-            a[i] = x1 * cs.x - x2 * cs.y; b[i] = x2 * cs.x + x1 * cs.y;
-            x1 = a[i + 1]; x2 = b[i + 1];
-            a[i + 1] = x1 * cs.z - x2 * cs.w; b[i + 1] = x2 * cs.z + x1 * cs.w;
+            for (int i = 0; i < 32; i += 2) {
+              float4 cs = *reinterpret_cast<const float4*>(tab + j + i);   // (cos, sin) of two frequencies
+              float x1 = a[i], x2 = b[i];
+              a[i] = x1 * cs.x - x2 * cs.y; b[i] = x2 * cs.x + x1 * cs.y;
+              x1 = a[i + 1]; x2 = b[i + 1];
+              a[i + 1] = x1 * cs.z - x2 * cs.w; b[i + 1] = x2 * cs.z + x1 * cs.w;
+            }
           }
         }
-        bf16* dst = p.C + (size_t)m * p.ldc + n;
-        if (p.c_is_half) {
+        // A thread owns a ROW here, and 16-byte stores of 32 different rows cost four times the memory transactions of
+        // 64-byte row pieces: the two 32 x 32 blocks (first and second half of the head) go through this warp's
+        // shared-memory slot as 16-bit values (16-byte pieces swizzled by the row) and leave as 8 rows x 64 bytes per store.
+        auto stage_and_store = [&](bool as_half, bool remainder, bf16* base, int ld, int col) {
+          __syncwarp();                        // the slot's previous contents have been read
 #pragma unroll
           for (int g = 0; g < 4; ++g) {
-            *reinterpret_cast<uint4*>(dst + g * 8) = pack8_half(a + g * 8);
-            *reinterpret_cast<uint4*>(dst + half + g * 8) = pack8_half(b + g * 8);
+            const uint32_t off = lane * 64 + ((g ^ ((lane >> 1) & 3)) << 4);
+            const uint4 ua = as_half ? pack8_half(a + g * 8) : (remainder ? pack8_lo(a + g * 8) : pack8(a + g * 8));
+            const uint4 ub = as_half ? pack8_half(b + g * 8) : (remainder ? pack8_lo(b + g * 8) : pack8(b + g * 8));
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(slot + off), "r"(ua.x), "r"(ua.y), "r"(ua.z), "r"(ua.w) : "memory");
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(slot + 2048 + off), "r"(ub.x), "r"(ub.y), "r"(ub.z), "r"(ub.w) : "memory");
           }
-        } else {
-          store32_bf16(dst, a, 32);
-          store32_bf16(dst + half, b, 32);
-        }
-        if (p.C_lo && n >= p.lo_col_begin) {
-          bf16* lo = p.C_lo + (size_t)m * p.ld_lo + (n - p.lo_col_begin);
-          if (p.lo_is_half) {
+          __syncwarp();
 #pragma unroll
-            for (int g = 0; g < 4; ++g) {
-              *reinterpret_cast<uint4*>(lo + g * 8) = pack8_half(a + g * 8);
-              *reinterpret_cast<uint4*>(lo + half + g * 8) = pack8_half(b + g * 8);
-            }
-          } else {
-#pragma unroll
-            for (int g = 0; g < 4; ++g) {
-              *reinterpret_cast<uint4*>(lo + g * 8) = pack8_lo(a + g * 8);
-              *reinterpret_cast<uint4*>(lo + half + g * 8) = pack8_lo(b + g * 8);
+          for (int i = 0; i < 4; ++i) {
+            const int r = 8 * i + (lane >> 2), cq = lane & 3;
+            if (row_base + r < p.M) {
+              const uint32_t off = r * 64 + ((cq ^ ((r >> 1) & 3)) << 4);
+              uint4 ua, ub;
+              asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(ua.x), "=r"(ua.y), "=r"(ua.z), "=r"(ua.w) : "r"(slot + off));
+              asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(ub.x), "=r"(ub.y), "=r"(ub.z), "=r"(ub.w) : "r"(slot + 2048 + off));
+              bf16* dst = base + (size_t)(row_base + r) * ld + col + 8 * cq;
+              *reinterpret_cast<uint4*>(dst) = ua;
+              *reinterpret_cast<uint4*>(dst + half) = ub;
             }
           }
-        }
+        };
+        stage_and_store(p.c_is_half != 0, false, p.C, p.ldc, n);
+        if (p.C_lo && n >= p.lo_col_begin) stage_and_store(p.lo_is_half != 0, p.lo_is_half == 0, p.C_lo, p.ld_lo, n - p.lo_col_begin);
       }
     }
   }
@@ -632,7 +637,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           }
         }
       } else {
-        epilogue_tile<EPI, BN>(p, tmem_acc, m, w.n0, m < p.M, half, NH);
+        epilogue_tile<EPI, BN>(p, tmem_acc, m, w.n0, m < p.M, half, NH, xring, w.m0 + quarter * 32);
       }
       tc_fence_before();
       __syncwarp();
