@@ -30,6 +30,7 @@ CASES = [
     ("t_scaled", [100, 33, 257], "fanin"),
     ("t_scaled", [100, 33, 257], "n002"),
     ("t_bias", [40, 90], "fanin"),
+    ("t_hd32", [150, 37, 1, 64, 65], "fanin"),      # predictor columns leave as 64-byte pieces (segment boundaries at 96)
     # layer-pruned auxiliary model (KVP-LP): same width as the base, square predictor matrices
     ("t_lp", [100, 59, 59, 7], "fanin"),
     ("t_lp", [130], "n002"),

@@ -172,6 +172,10 @@ def pair(name: str) -> PairCfg:
         aux = layerwise_scaled_model(4, 256, 4, 8, 64, 1500, 0.5, 2.0)
         base = layerwise_scaled_model(6, 384, 4, 12, 64, 1500, 0.5, 2.0)
         return PairCfg("t_scaled", aux, base, (0, 0, 1, 1, 2, 3))
+    if name == "t_hd32":      # base head_dim 32 with 3 kv heads: predicted widths (96 per layer) that are no multiples of 64
+        aux = uniform_model(3, 192, 4, 1, 64, 320, 1000)
+        base = uniform_model(4, 256, 6, 3, 32, 448, 1000)
+        return PairCfg("t_hd32", aux, base, (0, 0, 1, 2))
     if name == "t_mha":       # one query head per kv head (head_dim 64)
         aux = uniform_model(2, 192, 3, 3, 64, 320, 1000)
         base = uniform_model(4, 256, 4, 4, 64, 448, 1000)
