@@ -229,11 +229,11 @@ bool step_uses_tc(const kvp_handle* h, int batch) {
 // gate/up row, or as they are), output cleared first unless it is the residual stream.
 void step_proj_tc(kvp_handle* h, const LaunchCtx& ctx, const WsLayout& w, char* ws, int mode, const float* src, int ld_src,
                   int K, int batch, const float* gain, int G, const void* W, int N, float* Y, int ldy, bool clear,
-                  cudaError_t* err) {
+                  cudaError_t* err, const void* next_w = nullptr, size_t next_bytes = 0) {
   bf16* XB = (bf16*)(ws + w.xbt);
   KVP_TIMED(KVP_CLASS_STEP_GEMV, launch_step_prep(ctx, mode, src, ld_src, K, batch, gain, h->base.eps, G, XB, clear ? Y : nullptr, ldy, N));
   TimedScope ts(h, ctx.st, KVP_CLASS_STEP_GEMV);
-  cudaError_t e = launch_step_gemm_tc((const bf16*)W, K, N, K, XB, batch, Y, ldy, h->step_grid_sms, ctx.status, ctx.st, ctx.n_launch);
+  cudaError_t e = launch_step_gemm_tc((const bf16*)W, K, N, K, XB, batch, Y, ldy, h->step_grid_sms, ctx.status, ctx.st, ctx.n_launch, next_w, next_bytes);
   if (e != cudaSuccess && *err == cudaSuccess) *err = e;
 }
 
@@ -251,8 +251,14 @@ void base_layer_step(kvp_handle* h, const LaunchCtx& ctx, int i, const kvp_cache
   // the first step needs q only (keys and values are the predicted ones); generation needs q, k, v
   int n_out = generation ? L.nqkv : L.dq;
   const bool tc = step_uses_tc(h, batch);
+  // every projection names the weights of the one after it (the next layer's queries, or the LM head, after the down projection)
+  const size_t es = (size_t)h->es;
+  const bool last_layer = i + 1 == B.n_layers;
+  const void* w_after = last_layer ? P + B.lm_head : P + B.L[last_layer ? i : i + 1].wqkv;
+  const size_t b_after = last_layer ? (size_t)B.vocab * B.d * es : (size_t)(generation ? B.L[i + 1].nqkv : B.L[i + 1].dq) * B.d * es;
   if (tc)
-    step_proj_tc(h, ctx, w, ws, PREP_NORM, xb, B.d, B.d, batch, (const float*)(P + L.attn_norm), 0, P + L.wqkv, n_out, qkvb, n_out, true, err);
+    step_proj_tc(h, ctx, w, ws, PREP_NORM, xb, B.d, B.d, batch, (const float*)(P + L.attn_norm), 0, P + L.wqkv, n_out, qkvb, n_out, true, err,
+                 P + L.wo, (size_t)B.d * L.dq * es);
   else
     KVP_TIMED(KVP_CLASS_STEP_GEMV, launch_step_gemv(ctx, P + L.wqkv, B.d, n_out, B.d, xb, B.d, batch, qkvb, n_out, GEMV_STORE, 0, 0,
                                                     (const float*)(P + L.attn_norm), B.eps, hb));
@@ -266,9 +272,10 @@ void base_layer_step(kvp_handle* h, const LaunchCtx& ctx, int i, const kvp_cache
                    (float*)(ws + w.part), ab, qn, B.eps, (int*)(ws + w.attn_done)));
   if (tc) {
     float* gub = (float*)(ws + w.gub);
-    step_proj_tc(h, ctx, w, ws, PREP_PLAIN, ab, L.dq, L.dq, batch, nullptr, 0, P + L.wo, B.d, xb, B.d, false, err);
-    step_proj_tc(h, ctx, w, ws, PREP_NORM, xb, B.d, B.d, batch, (const float*)(P + L.ffn_norm), 0, P + L.wgu, 2 * L.ffn, gub, 2 * L.ffn, true, err);
-    step_proj_tc(h, ctx, w, ws, PREP_SWIGLU, gub, 2 * L.ffn, L.ffn, batch, nullptr, L.G, P + L.wd, B.d, xb, B.d, false, err);
+    step_proj_tc(h, ctx, w, ws, PREP_PLAIN, ab, L.dq, L.dq, batch, nullptr, 0, P + L.wo, B.d, xb, B.d, false, err, P + L.wgu, (size_t)2 * L.ffn * B.d * es);
+    step_proj_tc(h, ctx, w, ws, PREP_NORM, xb, B.d, B.d, batch, (const float*)(P + L.ffn_norm), 0, P + L.wgu, 2 * L.ffn, gub, 2 * L.ffn, true, err,
+                 P + L.wd, (size_t)B.d * L.ffn * es);
+    step_proj_tc(h, ctx, w, ws, PREP_SWIGLU, gub, 2 * L.ffn, L.ffn, batch, nullptr, L.G, P + L.wd, B.d, xb, B.d, false, err, w_after, b_after);
     return;
   }
   KVP_TIMED(KVP_CLASS_STEP_GEMV, launch_step_gemv(ctx, P + L.wo, L.dq, B.d, L.dq, ab, L.dq, batch, xb, B.d, GEMV_RESID, 0, 0));

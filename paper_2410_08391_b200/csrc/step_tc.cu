@@ -21,6 +21,7 @@ constexpr int BM = 128, BK = 64;
 constexpr int W_BYTES = BM * BK * 2;
 constexpr int N_THREADS = 192;
 constexpr int SMEM_LIMIT = 220 * 1024;
+constexpr size_t STEP_PREFETCH_MAX = 32u << 20;   // bytes of the next weight matrix asked into L2 (L2 holds 126 MB; this kernel streams through it too)
 
 struct Params {
   int N, K, batch, Bp;
@@ -28,6 +29,10 @@ struct Params {
   int acc_stride;           // tensor-memory columns between the two accumulators
   float* Y; int ldy;
   int* status;
+  // The weights the NEXT projection will stream (null = none): once this kernel has requested all of its own tiles, every CTA
+  // asks for its share of them to be brought into L2, so HBM keeps streaming through this kernel's tail, the operand
+  // preparation and the launch gap.
+  const char* next_w; long long next_bytes;
 };
 
 __device__ __forceinline__ void red_add(float* dst, float v) {
@@ -119,6 +124,14 @@ step_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constan
           }
           tma_load_2d(sw + W_BYTES, &map_x, kb * BK, 0, full_bar(stage));
           if (++stage == S) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (ok && p.next_w) {
+        constexpr long long CHUNK = 64 * 1024;
+        const long long n_chunks = (p.next_bytes + CHUNK - 1) / CHUNK;
+        for (long long c = blockIdx.x; c < n_chunks; c += gridDim.x) {
+          const long long off = c * CHUNK, len = min(CHUNK, p.next_bytes - off) & ~15ll;
+          if (len > 0) bulk_prefetch_l2(p.next_w + off, (uint32_t)len);
         }
       }
       if (!ok) drain_after_abort();
@@ -287,13 +300,15 @@ void launch_step_prep(const LaunchCtx& ctx, int mode, const float* x, int ldx, i
 }
 
 cudaError_t launch_step_gemm_tc(const bf16* W, int ldw, int N, int K, const bf16* XB, int batch, float* Y, int ldy, int n_sm,
-                                int* status, cudaStream_t st, int64_t* n_launch) {
+                                int* status, cudaStream_t st, int64_t* n_launch, const void* next_w, size_t next_bytes) {
   const int Bp = step_tc_rows(batch);
   CUtensorMap mw, mx;
   if (!tc_make_map_bf16(&mw, W, N, K, ldw, BM)) return cudaErrorInvalidValue;
   if (!tc_make_map_bf16(&mx, XB, 2 * Bp, K, K, 2 * Bp)) return cudaErrorInvalidValue;
   Params p{};
   p.N = N; p.K = K; p.batch = batch; p.Bp = Bp; p.Y = Y; p.ldy = ldy; p.status = status;
+  p.next_w = (((uintptr_t)next_w & 15) == 0) ? (const char*)next_w : nullptr;
+  p.next_bytes = (long long)(next_bytes < STEP_PREFETCH_MAX ? next_bytes : STEP_PREFETCH_MAX);
   p.x_bytes = (2 * Bp * BK * 2 + 1023) / 1024 * 1024;
   p.stages = (SMEM_LIMIT - 2048) / (W_BYTES + p.x_bytes);
   if (p.stages > 12) p.stages = 12;

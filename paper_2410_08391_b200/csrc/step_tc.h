@@ -18,5 +18,7 @@ void launch_step_prep(const LaunchCtx&, int mode, const float* x, int ldx, int K
                       int G, bf16* XB, float* zero_ptr, int zero_ld, int zero_n);
 
 // Y[b, n] += sum_k W[n, k] (XB[b, k] + XB[Bp + b, k]) for b < batch, n < N; fp32 atomic adds.
+// next_w / next_bytes: the weight matrix the next projection will read (or null): its first megabytes are asked into L2.
 cudaError_t launch_step_gemm_tc(const bf16* W, int ldw, int N, int K, const bf16* XB, int batch, float* Y, int ldy,
-                                int n_sm, int* status, cudaStream_t st, int64_t* n_launch);
+                                int n_sm, int* status, cudaStream_t st, int64_t* n_launch, const void* next_w = nullptr,
+                                size_t next_bytes = 0);
