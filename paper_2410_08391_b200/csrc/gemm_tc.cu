@@ -92,7 +92,7 @@ struct Params {
   int c_is_half;         // TC_QKV: C itself is written as IEEE halves (attention with half operands)
   int f16_operands;      // A and W hold IEEE halves (both operands of one MMA have the same type)
   int rot_cols; int hd;
-  const float2* rope_tab; const int* tok_pos;
+  const float2* rope_tab; int tab_stride; const int* tok_pos;
   int ffn;               // SwiGLU: output width
   const float* q_gain; const float* k_gain; int q_cols; float eps;   // TC_QKV: query / key norm (null = off)
   PagedOut paged;
@@ -193,7 +193,9 @@ __device__ __forceinline__ void epilogue_tile(const Params& p, uint32_t tmem_acc
   } else {  // TC_QKV: RoPE on columns < rot_cols, hi part to C, lo part of columns >= lo_col_begin to C_lo
     int half = p.hd >> 1;
     const int lane = threadIdx.x & 31;
-    const float2* tab = row_ok ? p.rope_tab + (size_t)p.tok_pos[m] * half : nullptr;
+    // (cos, sin) of two neighbouring frequencies per 16-byte entry, entries of consecutive POSITIONS next to each other: the 32
+    // rows of a warp (consecutive tokens) read 512 contiguous bytes per load
+    const float4* tab = row_ok ? reinterpret_cast<const float4*>(p.rope_tab) + p.tok_pos[m] : nullptr;
     const float rinv = (p.ss_in && row_ok) ? rsqrtf(p.ss_in[m] / (float)p.K + p.rms_eps) : 1.f;
 #pragma unroll 1
     for (int h0 = part * p.hd; h0 < BN; h0 += p.hd * n_parts) {
@@ -232,7 +234,7 @@ __device__ __forceinline__ void epilogue_tile(const Params& p, uint32_t tmem_acc
           if (n < p.rot_cols) {
 #pragma unroll
             for (int i = 0; i < 32; i += 2) {
-              float4 cs = *reinterpret_cast<const float4*>(tab + j + i);   // (cos, sin) of two frequencies
+              const float4 cs = tab[(size_t)((j + i) >> 1) * p.tab_stride];   // (cos, sin) of two frequencies
               float x1 = a[i], x2 = b[i];
               a[i] = x1 * cs.x - x2 * cs.y; b[i] = x2 * cs.x + x1 * cs.y;
               x1 = a[i + 1]; x2 = b[i + 1];
@@ -743,7 +745,7 @@ cudaError_t launch_gemm_tc(const TcGemm& g, int* status, cudaStream_t st, int64_
   p.stream_k = stream_k ? 1 : 0;
   p.C = g.C; p.ldc = g.ldc; p.X = g.X; p.ldx = g.ldx; p.C_lo = g.C_lo; p.ld_lo = g.ld_lo; p.lo_col_begin = g.lo_col_begin;
   p.q_gain = g.q_gain; p.k_gain = g.k_gain; p.q_cols = g.q_cols; p.eps = g.eps;
-  p.rot_cols = g.rot_cols; p.hd = g.hd; p.rope_tab = g.rope_tab; p.tok_pos = g.tok_pos; p.ffn = g.ffn; p.paged = g.paged;
+  p.rot_cols = g.rot_cols; p.hd = g.hd; p.rope_tab = g.rope_tab; p.tab_stride = g.tab_stride; p.tok_pos = g.tok_pos; p.ffn = g.ffn; p.paged = g.paged;
   p.H = g.H; p.H_lo = g.H_lo; p.ldh = g.ldh; p.gain_next = g.gain_next; p.ss_out = g.ss_out;
   p.ss_in = g.ss_in; p.rms_eps = g.rms_eps;
   p.paged_wide = 0;
@@ -759,14 +761,14 @@ cudaError_t launch_gemm_tc(const TcGemm& g, int* status, cudaStream_t st, int64_
   return bn == 256 ? go_epi<256>(g.epi, ma, ma2, mw, mx, p, grid, st) : go_epi<128>(g.epi, ma, ma2, mw, mx, p, grid, st);
 }
 
-// ---- RoPE table: tab[pos][c] = (cos, sin)(pos * theta^(-2c/hd)) -----------------------------
+// ---- RoPE table: entry [c / 2][pos] = (cos, sin)(pos * theta^(-2c/hd)) for c and c + 1 (16 bytes), positions contiguous ----
 __global__ void rope_table_kernel(float2* tab, int n_pos, int half, const __grid_constant__ InvFreq inv) {
   int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n_pos * half) return;
-  int pos = i / half, c = i - pos * half;
+  int c = i / n_pos, pos = i - c * n_pos;
   float s, co;
   rope_sincos(pos, inv.f[c], &s, &co);
-  tab[i] = make_float2(co, s);
+  tab[((size_t)(c >> 1) * n_pos + pos) * 2 + (c & 1)] = make_float2(co, s);
 }
 
 void launch_rope_table(const LaunchCtx& ctx, float2* tab, int n_pos, int hd, float theta) {

@@ -21,7 +21,8 @@ struct TcGemm {
   float* X; int ldx;
   bf16* C_lo; int ld_lo; int lo_col_begin;
   int rot_cols; int hd;
-  const float2* rope_tab;          // [position][hd/2] (cos, sin)
+  const float2* rope_tab;          // [hd/4][position] entries of (cos, sin) of two neighbouring frequencies
+  int tab_stride;                  // positions in the table
   const int* tok_pos;              // [M] position of each row in its sequence
   int ffn;
   // TC_QKV with query / key norm: columns < q_cols are query heads (gain q_gain), the other rotated columns key

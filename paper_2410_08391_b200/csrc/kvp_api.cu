@@ -125,7 +125,7 @@ WsLayout ws_layout(const kvp_handle* h, int64_t Bm, int64_t Tm) {
   w.last_idx = take(Bm * 4);
   w.tok_pos = take(Tm * 4);
   w.tok_slot = take(Tm * 4);
-  w.rope_tab = take(Tm * (size_t)(A.L[0].hd / 2) * 8);
+  w.rope_tab = take(Tm * (size_t)((A.L[0].hd / 2 + 1) & ~1) * 8);     // entries hold two frequencies: an even number of them
   w.x = take(Tm * A.d * 4);
   w.h = take(Tm * A.d * es);
   w.h_lo = take(Tm * A.d * es);
@@ -713,7 +713,7 @@ static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int
     kp.Wkv = (const bf16*)(P + L.wqkv + (size_t)L.dq * A.d * es); kp.ldw = A.d; kp.M = T; kp.K = A.d;
     kp.dkv = L.dkv; kp.hd = L.hd; kp.kv_begin = 0; kp.kv_end = 2;
     if (qkv_fused) { kp.ss_in = norm_ss + (size_t)(2 * j) * T; kp.rms_eps = A.eps; }
-    kp.rope_tab = rope_tab; kp.tok_pos = tok_pos; kp.k_gain = A.qk_norm ? (const float*)(P + L.k_norm) : nullptr; kp.eps = A.eps;
+    kp.rope_tab = rope_tab; kp.tab_stride = cs.max_len; kp.tok_pos = tok_pos; kp.k_gain = A.qk_norm ? (const float*)(P + L.k_norm) : nullptr; kp.eps = A.eps;
     kp.C = (bf16*)qkv; kp.ldc = L.nqkv; kp.k_col = L.dq;
     kp.FK = P + pg.fk; kp.FV = P + pg.fv; kp.n_tot = pg.col0[pg.n_seg]; kp.paged[0] = paged[0]; kp.paged[1] = paged[1];
     kp.n_sm = h->gemm_sms;
@@ -727,7 +727,7 @@ static kvp_status prefill_direct(kvp_handle* h, const int32_t* tokens, const int
     tq.W = (const bf16*)(P + L.wqkv + (size_t)col_begin * A.d * es); tq.ldw = A.d; tq.M = T; tq.N = n_out; tq.K = A.d;
     tq.epi = TC_QKV; tq.C = (bf16*)(qkv + (size_t)col_begin * es); tq.ldc = L.nqkv;
     tq.C_lo = (bf16*)kv_lo; tq.ld_lo = 2 * L.dkv; tq.lo_col_begin = q_heads * L.hd;
-    tq.rot_cols = (q_heads + L.nkv) * L.hd; tq.hd = L.hd; tq.rope_tab = rope_tab; tq.tok_pos = tok_pos;
+    tq.rot_cols = (q_heads + L.nkv) * L.hd; tq.hd = L.hd; tq.rope_tab = rope_tab; tq.tab_stride = cs.max_len; tq.tok_pos = tok_pos;
     if (fused_kv) { tq.C_lo = nullptr; tq.rot_cols = q_heads * L.hd; tq.A2 = nullptr; }
     if (qkv_half) { tq.A2 = nullptr; tq.f16_operands = 1; }      // h and W_qkv are halves: one pass over every column
     const float* qn = A.qk_norm ? (const float*)(P + L.q_norm) : nullptr;
@@ -1063,7 +1063,7 @@ TrainWs train_ws_layout(const kvp_handle* h, int64_t Bm, int64_t Tm) {
   w.last_idx = take(Bm * 4);
   w.tok_pos = take(Tm * 4);
   w.tok_slot = take(Tm * 4);
-  w.rope_tab = take(Tm * (size_t)(B.L[0].hd / 2) * 8);
+  w.rope_tab = take(Tm * (size_t)((B.L[0].hd / 2 + 1) & ~1) * 8);
   w.x = take(Tm * B.d * 4);
   w.h = take(Tm * B.d * es);
   w.h_lo = take(Tm * B.d * es);
@@ -1160,7 +1160,7 @@ extern "C" kvp_status kvp_train_forward(kvp_handle* h, const int32_t* tokens, co
       tq.W = (const bf16*)(P + L.wqkv + (size_t)col_begin * B.d * es); tq.ldw = B.d; tq.M = T; tq.N = n_out; tq.K = B.d;
       tq.epi = TC_QKV; tq.C = (bf16*)(qkv + (size_t)col_begin * es); tq.ldc = L.nqkv;
       tq.C_lo = (bf16*)kv_lo; tq.ld_lo = 2 * L.dkv; tq.lo_col_begin = q_heads * L.hd;
-      tq.rot_cols = (q_heads + L.nkv) * L.hd; tq.hd = L.hd; tq.rope_tab = rope_tab; tq.tok_pos = tok_pos;
+      tq.rot_cols = (q_heads + L.nkv) * L.hd; tq.hd = L.hd; tq.rope_tab = rope_tab; tq.tab_stride = cs.max_len; tq.tok_pos = tok_pos;
       tq.q_gain = qn; tq.k_gain = kn; tq.q_cols = q_heads * L.hd; tq.eps = B.eps;
       if (hp) { tq.c_is_half = 1; tq.C_lo = nullptr; }
       if (!try_tc(h, ctx, tq, KVP_CLASS_OTHER, &tc_err)) {

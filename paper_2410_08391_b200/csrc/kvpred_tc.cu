@@ -35,7 +35,7 @@ struct Params {
   int stages1, slots2, stage1_bytes, a2_bytes;
   int has_lo;
   const float* ss_in; float rms_eps;
-  const float2* rope_tab; const int* tok_pos;
+  const float2* rope_tab; int tab_stride; const int* tok_pos;
   const float* k_gain; float eps;
   bf16* C; int ldc; int k_col;
   PagedOut paged[2];
@@ -257,7 +257,7 @@ kvpred_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
       const int col0 = p.k_col + kv * p.dkv;
       if (kv == 0) {      // keys: (key norm,) RoPE on the pairs (c, c + hd / 2) of every head
         const int half = p.hd >> 1;
-        const float2* tab = p.rope_tab + (size_t)(row_ok ? p.tok_pos[m] : 0) * half;
+        const float4* tab = reinterpret_cast<const float4*>(p.rope_tab) + (row_ok ? p.tok_pos[m] : 0);
 #pragma unroll 1
         for (int h0 = 0; h0 < p.dkv; h0 += p.hd) {
           float rn = rinv;
@@ -286,7 +286,7 @@ kvpred_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             }
 #pragma unroll
             for (int i = 0; i < 32; i += 2) {
-              const float4 cs = *reinterpret_cast<const float4*>(tab + j + i);     // (cos, sin) of two frequencies
+              const float4 cs = tab[(size_t)((j + i) >> 1) * p.tab_stride];     // (cos, sin) of two frequencies
               float x1 = a[i], x2 = b[i];
               a[i] = x1 * cs.x - x2 * cs.y; b[i] = x2 * cs.x + x1 * cs.y;
               x1 = a[i + 1]; x2 = b[i + 1];
@@ -388,7 +388,7 @@ cudaError_t launch_kvpred_tc(const KvPred& g, int* status, cudaStream_t st, int6
   Params p{};
   p.M = g.M; p.K = g.K; p.dkv = g.dkv; p.n_tot = g.n_tot; p.hd = g.hd; p.kv_begin = g.kv_begin; p.kv_end = g.kv_end;
   p.has_lo = g.A_lo != nullptr;
-  p.ss_in = g.ss_in; p.rms_eps = g.rms_eps; p.rope_tab = g.rope_tab; p.tok_pos = g.tok_pos; p.k_gain = g.k_gain; p.eps = g.eps;
+  p.ss_in = g.ss_in; p.rms_eps = g.rms_eps; p.rope_tab = g.rope_tab; p.tab_stride = g.tab_stride; p.tok_pos = g.tok_pos; p.k_gain = g.k_gain; p.eps = g.eps;
   p.C = g.C; p.ldc = g.ldc; p.k_col = g.k_col; p.paged[0] = g.paged[0]; p.paged[1] = g.paged[1]; p.status = status;
   p.a2_bytes = (g.dkv / BK) * A_BYTES;
   p.stage1_bytes = A_BYTES + g.dkv * BK * 2;

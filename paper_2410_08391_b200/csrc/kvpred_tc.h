@@ -10,7 +10,7 @@ struct KvPred {
   int dkv, hd;                       // auxiliary layer's kv width (multiple of 64, <= 384) and head_dim (64 | 128)
   int kv_begin, kv_end;              // which of (0 = K, 1 = V) this launch computes
   const float* ss_in; float rms_eps; // folded RMSNorm: rows scaled by rsqrt(ss_in[m] / K + rms_eps); null = off
-  const float2* rope_tab; const int* tok_pos;
+  const float2* rope_tab; int tab_stride; const int* tok_pos;
   const float* k_gain; float eps;    // key norm gain [hd] or null
   bf16* C; int ldc; int k_col;       // q|k|v buffer of the layer: keys at column k_col, values at k_col + dkv
   const void* FK; const void* FV;    // stacked predictor matrices [n_tot, dkv], IEEE halves
