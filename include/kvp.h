@@ -33,7 +33,7 @@
  *   - Matrices are [out_features, in_features], row-major, dense.
  *   - Reproducibility: some projections add partial sums with fp32 atomic adds, so two runs
  *     on the same inputs agree up to fp32 reassociation (about 1e-6 relative in the fp32
- *     quantities, occasionally one bf16 unit in a stored cache element), not bit for bit.
+ *     quantities, occasionally one unit in the last place of a stored 16-bit cache element), not bit for bit.
  */
 #ifndef KVP_H_
 #define KVP_H_
@@ -103,7 +103,8 @@ typedef struct {
  *   KVP_OPT_SEPARATE_NORM  RMSNorm as a kernel of its own in front of every projection.  By default, wherever every
  *                          output tile of the residual GEMMs belongs to one CTA (calls of some thousand tokens and
  *                          more), RMSNorm is folded into the GEMMs around it: the residual GEMM that completes x also
- *                          writes bf16(x * gain) and the rows' sums of squares, the next GEMM scales its rows by 1 / rms. */
+ *                          writes x * gain as the next GEMM's 16-bit operand and the rows' sums of squares, the next GEMM
+ *                          scales its rows by 1 / rms. */
 enum { KVP_OPT_FUSED_KV_PRED = 1, KVP_OPT_SEPARATE_NORM = 2 };
 
 /* A named tensor handed to kvp_load_weights().  Names:
@@ -266,7 +267,7 @@ kvp_status kvp_decode_step_static(kvp_handle* h, const int32_t* tokens /* dev [b
  *       keys and values (query t sees predicted entries 0..t: "masked cross-attention"):
  *       logits_out = dev fp32 [sum(lengths), vocab], row t = logits after token t (the input of the paper's
  *       base loss L_B); may be NULL, then pass (2) is skipped.
- * The predicted cache is read in the run dtype (bf16 entries in bf16 mode).  The cache and seq_lens are not
+ * The predicted cache is read in its own element type (IEEE halves in KVP_BF16 mode, fp32 in KVP_F32 mode).  The cache and seq_lens are not
  * changed.  workspace: dev, 256-byte aligned, >= kvp_train_workspace_bytes(batch, sum(lengths)) (its own
  * layout: base-model widths for every token).  Launches kernel by kernel on `stream`, no synchronisation.
  * Needs every base tensor including wk / wv.  Errors as kvp_prefill_predict. */
