@@ -30,6 +30,11 @@ using namespace tcp;
 
 constexpr int BQ = 128;                 // queries per tile; a CTA has two tiles
 constexpr int N_THREADS = 384;          // warps: 0 TMA, 1 / 2 issuers of tile 0 / 1, 3 idle, 4-7 softmax of tile 0, 8-11 of tile 1
+// Registers move from the loader / issuer warp group to the two softmax groups once the roles split (setmaxnreg): the
+// kernel is launched with 168 per thread, 128 x REGS_LOW + 256 x REGS_HIGH = 384 x 168.  The launcher refuses the kernel
+// if it was compiled with fewer (the raise would wait for registers that do not exist).
+constexpr int REGS_LAUNCH = 168, REGS_LOW = 56, REGS_HIGH = 224;
+static_assert(128 * REGS_LOW + 256 * REGS_HIGH <= 384 * REGS_LAUNCH, "register split exceeds the launch's registers");
 constexpr float RESCALE_LOG2 = 8.f;     // tolerated growth of a row maximum before O is rescaled
 
 template <int HD> struct Cfg {
@@ -187,6 +192,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   n_kv[1] = (p.tiles == 2 && q0 + BQ < L) ? (min(L, q0 + 2 * BQ) + BKV - 1) / BKV : 0;
   const int n_max = max(n_kv[0], n_kv[1]);
 
+  if (warp < 4) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_LOW));
   if (warp == 0) {
     if (lane == 0) {
       bool ok = true;
@@ -323,6 +329,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     if (!ok && lane == 0) drain_after_abort();
     __syncwarp();
   } else if (warp >= 4) {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS_HIGH));
     const int g = (warp - 4) >> 2;              // query tile of this warp's group
     const int quarter = warp & 3;               // tensor-memory lane quarter this warp may access
     const int r = quarter * 32 + lane;          // row of the query tile owned by this thread
@@ -510,6 +517,14 @@ cudaError_t go(const CUtensorMap& mq, const CUtensorMap& mkv, const Params& p, d
   static bool raised[TC_MAX_DEVICES] = {};
   cudaError_t e = tc_raise_smem_limit(attn_tc_kernel<HD, F16>, Cfg<HD>::SMEM, raised);
   if (e != cudaSuccess) return e;
+  static int regs = 0;                  // a property of the compiled kernel, the same on every device
+  if (regs == 0) {
+    cudaFuncAttributes fa;
+    e = cudaFuncGetAttributes(&fa, attn_tc_kernel<HD, F16>);
+    if (e != cudaSuccess) return e;
+    regs = fa.numRegs;
+  }
+  if (regs < REGS_LAUNCH) return cudaErrorLaunchOutOfResources;
   return launch_overlapped(attn_tc_kernel<HD, F16>, grid, dim3(N_THREADS), Cfg<HD>::SMEM, st, mq, mkv, p);
 }
 }  // namespace
